@@ -1,0 +1,221 @@
+/*
+ * ebrl_actgen -- batched action generation for independently progressing environments on one
+ * NVIDIA B200 (sm_100a), behind a C ABI.
+ *
+ * The operation (paper section 2.1): a diffusion-style action head turns a random tensor into
+ * an action chunk over several denoising steps, conditioned on a representation the backbone
+ * has cached (here: per-environment prefix K/V planes).  Environments are independent and are
+ * served in groups (section 4.2.2); generation runs under an SM quota smaller than the chip
+ * so that other stages can share the GPU (sections 4.2.1 and 4.3.1).
+ *
+ * Per environment e, with action state a in R^{H x A}, prefix planes Kc, Vc in R^{P_e x d} and
+ * step index k_e, the library computes, for k = k_e .. k_end-1 (t_k = k/K):
+ *
+ *     x_h   = W_in a_h + temb(t_k)                                   (h = 0..H-1)
+ *     for each layer l:
+ *         [q|k|v] = W_qkv RMSNorm(x; g1);  x += W_o  concat_heads softmax(q k^T / sqrt(hd)) v
+ *         qc      = W_qc  RMSNorm(x; g2);  x += W_oc concat_heads softmax(qc Kc^T / sqrt(hd)) Vc
+ *         x      += W_2 GELU(W_1 RMSNorm(x; g3))                      (GELU in its erf form)
+ *     v     = W_out RMSNorm(x; g_final) + b_out
+ *     a    += v / K                                                   (explicit Euler)
+ *
+ *     temb(t)_j = sin(temb_scale * t * w_j), temb(t)_{d/2+j} = cos(temb_scale * t * w_j),
+ *     w_j = temb_max_period^(-j/(d/2));   RMSNorm(x; g)_j = g_j x_j / sqrt(mean(x^2) + rms_eps).
+ *
+ * Matrices are row-major [out][in] (y = W x).  Accumulation is always fp32; the action state,
+ * gains and b_out are fp32; matrices and prefix planes are fp32 or bf16 (param_dtype/kv_dtype).
+ *
+ * The result for an environment is a pure function of (weights, its planes, its state, its
+ * step index, the step count): it does not depend on environment ids, on which group the
+ * environment arrives in, on the order inside the group, or on the SM quota.  Results are
+ * bit-identical across those choices.
+ *
+ * Error behaviour: every call returns a status; nothing throws, aborts or traps across this
+ * boundary.  Invalid arguments are detected before anything is enqueued.  Asynchronous
+ * failures (a CUDA error, a bounded device-side wait that ran out) are sticky and are returned
+ * by ebrl_actgen_sync.  There is no CPU fallback: without a usable CUDA device the calls fail.
+ */
+#ifndef EBRL_ACTGEN_H_
+#define EBRL_ACTGEN_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define EBRL_ACTGEN_ABI_VERSION 1u
+
+typedef struct ebrl_actgen *ebrl_actgen_t;
+
+typedef enum {
+    EBRL_OK = 0,
+    EBRL_ERR_INVALID_ARG = 1,   /* bad pointer, size, dtype, step index, duplicate env id ...   */
+    EBRL_ERR_UNSUPPORTED = 2,   /* valid but outside what the kernels cover (see create)        */
+    EBRL_ERR_NOMEM = 3,         /* host or device allocation failed                             */
+    EBRL_ERR_CUDA = 4,          /* a CUDA call or kernel failed; text in last_error             */
+    EBRL_ERR_ENV_BUSY = 5,      /* an env id of this group is in a group not yet synced         */
+    EBRL_ERR_QUOTA = 6,         /* sm_quota outside 0..#SMs                                     */
+    EBRL_ERR_TIMEOUT = 7        /* a bounded device-side wait gave up                           */
+} ebrl_status_t;
+
+typedef enum { EBRL_F32 = 0, EBRL_BF16 = 1 } ebrl_dtype_t;
+
+/* cfg.flags */
+#define EBRL_FLAG_TEST_PULL   1u  /* replace the network by v = b_out - a (integrator check)    */
+#define EBRL_FLAG_GREEN_CTX   2u  /* run under a green context of sm_quota SMs when available   */
+#define EBRL_FLAG_TIMING      4u  /* record per-kernel-class device time (see get_stats)        */
+#define EBRL_FLAG_FORCE_SIMT  8u  /* bf16 models: use the plain-ALU kernels, not tensor cores    */
+
+/* Plain data, copied at create. */
+typedef struct {
+    uint32_t abi_version;        /* EBRL_ACTGEN_ABI_VERSION                                     */
+    int32_t H, A, d;             /* action tokens, action dims, model width                     */
+    int32_t n_layers, n_heads;   /* head_dim = d / n_heads                                      */
+    int32_t mlp_mult;            /* MLP hidden width = mlp_mult * d                             */
+    int32_t K_steps;             /* Euler steps from t = 0 to t = 1                             */
+    int32_t max_prefix_len;      /* upper bound on any P_e                                      */
+    int32_t max_group_envs;      /* upper bound on n_envs of one submit                         */
+    int32_t max_inflight_groups; /* groups that may be submitted before a sync (>= 1)           */
+    int32_t param_dtype;         /* ebrl_dtype_t of the matrices                                */
+    int32_t kv_dtype;            /* ebrl_dtype_t of the prefix planes                           */
+    int32_t kv_layers;           /* 1: one K/V plane pair for all layers; n_layers: per layer   */
+    float rms_eps;               /* 1e-6                                                        */
+    float temb_scale;            /* 1000                                                        */
+    float temb_max_period;       /* 10000                                                       */
+    uint32_t flags;              /* EBRL_FLAG_*                                                 */
+    int32_t device;              /* CUDA device ordinal                                         */
+    uint64_t wait_limit_ns;      /* bound for device-side waits; 0 = default                    */
+} ebrl_actgen_cfg_t;
+
+typedef struct {
+    const float *g1, *g2, *g3;   /* [d] fp32 RMSNorm gains                                      */
+    const void *w_qkv;           /* [3d][d]: rows 0..d-1 Q, d..2d-1 K, 2d..3d-1 V;
+                                    head h = rows h*hd..(h+1)*hd-1 of each third               */
+    const void *w_o;             /* [d][d]   self-attention output projection                   */
+    const void *w_qc;            /* [d][d]   cross-attention query projection                   */
+    const void *w_oc;            /* [d][d]   cross-attention output projection                  */
+    const void *w_1;             /* [mlp_mult*d][d]                                             */
+    const void *w_2;             /* [d][mlp_mult*d]                                             */
+} ebrl_layer_weights_t;
+
+/* Pointers may be host or device memory; everything is copied to the device at create and the
+ * caller's buffers are not referenced afterwards. */
+typedef struct {
+    const void *w_in;            /* [d][A] param_dtype                                          */
+    const void *w_out;           /* [A][d] param_dtype                                          */
+    const float *b_out;          /* [A] fp32                                                    */
+    const float *g_final;        /* [d] fp32                                                    */
+    const ebrl_layer_weights_t *layers;   /* [n_layers]                                         */
+} ebrl_actgen_weights_t;
+
+/* Optional per-submit extension; NULL means the defaults. */
+typedef struct {
+    const int32_t *prefix_len;   /* host [n]; NULL: every P_e = cfg.max_prefix_len              */
+    const int32_t *step_index;   /* host [n], k_e in [0, K); NULL: all 0                        */
+    int32_t n_steps;             /* 0: run every env to step K; s > 0: advance by min(s, K-k_e) */
+} ebrl_submit_ext_t;
+
+/* Kernel classes of the per-class timing (EBRL_FLAG_TIMING). */
+enum { EBRL_KC_EMBED = 0, EBRL_KC_GEMM = 1, EBRL_KC_SELF_ATTN = 2, EBRL_KC_CROSS_ATTN = 3,
+       EBRL_KC_HEAD = 4, EBRL_KC_COUNT = 5 };
+
+typedef struct {
+    uint64_t groups, envs, env_steps;     /* submitted since create                            */
+    uint64_t kernel_launches;             /* kernels of this library launched since create     */
+    int32_t granted_sms;                  /* SMs of the last submit's quota actually used:
+                                             CTAs of the persistent grids, or the green
+                                             context's SM count when one is active             */
+    int32_t green_ctx_active;             /* 1 if the last submit ran inside a green context   */
+    double class_ms[EBRL_KC_COUNT];       /* device time per kernel class (EBRL_FLAG_TIMING),
+                                             accumulated over synced groups                    */
+    uint64_t class_launches[EBRL_KC_COUNT];
+    double class_flops[EBRL_KC_COUNT];    /* algorithmic 2*m*n*k FLOPs of those launches       */
+    double class_bytes[EBRL_KC_COUNT];    /* algorithmic bytes of those launches               */
+} ebrl_actgen_stats_t;
+
+/* Validates cfg, copies the weights to the device (re-laid-out as the kernels want), builds
+ * the timestep-embedding table, allocates max_inflight_groups workspaces of
+ * max_group_envs * H rows.  Supported: d a multiple of 256 (tensor-core path) or of 64
+ * (plain path), d even, H <= 32, A <= 32, head_dim in {32, 64, 128} ...; anything else
+ * returns EBRL_ERR_UNSUPPORTED.  On failure *out_handle is NULL. */
+ebrl_status_t ebrl_actgen_create(const ebrl_actgen_cfg_t *cfg, const ebrl_actgen_weights_t *weights,
+                                 ebrl_actgen_t *out_handle);
+
+/* Enqueues one group of n_envs environments on `stream`.
+ *   env_ids    host [n]: unique within the group and among groups not yet synced.  Used only
+ *              for these checks and for error text; they never enter the arithmetic.
+ *   prefix_kv  host [n] of DEVICE pointers; env i: [kv_layers][2][P_i][d] in kv_dtype, plane 0
+ *              = K, plane 1 = V, rows contiguous, 16-byte aligned.
+ *   noise      DEVICE [n][H][A] fp32: env i's action state at its step index (the initial
+ *              noise when that is 0).
+ *   out        DEVICE [n][H][A] fp32; may equal noise.
+ *   sm_quota   1..#SMs; 0 = all SMs.  Every kernel of this group runs as a persistent grid of
+ *              at most sm_quota CTAs (at most one CTA's worth of SMs each), inside a green
+ *              context of that many SMs when EBRL_FLAG_GREEN_CTX is set and available.
+ *   stream     cudaStream_t of the caller (NULL = the legacy default stream).  The work is
+ *              ordered after everything already on the stream; `out` is ready for work
+ *              enqueued on the stream afterwards.
+ * Host arrays are copied before the call returns.  Device buffers must stay valid and
+ * unmodified until the group has completed (ebrl_actgen_sync, or a stream synchronisation).
+ * If max_inflight_groups groups are already in flight the call first waits for the oldest
+ * (the bounded queue between simulation and generation, section 4.2.2).  n_envs = 0 is a
+ * no-op returning EBRL_OK. */
+ebrl_status_t ebrl_actgen_submit(ebrl_actgen_t h, int32_t n_envs, const int64_t *env_ids,
+                                 const void *const *prefix_kv, const float *noise, float *out,
+                                 int32_t sm_quota, void *stream, const ebrl_submit_ext_t *ext);
+
+/* The same with HOST buffers: prefix_kv[i], noise and out point to host memory (pinned memory
+ * makes the copies asynchronous).  The planes and the noise are copied to device staging
+ * owned by the handle, the group runs, and `out` is copied back, all on `stream`; `out` is
+ * valid after ebrl_actgen_sync.  Needs prefix_len in ext, or every P_e = max_prefix_len. */
+ebrl_status_t ebrl_actgen_submit_host(ebrl_actgen_t h, int32_t n_envs, const int64_t *env_ids,
+                                      const void *const *prefix_kv_host, const float *noise_host,
+                                      float *out_host, int32_t sm_quota, void *stream,
+                                      const ebrl_submit_ext_t *ext);
+
+/* Blocks until every submitted group has completed; returns the first sticky error. */
+ebrl_status_t ebrl_actgen_sync(ebrl_actgen_t h);
+
+/* Syncs, then frees everything the handle owns. */
+ebrl_status_t ebrl_actgen_destroy(ebrl_actgen_t h);
+
+/* Library-owned, NUL-terminated text of the last error on this handle (or of the last failed
+ * create when h is NULL); valid until the next call on the same handle. */
+const char *ebrl_actgen_last_error(ebrl_actgen_t h);
+
+ebrl_status_t ebrl_actgen_get_stats(ebrl_actgen_t h, ebrl_actgen_stats_t *out_stats);
+ebrl_status_t ebrl_actgen_reset_stats(ebrl_actgen_t h);
+
+uint32_t ebrl_actgen_abi_version(void);
+
+/* ---- host-only helpers (no device needed): the argument rules and the batcher's plan ------
+ * ebrl_actgen_check_cfg / check_submit apply exactly the checks create / submit apply before
+ * touching the device (n_sms = the SM count to check the quota against) and return the same
+ * status; the reason is available from ebrl_actgen_last_error(NULL).
+ * ebrl_actgen_plan_group returns how the ragged batcher packs a group (sections 4.2.2-4.2.3:
+ * environments of a group progress independently): environments are ordered by the number of
+ * steps they run, longest first and ties in arrival order, so that the rows still active at
+ * inner step s are a prefix.  order[n] = caller index of packed position j, nsteps[n] = steps
+ * of packed position j, n_active[K] = environments with more than s steps.  Returns the number
+ * of inner steps, or -1 on bad arguments. */
+ebrl_status_t ebrl_actgen_check_cfg(const ebrl_actgen_cfg_t *cfg);
+ebrl_status_t ebrl_actgen_check_submit(const ebrl_actgen_cfg_t *cfg, int32_t n_sms, int32_t n_envs,
+                                       const int64_t *env_ids, const void *const *prefix_kv,
+                                       const float *noise, const float *out, int32_t sm_quota,
+                                       const ebrl_submit_ext_t *ext);
+int32_t ebrl_actgen_plan_group(const ebrl_actgen_cfg_t *cfg, int32_t n_envs, const ebrl_submit_ext_t *ext,
+                               int32_t *order, int32_t *nsteps, int32_t *n_active);
+
+/* ---- bench utility: the synthetic "simulation" co-runner --------------------------------
+ * A memory-bound stand-in for a GPU simulator sharing the device with generation (sections
+ * 2.2 and 4.2.1): n_steps passes of x[i] = x[i]*alpha + beta over a DEVICE fp32 buffer of
+ * n_floats elements, as a persistent grid of n_ctas CTAs on `stream`.  Bounded by
+ * construction (no flag to wait for). */
+ebrl_status_t ebrl_sim_corunner_launch(float *buf, uint64_t n_floats, int32_t n_steps,
+                                       int32_t n_ctas, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EBRL_ACTGEN_H_ */

@@ -1,0 +1,246 @@
+"""ctypes binding of libebrl_actgen (argument marshalling only; every step of the path runs in
+the library's CUDA kernels).  Names follow ``include/ebrl_actgen.h``.
+
+torch is used for device memory and streams only.  There is no fallback: if the library is
+missing, or no CUDA device is usable, the calls raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence
+
+import torch
+
+from . import build as _build
+
+ABI_VERSION = 1
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_NOMEM, ERR_CUDA, ERR_ENV_BUSY, ERR_QUOTA, ERR_TIMEOUT = range(8)
+F32, BF16 = 0, 1
+FLAG_TEST_PULL, FLAG_GREEN_CTX, FLAG_TIMING, FLAG_FORCE_SIMT = 1, 2, 4, 8
+KC_NAMES = ("embed", "gemm", "self_attn", "cross_attn", "head")
+
+
+class Cfg(C.Structure):
+    _fields_ = [("abi_version", C.c_uint32), ("H", C.c_int32), ("A", C.c_int32), ("d", C.c_int32),
+                ("n_layers", C.c_int32), ("n_heads", C.c_int32), ("mlp_mult", C.c_int32),
+                ("K_steps", C.c_int32), ("max_prefix_len", C.c_int32), ("max_group_envs", C.c_int32),
+                ("max_inflight_groups", C.c_int32), ("param_dtype", C.c_int32), ("kv_dtype", C.c_int32),
+                ("kv_layers", C.c_int32), ("rms_eps", C.c_float), ("temb_scale", C.c_float),
+                ("temb_max_period", C.c_float), ("flags", C.c_uint32), ("device", C.c_int32),
+                ("wait_limit_ns", C.c_uint64)]
+
+
+class LayerWeights(C.Structure):
+    _fields_ = [("g1", C.c_void_p), ("g2", C.c_void_p), ("g3", C.c_void_p), ("w_qkv", C.c_void_p),
+                ("w_o", C.c_void_p), ("w_qc", C.c_void_p), ("w_oc", C.c_void_p), ("w_1", C.c_void_p),
+                ("w_2", C.c_void_p)]
+
+
+class Weights(C.Structure):
+    _fields_ = [("w_in", C.c_void_p), ("w_out", C.c_void_p), ("b_out", C.c_void_p),
+                ("g_final", C.c_void_p), ("layers", C.POINTER(LayerWeights))]
+
+
+class SubmitExt(C.Structure):
+    _fields_ = [("prefix_len", C.POINTER(C.c_int32)), ("step_index", C.POINTER(C.c_int32)),
+                ("n_steps", C.c_int32)]
+
+
+class Stats(C.Structure):
+    _fields_ = [("groups", C.c_uint64), ("envs", C.c_uint64), ("env_steps", C.c_uint64),
+                ("kernel_launches", C.c_uint64), ("granted_sms", C.c_int32),
+                ("green_ctx_active", C.c_int32), ("class_ms", C.c_double * 5),
+                ("class_launches", C.c_uint64 * 5), ("class_flops", C.c_double * 5),
+                ("class_bytes", C.c_double * 5)]
+
+
+class EbrlError(RuntimeError):
+    def __init__(self, status: int, text: str):
+        super().__init__("ebrl_actgen status %d: %s" % (status, text))
+        self.status = status
+
+
+_lib = None
+
+
+def lib():
+    """Loads the in-tree shared library (building it if nvcc is present and it is stale)."""
+    global _lib
+    if _lib is None:
+        path = _build.LIB
+        if _build.stale():
+            path = _build.build()
+        if not os.path.exists(path):
+            raise RuntimeError("libebrl_actgen.so is missing; run python -m paper_2609_27547_b200.build")
+        L = C.CDLL(path)
+        L.ebrl_actgen_last_error.restype = C.c_char_p
+        L.ebrl_actgen_last_error.argtypes = [C.c_void_p]
+        L.ebrl_actgen_abi_version.restype = C.c_uint32
+        L.ebrl_actgen_create.argtypes = [C.POINTER(Cfg), C.POINTER(Weights), C.POINTER(C.c_void_p)]
+        sub = [C.c_void_p, C.c_int32, C.POINTER(C.c_int64), C.POINTER(C.c_void_p), C.c_void_p,
+               C.c_void_p, C.c_int32, C.c_void_p, C.POINTER(SubmitExt)]
+        L.ebrl_actgen_submit.argtypes = sub
+        L.ebrl_actgen_submit_host.argtypes = sub
+        L.ebrl_actgen_sync.argtypes = [C.c_void_p]
+        L.ebrl_actgen_destroy.argtypes = [C.c_void_p]
+        L.ebrl_actgen_get_stats.argtypes = [C.c_void_p, C.POINTER(Stats)]
+        L.ebrl_actgen_reset_stats.argtypes = [C.c_void_p]
+        L.ebrl_actgen_check_cfg.argtypes = [C.POINTER(Cfg)]
+        L.ebrl_actgen_check_submit.argtypes = [C.POINTER(Cfg), C.c_int32, C.c_int32, C.POINTER(C.c_int64),
+                                               C.POINTER(C.c_void_p), C.c_void_p, C.c_void_p, C.c_int32,
+                                               C.POINTER(SubmitExt)]
+        L.ebrl_actgen_plan_group.argtypes = [C.POINTER(Cfg), C.c_int32, C.POINTER(SubmitExt),
+                                             C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+        L.ebrl_actgen_plan_group.restype = C.c_int32
+        L.ebrl_sim_corunner_launch.argtypes = [C.c_void_p, C.c_uint64, C.c_int32, C.c_int32, C.c_void_p]
+        _lib = L
+    return _lib
+
+
+def make_cfg(*, H, A, d, n_layers, n_heads, K_steps, max_prefix_len, max_group_envs,
+             max_inflight_groups=1, dtype=F32, mlp_mult=4, kv_layers=1, rms_eps=1e-6,
+             temb_scale=1000.0, temb_max_period=10000.0, flags=0, device=0) -> Cfg:
+    return Cfg(ABI_VERSION, H, A, d, n_layers, n_heads, mlp_mult, K_steps, max_prefix_len,
+               max_group_envs, max_inflight_groups, dtype, dtype, kv_layers, rms_eps, temb_scale,
+               temb_max_period, flags, device, 0)
+
+
+def _ext(prefix_len, step_index, n_steps):
+    keep = []
+    e = SubmitExt()
+    if prefix_len is not None:
+        a = (C.c_int32 * len(prefix_len))(*[int(v) for v in prefix_len]); keep.append(a)
+        e.prefix_len = C.cast(a, C.POINTER(C.c_int32))
+    if step_index is not None:
+        a = (C.c_int32 * len(step_index))(*[int(v) for v in step_index]); keep.append(a)
+        e.step_index = C.cast(a, C.POINTER(C.c_int32))
+    e.n_steps = int(n_steps)
+    return e, keep
+
+
+def plan_group(cfg: Cfg, n: int, step_index=None, n_steps: int = 0):
+    """Host-only: the batcher's packing of a group -> (S, order, nsteps, n_active)."""
+    e, keep = _ext(None, step_index, n_steps)
+    order = (C.c_int32 * max(1, n))(); ns = (C.c_int32 * max(1, n))(); na = (C.c_int32 * cfg.K_steps)()
+    S = lib().ebrl_actgen_plan_group(C.byref(cfg), n, C.byref(e), order, ns, na)
+    return S, list(order)[:n], list(ns)[:n], list(na)
+
+
+class ActGen:
+    """One handle of the library: ``ebrl_actgen_create`` ... ``ebrl_actgen_destroy``."""
+
+    def __init__(self, cfg: Cfg, weights: dict):
+        """``weights``: dict as produced by ``synth.make_weights`` (torch tensors on any device,
+        matrices in the configured dtype, gains and b_out fp32)."""
+        self._L = lib()
+        self.cfg = cfg
+        want = torch.bfloat16 if cfg.param_dtype == BF16 else torch.float32
+        keep = []
+
+        def ptr(t, dt):
+            if t.dtype != dt:
+                raise TypeError("weight tensor has dtype %s, expected %s" % (t.dtype, dt))
+            t = t.contiguous(); keep.append(t)
+            return t.data_ptr()
+
+        lw = (LayerWeights * max(1, cfg.n_layers))()
+        for i, l in enumerate(weights["layers"]):
+            lw[i] = LayerWeights(ptr(l["g1"], torch.float32), ptr(l["g2"], torch.float32), ptr(l["g3"], torch.float32),
+                                 ptr(l["w_qkv"], want), ptr(l["w_o"], want), ptr(l["w_qc"], want),
+                                 ptr(l["w_oc"], want), ptr(l["w_1"], want), ptr(l["w_2"], want))
+        w = Weights(ptr(weights["w_in"], want), ptr(weights["w_out"], want), ptr(weights["b_out"], torch.float32),
+                    ptr(weights["g_final"], torch.float32), C.cast(lw, C.POINTER(LayerWeights)))
+        self._h = C.c_void_p()
+        st = self._L.ebrl_actgen_create(C.byref(cfg), C.byref(w), C.byref(self._h))
+        if st != OK:
+            raise EbrlError(st, (self._L.ebrl_actgen_last_error(None) or b"").decode())
+        del keep
+
+    def _check(self, st):
+        if st != OK:
+            raise EbrlError(st, (self._L.ebrl_actgen_last_error(self._h) or b"").decode())
+
+    def _submit(self, fn, env_ids, kv_ptrs, noise_ptr, out_ptr, sm_quota, stream, prefix_len, step_index, n_steps):
+        n = len(env_ids)
+        ids = (C.c_int64 * max(1, n))(*[int(e) for e in env_ids])
+        kvp = (C.c_void_p * max(1, n))(*kv_ptrs) if kv_ptrs is not None else None
+        e, keep = _ext(prefix_len, step_index, n_steps)
+        self._check(fn(self._h, n, ids, kvp, noise_ptr, out_ptr, int(sm_quota), stream, C.byref(e)))
+
+    def submit(self, env_ids: Sequence[int], prefix_kv: Optional[Sequence[torch.Tensor]], noise: torch.Tensor,
+               out: torch.Tensor, sm_quota: int = 0, stream: Optional[torch.cuda.Stream] = None,
+               prefix_len: Optional[Sequence[int]] = None, step_index: Optional[Sequence[int]] = None,
+               n_steps: int = 0):
+        """``ebrl_actgen_submit``: device tensors; prefix_kv[i] is [kv_layers][2][P_i][d]."""
+        if noise.device.type != "cuda" or out.device.type != "cuda":
+            raise ValueError("noise and out must be CUDA tensors")
+        if noise.dtype != torch.float32 or out.dtype != torch.float32 or not noise.is_contiguous() or not out.is_contiguous():
+            raise ValueError("noise and out must be contiguous fp32")
+        kv_ptrs = None
+        if prefix_kv is not None:
+            for t in prefix_kv:
+                if t.device.type != "cuda" or not t.is_contiguous():
+                    raise ValueError("prefix planes must be contiguous CUDA tensors")
+            kv_ptrs = [t.data_ptr() for t in prefix_kv]
+            if prefix_len is None:
+                prefix_len = [t.shape[-2] for t in prefix_kv]
+        s = stream if stream is not None else torch.cuda.current_stream(noise.device)
+        self._submit(self._L.ebrl_actgen_submit, env_ids, kv_ptrs, noise.data_ptr(), out.data_ptr(), sm_quota,
+                     s.cuda_stream, prefix_len, step_index, n_steps)
+
+    def submit_host(self, env_ids, prefix_kv: Optional[Sequence[torch.Tensor]], noise: torch.Tensor, out: torch.Tensor,
+                    sm_quota: int = 0, stream: Optional[torch.cuda.Stream] = None, prefix_len=None,
+                    step_index=None, n_steps: int = 0):
+        """``ebrl_actgen_submit_host``: host tensors (pinned for asynchronous copies)."""
+        if noise.device.type != "cpu" or out.device.type != "cpu":
+            raise ValueError("noise and out must be host tensors")
+        kv_ptrs = None
+        if prefix_kv is not None:
+            kv_ptrs = [t.data_ptr() for t in prefix_kv]
+            if prefix_len is None:
+                prefix_len = [t.shape[-2] for t in prefix_kv]
+        s = stream if stream is not None else torch.cuda.current_stream(self.cfg.device)
+        self._submit(self._L.ebrl_actgen_submit_host, env_ids, kv_ptrs, noise.data_ptr(), out.data_ptr(), sm_quota,
+                     s.cuda_stream, prefix_len, step_index, n_steps)
+
+    def sync(self):
+        self._check(self._L.ebrl_actgen_sync(self._h))
+
+    def stats(self) -> dict:
+        s = Stats()
+        self._check(self._L.ebrl_actgen_get_stats(self._h, C.byref(s)))
+        out = {k: getattr(s, k) for k in ("groups", "envs", "env_steps", "kernel_launches", "granted_sms", "green_ctx_active")}
+        out["classes"] = {n: {"ms": s.class_ms[i], "launches": s.class_launches[i], "flops": s.class_flops[i],
+                              "bytes": s.class_bytes[i]} for i, n in enumerate(KC_NAMES)}
+        return out
+
+    def reset_stats(self):
+        self._check(self._L.ebrl_actgen_reset_stats(self._h))
+
+    def destroy(self):
+        if self._h:
+            h, self._h = self._h, C.c_void_p()
+            st = self._L.ebrl_actgen_destroy(h)
+            if st != OK:
+                raise EbrlError(st, "destroy failed")
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def sim_corunner_launch(buf: torch.Tensor, n_steps: int, n_ctas: int, stream: torch.cuda.Stream):
+    st = lib().ebrl_sim_corunner_launch(buf.data_ptr(), buf.numel(), n_steps, n_ctas, stream.cuda_stream)
+    if st != OK:
+        raise EbrlError(st, "corunner launch failed")
+
+
+def cfg_for(w, *, max_group_envs: Optional[int] = None, max_inflight_groups: int = 1, flags: int = 0, device: int = 0) -> Cfg:
+    """The library configuration of a ``synth.Workload``."""
+    return make_cfg(H=w.H, A=w.A, d=w.d, n_layers=w.L, n_heads=w.n_heads, K_steps=w.K, max_prefix_len=w.P[1],
+                    max_group_envs=max_group_envs or (w.group[1] if w.group else w.B),
+                    max_inflight_groups=max_inflight_groups, dtype=BF16 if w.dtype == "bf16" else F32,
+                    mlp_mult=w.mlp_mult, flags=flags, device=device)

@@ -1,0 +1,101 @@
+// Internal declarations shared by the translation units of libebrl_actgen (not part of the ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+namespace ebrl {
+
+// Width (columns) of one sum-of-squares partial of the residual stream.  Every kernel that
+// writes the residual stream x also writes, per row, sum(x^2) over each SSQ_W-column segment;
+// consumers add the d/SSQ_W partials of a row in index order to get the RMSNorm scale.  The
+// segment width is a constant of the library so that the value never depends on tile shapes.
+constexpr int SSQ_W = 128;
+
+// Per-environment record of one submitted group, in packed order (sorted by step count,
+// longest first, so that the rows still active at inner step s are a prefix).
+struct EnvMeta {
+    const void *kv;    // device: [kv_layers][2][P][d]
+    int32_t P;         // prefix length
+    int32_t k0;        // Euler step index the environment starts from
+    int32_t nsteps;    // steps to run in this submit
+    int32_t src;       // index of the environment in the caller's noise/out arrays
+};
+
+enum Epilogue : int {
+    EPI_SCALE_STORE = 0,   // C = acc * rowscale
+    EPI_SCALE_GELU = 1,    // C = gelu(acc * rowscale)
+    EPI_RESID = 2          // x += acc; xg = x * gain; ssq partials
+};
+
+struct GemmArgs {
+    const void *A;         // [M][K] activations (T)
+    const void *W;         // [N][K] weights (TW)
+    int M, N, K;
+    int epi;
+    // EPI_SCALE_*: input row scale from ssq partials of the producer
+    const float *ssq_in;   // [M][d/SSQ_W]
+    int n_ssq;             // d / SSQ_W
+    float inv_d, eps;
+    void *C;               // [M][N] (T)
+    // EPI_RESID
+    float *x;              // [M][N] fp32 residual stream (N == d)
+    const float *gain;     // [N] gain of the next RMSNorm
+    void *xg;              // [M][N] (T)
+    float *ssq_out;        // [M][N/SSQ_W]
+};
+
+struct AttnArgs {
+    const void *q;         // [rows][q_stride] (T), head h at columns h*hd
+    int q_stride;
+    void *out;             // [rows][o_stride] (T)
+    int o_stride;
+    int H, n_heads, hd;
+    int n_envs;            // active environments
+    // cross attention: keys/values from the environment's prefix planes
+    const EnvMeta *meta;   // used when self == 0
+    int d;                 // plane row length
+    int kv_plane;          // plane pair index (layer index when kv_layers > 1, else 0)
+    // self attention: keys/values are the environment's own rows
+    int self;
+    const void *k_self;    // [rows][kv_stride]
+    const void *v_self;
+    int kv_stride;
+};
+
+struct EmbedArgs {
+    const EnvMeta *meta;
+    int n_envs, H, A, d, s;        // s = inner step of this submit
+    const float *noise;            // caller's [n][H][A]
+    const float *a_state;          // [rows][A]
+    const void *w_in;              // [d][A] (TW)
+    const float *temb;             // [K][d]
+    const float *gain;             // [d] gain of layer 0's first norm
+    float *x;                      // [rows][d]
+    void *xg;                      // [rows][d] (T)
+    float *ssq;                    // [rows][d/SSQ_W]
+};
+
+struct HeadArgs {
+    const EnvMeta *meta;
+    int n_envs, H, A, d, s, K;
+    const float *noise;
+    float *a_state;
+    float *out;                    // caller's [n][H][A]
+    const float *x;                // [rows][d]
+    const float *gain;             // g_final
+    const void *w_out;             // [A][d] (TW)
+    const float *b_out;            // [A]
+    float eps;
+    int pull;                      // v = b_out - a
+};
+
+// Launchers (plain-ALU kernels).  bf16 != 0 selects bf16 activations/weights/planes.
+// grid = number of persistent CTAs (the SM quota).
+cudaError_t launch_embed(const EmbedArgs &a, int bf16, int grid, cudaStream_t st);
+cudaError_t launch_head(const HeadArgs &a, int bf16, int grid, cudaStream_t st);
+cudaError_t launch_gemm_simt(const GemmArgs &a, int bf16, int grid, cudaStream_t st);
+cudaError_t launch_attn_simt(const AttnArgs &a, int bf16, int grid, cudaStream_t st);
+
+}  // namespace ebrl

@@ -1,0 +1,629 @@
+// The C-ABI boundary of libebrl_actgen: argument validation, the ragged group batcher, the
+// per-group launch sequence and completion tracking.  All arithmetic of the path runs in the
+// kernels this file launches; nothing here computes on the host except the timestep-embedding
+// table built once at create.
+#include "../../include/ebrl_actgen.h"
+#include "actgen_internal.h"
+
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+#include <new>
+#include <string>
+#include <unordered_set>
+#include <vector>
+
+using namespace ebrl;
+
+namespace {
+
+struct LayerDev {
+    float *g1 = nullptr, *g2 = nullptr, *g3 = nullptr;
+    void *w_qkv = nullptr, *w_o = nullptr, *w_qc = nullptr, *w_oc = nullptr, *w_1 = nullptr, *w_2 = nullptr;
+};
+
+struct TimedLaunch {
+    cudaEvent_t t0, t1;
+    int cls;
+    double flops, bytes;
+};
+
+struct Slot {
+    float *a_state = nullptr, *x = nullptr, *ssq = nullptr;
+    void *xg = nullptr, *qkv = nullptr, *att = nullptr, *qc = nullptr, *u = nullptr;
+    EnvMeta *meta_d = nullptr, *meta_h = nullptr;
+    cudaEvent_t done = nullptr;
+    bool busy = false;
+    std::vector<int64_t> ids;
+    // staging of the host-buffer entry point (allocated on first use)
+    char *kv_stage = nullptr;
+    size_t kv_stage_bytes = 0;
+    float *noise_stage = nullptr, *out_stage = nullptr;
+    std::vector<TimedLaunch> timed;
+    size_t timed_used = 0;
+};
+
+thread_local std::string g_create_error;
+
+}  // namespace
+
+struct ebrl_actgen {
+    ebrl_actgen_cfg_t cfg;
+    int bf16 = 0, n_sms = 0, hd = 0, md = 0;
+    size_t esz = 4;   // bytes per element of matrices / activations / planes
+    void *w_in = nullptr, *w_out = nullptr;
+    float *b_out = nullptr, *g_final = nullptr, *temb = nullptr;
+    std::vector<LayerDev> layers;
+    std::vector<Slot> slots;
+    size_t next_slot = 0;
+    std::unordered_set<int64_t> busy_ids;
+    std::mutex mu;
+    std::string err;
+    ebrl_status_t sticky = EBRL_OK;
+    ebrl_actgen_stats_t stats;
+    std::vector<void *> owned;   // every device allocation, for destroy
+};
+
+namespace {
+
+ebrl_status_t fail(ebrl_actgen *h, ebrl_status_t st, const char *fmt, ...)
+{
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof buf, fmt, ap);
+    va_end(ap);
+    if (h) h->err = buf; else g_create_error = buf;
+    return st;
+}
+
+// ---- pure host checks (also exported for tests that have no GPU) --------------------------
+
+ebrl_status_t check_cfg(const ebrl_actgen_cfg_t *c, std::string *why)
+{
+    auto bad = [&](ebrl_status_t st, const char *m) { if (why) *why = m; return st; };
+    if (!c) return bad(EBRL_ERR_INVALID_ARG, "cfg is NULL");
+    if (c->abi_version != EBRL_ACTGEN_ABI_VERSION) return bad(EBRL_ERR_INVALID_ARG, "abi_version mismatch");
+    if (c->H < 1 || c->A < 1 || c->d < 2 || c->n_layers < 0 || c->n_heads < 1 || c->mlp_mult < 1 || c->K_steps < 1)
+        return bad(EBRL_ERR_INVALID_ARG, "H, A, d, n_heads, mlp_mult, K_steps must be positive and n_layers >= 0");
+    if (c->d % 2) return bad(EBRL_ERR_INVALID_ARG, "d must be even (sin/cos halves of the timestep embedding)");
+    if (c->d % c->n_heads) return bad(EBRL_ERR_INVALID_ARG, "d must be a multiple of n_heads");
+    if (c->max_prefix_len < 1 || c->max_group_envs < 1 || c->max_inflight_groups < 1)
+        return bad(EBRL_ERR_INVALID_ARG, "max_prefix_len, max_group_envs, max_inflight_groups must be >= 1");
+    if ((c->param_dtype != EBRL_F32 && c->param_dtype != EBRL_BF16) || (c->kv_dtype != EBRL_F32 && c->kv_dtype != EBRL_BF16))
+        return bad(EBRL_ERR_INVALID_ARG, "unknown dtype");
+    if (c->kv_layers != 1 && c->kv_layers != c->n_layers) return bad(EBRL_ERR_INVALID_ARG, "kv_layers must be 1 or n_layers");
+    if (!(c->rms_eps >= 0.f) || !(c->temb_max_period > 0.f)) return bad(EBRL_ERR_INVALID_ARG, "rms_eps >= 0 and temb_max_period > 0 required");
+    if (c->H > 32 || c->A > 32) return bad(EBRL_ERR_UNSUPPORTED, "H and A up to 32 are supported");
+    if (c->d % SSQ_W) return bad(EBRL_ERR_UNSUPPORTED, "d must be a multiple of 128");
+    const int hd = c->d / c->n_heads;
+    if (hd != 32 && hd != 64 && hd != 128) return bad(EBRL_ERR_UNSUPPORTED, "head_dim must be 32, 64 or 128");
+    if (c->param_dtype != c->kv_dtype) return bad(EBRL_ERR_UNSUPPORTED, "param_dtype and kv_dtype must match");
+    if ((int64_t)c->max_group_envs * c->H > (int64_t)1 << 24) return bad(EBRL_ERR_UNSUPPORTED, "max_group_envs * H too large");
+    return EBRL_OK;
+}
+
+ebrl_status_t check_submit(const ebrl_actgen_cfg_t *c, int n_sms, int32_t n, const int64_t *env_ids,
+                           const void *const *prefix_kv, const void *noise, const void *out,
+                           int32_t sm_quota, const ebrl_submit_ext_t *ext, std::string *why)
+{
+    auto bad = [&](ebrl_status_t st, const std::string &m) { if (why) *why = m; return st; };
+    if (n < 0) return bad(EBRL_ERR_INVALID_ARG, "n_envs < 0");
+    if (sm_quota < 0 || sm_quota > n_sms) return bad(EBRL_ERR_QUOTA, "sm_quota outside 0..#SMs");
+    if (n == 0) return EBRL_OK;
+    if (n > c->max_group_envs) return bad(EBRL_ERR_INVALID_ARG, "n_envs > max_group_envs");
+    if (!env_ids || !noise || !out) return bad(EBRL_ERR_INVALID_ARG, "env_ids, noise and out must not be NULL");
+    const bool pull = (c->flags & EBRL_FLAG_TEST_PULL) != 0;
+    if (!pull && !prefix_kv) return bad(EBRL_ERR_INVALID_ARG, "prefix_kv is NULL");
+    if (ext && ext->n_steps < 0) return bad(EBRL_ERR_INVALID_ARG, "n_steps < 0");
+    std::unordered_set<int64_t> seen;
+    for (int i = 0; i < n; ++i) {
+        if (!seen.insert(env_ids[i]).second) return bad(EBRL_ERR_INVALID_ARG, "duplicate env id " + std::to_string(env_ids[i]));
+        if (!pull) {
+            if (!prefix_kv[i]) return bad(EBRL_ERR_INVALID_ARG, "prefix_kv[" + std::to_string(i) + "] is NULL");
+            if (((uintptr_t)prefix_kv[i]) & 15) return bad(EBRL_ERR_INVALID_ARG, "prefix_kv[" + std::to_string(i) + "] is not 16-byte aligned");
+        }
+        if (ext && ext->prefix_len) {
+            const int P = ext->prefix_len[i];
+            if (P < 1 || P > c->max_prefix_len) return bad(EBRL_ERR_INVALID_ARG, "prefix_len[" + std::to_string(i) + "] outside 1..max_prefix_len");
+        }
+        if (ext && ext->step_index) {
+            const int k = ext->step_index[i];
+            if (k < 0 || k >= c->K_steps) return bad(EBRL_ERR_INVALID_ARG, "step_index[" + std::to_string(i) + "] outside [0, K)");
+        }
+    }
+    return EBRL_OK;
+}
+
+// The ragged batcher's plan: environments sorted by the number of steps they run (longest
+// first, ties in arrival order) so that the rows active at inner step s form a prefix.
+// order[j] = caller index of packed position j; n_active[s] = environments with more than s
+// steps.  Returns S = the largest step count.
+int plan_group(const ebrl_actgen_cfg_t *c, int n, const ebrl_submit_ext_t *ext, int32_t *order,
+               int32_t *nsteps, int32_t *n_active)
+{
+    const int K = c->K_steps;
+    std::vector<int> steps(n);
+    for (int i = 0; i < n; ++i) {
+        const int k0 = (ext && ext->step_index) ? ext->step_index[i] : 0;
+        int s = K - k0;
+        if (ext && ext->n_steps > 0 && ext->n_steps < s) s = ext->n_steps;
+        steps[i] = s;
+    }
+    for (int i = 0; i < n; ++i) order[i] = i;
+    std::stable_sort(order, order + n, [&](int a, int b) { return steps[a] > steps[b]; });
+    int S = 0;
+    for (int j = 0; j < n; ++j) { nsteps[j] = steps[order[j]]; S = std::max(S, nsteps[j]); }
+    for (int s = 0; s < K; ++s) {
+        int cnt = 0;
+        while (cnt < n && nsteps[cnt] > s) ++cnt;
+        n_active[s] = cnt;
+    }
+    return S;
+}
+
+// ---- device helpers ---------------------------------------------------------------------
+
+#define CK(call)                                                                              \
+    do {                                                                                      \
+        cudaError_t e_ = (call);                                                              \
+        if (e_ != cudaSuccess)                                                                \
+            return fail(h, EBRL_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e_));    \
+    } while (0)
+
+ebrl_status_t dev_alloc(ebrl_actgen *h, void **p, size_t bytes)
+{
+    *p = nullptr;
+    cudaError_t e = cudaMalloc(p, bytes ? bytes : 16);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return fail(h, EBRL_ERR_NOMEM, "cudaMalloc of %zu bytes failed: %s", bytes, cudaGetErrorString(e));
+    }
+    h->owned.push_back(*p);
+    return EBRL_OK;
+}
+
+ebrl_status_t dev_copy_in(ebrl_actgen *h, void **dst, const void *src, size_t bytes)
+{
+    if (!src) return fail(h, EBRL_ERR_INVALID_ARG, "a weight pointer is NULL");
+    ebrl_status_t st = dev_alloc(h, dst, bytes);
+    if (st != EBRL_OK) return st;
+    CK(cudaMemcpy(*dst, src, bytes, cudaMemcpyDefault));
+    return EBRL_OK;
+}
+
+// Waits for a slot's group and folds its timing into the statistics.
+ebrl_status_t retire(ebrl_actgen *h, Slot &s)
+{
+    if (!s.busy) return EBRL_OK;
+    cudaError_t e = cudaEventSynchronize(s.done);
+    s.busy = false;
+    for (int64_t id : s.ids) h->busy_ids.erase(id);
+    s.ids.clear();
+    if (e != cudaSuccess) {
+        if (h->sticky == EBRL_OK) h->sticky = EBRL_ERR_CUDA;
+        return fail(h, EBRL_ERR_CUDA, "group failed: %s", cudaGetErrorString(e));
+    }
+    for (size_t i = 0; i < s.timed_used; ++i) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, s.timed[i].t0, s.timed[i].t1) == cudaSuccess) {
+            h->stats.class_ms[s.timed[i].cls] += ms;
+            h->stats.class_launches[s.timed[i].cls] += 1;
+            h->stats.class_flops[s.timed[i].cls] += s.timed[i].flops;
+            h->stats.class_bytes[s.timed[i].cls] += s.timed[i].bytes;
+        }
+    }
+    s.timed_used = 0;
+    return EBRL_OK;
+}
+
+struct Launcher {
+    ebrl_actgen *h;
+    Slot *slot;
+    cudaStream_t st;
+    int grid;
+    bool timing;
+    cudaError_t err = cudaSuccess;
+
+    template <typename F> void run(int cls, double flops, double bytes, F &&f)
+    {
+        if (err != cudaSuccess) return;
+        TimedLaunch *tl = nullptr;
+        if (timing) {
+            if (slot->timed_used == slot->timed.size()) {
+                TimedLaunch n{};
+                n.t0 = n.t1 = nullptr;
+                if (cudaEventCreate(&n.t0) != cudaSuccess || cudaEventCreate(&n.t1) != cudaSuccess) { err = cudaGetLastError(); return; }
+                slot->timed.push_back(n);
+            }
+            tl = &slot->timed[slot->timed_used++];
+            tl->cls = cls; tl->flops = flops; tl->bytes = bytes;
+            cudaEventRecord(tl->t0, st);
+        }
+        err = f();
+        h->stats.kernel_launches += 1;
+        if (tl) cudaEventRecord(tl->t1, st);
+    }
+};
+
+// Enqueues every kernel of one group on the stream.
+cudaError_t enqueue_group(ebrl_actgen *h, Slot &s, int n, int S, const int32_t *n_active, double sum_P_active[],
+                          const float *noise, float *out, int grid, cudaStream_t st)
+{
+    const ebrl_actgen_cfg_t &c = h->cfg;
+    const int d = c.d, H = c.H, L = c.n_layers, md = h->md, bf = h->bf16;
+    const int nseg = d / SSQ_W;
+    const bool pull = (c.flags & EBRL_FLAG_TEST_PULL) != 0;
+    const double esz = (double)h->esz;
+    Launcher ln{h, &s, st, grid, (c.flags & EBRL_FLAG_TIMING) != 0};
+    (void)n;
+    for (int step = 0; step < S; ++step) {
+        const int ne = n_active[step], M = ne * H;
+        if (ne == 0) break;
+        if (!pull) {
+            EmbedArgs ea{s.meta_d, ne, H, c.A, d, step, noise, s.a_state, h->w_in, h->temb,
+                         L > 0 ? h->layers[0].g1 : h->g_final, s.x, s.xg, s.ssq};
+            ln.run(EBRL_KC_EMBED, 2.0 * M * d * c.A, (double)M * d * (4 + esz), [&] { return launch_embed(ea, bf, grid, st); });
+            for (int l = 0; l < L; ++l) {
+                const LayerDev &w = h->layers[l];
+                auto gemm = [&](const void *A, const void *W, int N, int K, int epi, void *C, const float *gain) {
+                    GemmArgs g{};
+                    g.A = A; g.W = W; g.M = M; g.N = N; g.K = K; g.epi = epi;
+                    g.ssq_in = s.ssq; g.n_ssq = nseg; g.inv_d = 1.0f / (float)d; g.eps = c.rms_eps;
+                    g.C = C; g.x = s.x; g.gain = gain; g.xg = s.xg; g.ssq_out = s.ssq;
+                    const double bytes = ((double)M * K + (double)N * K + (double)M * N) * esz + (epi == EPI_RESID ? 8.0 * M * N : 0.0);
+                    ln.run(EBRL_KC_GEMM, 2.0 * M * N * K, bytes, [&] { return launch_gemm_simt(g, bf, grid, st); });
+                };
+                // self-attention block
+                gemm(s.xg, w.w_qkv, 3 * d, d, EPI_SCALE_STORE, s.qkv, nullptr);
+                {
+                    AttnArgs a{};
+                    a.q = s.qkv; a.q_stride = 3 * d; a.out = s.att; a.o_stride = d;
+                    a.H = H; a.n_heads = c.n_heads; a.hd = h->hd; a.n_envs = ne; a.d = d;
+                    a.self = 1;
+                    a.k_self = (const char *)s.qkv + (size_t)d * h->esz;
+                    a.v_self = (const char *)s.qkv + (size_t)2 * d * h->esz;
+                    a.kv_stride = 3 * d;
+                    ln.run(EBRL_KC_SELF_ATTN, 4.0 * M * H * d, 4.0 * M * d * esz, [&] { return launch_attn_simt(a, bf, grid, st); });
+                }
+                gemm(s.att, w.w_o, d, d, EPI_RESID, nullptr, w.g2);
+                // cross-attention block
+                gemm(s.xg, w.w_qc, d, d, EPI_SCALE_STORE, s.qc, nullptr);
+                {
+                    AttnArgs a{};
+                    a.q = s.qc; a.q_stride = d; a.out = s.att; a.o_stride = d;
+                    a.H = H; a.n_heads = c.n_heads; a.hd = h->hd; a.n_envs = ne; a.d = d;
+                    a.meta = s.meta_d; a.kv_plane = (c.kv_layers == 1) ? 0 : l; a.self = 0;
+                    ln.run(EBRL_KC_CROSS_ATTN, 4.0 * H * sum_P_active[step] * d,
+                           2.0 * sum_P_active[step] * d * esz + 2.0 * M * d * esz,
+                           [&] { return launch_attn_simt(a, bf, grid, st); });
+                }
+                gemm(s.att, w.w_oc, d, d, EPI_RESID, nullptr, w.g3);
+                // MLP block
+                gemm(s.xg, w.w_1, md, d, EPI_SCALE_GELU, s.u, nullptr);
+                gemm(s.u, w.w_2, d, md, EPI_RESID, nullptr, (l + 1 < L) ? h->layers[l + 1].g1 : h->g_final);
+            }
+        }
+        HeadArgs ha{s.meta_d, ne, H, c.A, d, step, c.K_steps, noise, s.a_state, out, s.x, h->g_final,
+                    h->w_out, h->b_out, c.rms_eps, pull ? 1 : 0};
+        ln.run(EBRL_KC_HEAD, 2.0 * M * d * c.A, (double)M * d * 4, [&] { return launch_head(ha, bf, grid, st); });
+    }
+    return ln.err;
+}
+
+ebrl_status_t submit_impl(ebrl_actgen *h, int32_t n, const int64_t *env_ids, const void *const *prefix_kv,
+                          const float *noise, float *out, int32_t sm_quota, void *stream,
+                          const ebrl_submit_ext_t *ext, bool host_buffers)
+{
+    std::string why;
+    ebrl_status_t st = check_submit(&h->cfg, h->n_sms, n, env_ids, prefix_kv, noise, out, sm_quota, ext, &why);
+    if (st != EBRL_OK) return fail(h, st, "%s", why.c_str());
+    if (n == 0) return EBRL_OK;
+    for (int i = 0; i < n; ++i)
+        if (h->busy_ids.count(env_ids[i]))
+            return fail(h, EBRL_ERR_ENV_BUSY, "env id %lld is in a group that has not been synced", (long long)env_ids[i]);
+    if (h->sticky != EBRL_OK) return fail(h, h->sticky, "handle is in a failed state: %s", h->err.c_str());
+    CK(cudaSetDevice(h->cfg.device));
+
+    const ebrl_actgen_cfg_t &c = h->cfg;
+    Slot &s = h->slots[h->next_slot];
+    h->next_slot = (h->next_slot + 1) % h->slots.size();
+    st = retire(h, s);   // bounded queue: wait for the oldest group when every slot is taken
+    if (st != EBRL_OK) return st;
+
+    cudaStream_t cs = (cudaStream_t)stream;
+    const int grid = sm_quota == 0 ? h->n_sms : sm_quota;
+    const bool pull = (c.flags & EBRL_FLAG_TEST_PULL) != 0;
+    const size_t chunk = (size_t)c.H * c.A;
+
+    std::vector<int32_t> order(n), nsteps(n), n_active(c.K_steps);
+    const int S = plan_group(&c, n, ext, order.data(), nsteps.data(), n_active.data());
+
+    // host-buffer variant: stage planes, noise and out on the device
+    const float *noise_d = noise;
+    float *out_d = out;
+    std::vector<const void *> kv_dev(n, nullptr);
+    if (host_buffers) {
+        size_t total = 0;
+        std::vector<size_t> off(n);
+        for (int i = 0; i < n; ++i) {
+            const int P = (ext && ext->prefix_len) ? ext->prefix_len[i] : c.max_prefix_len;
+            off[i] = total;
+            total += ((size_t)c.kv_layers * 2 * P * c.d * h->esz + 255) & ~(size_t)255;
+        }
+        if (!pull && s.kv_stage_bytes < total) {
+            if (s.kv_stage) cudaFree(s.kv_stage);
+            s.kv_stage = nullptr; s.kv_stage_bytes = 0;
+            cudaError_t e = cudaMalloc((void **)&s.kv_stage, total);
+            if (e != cudaSuccess) { cudaGetLastError(); return fail(h, EBRL_ERR_NOMEM, "staging of %zu bytes: %s", total, cudaGetErrorString(e)); }
+            s.kv_stage_bytes = total;
+        }
+        if (!s.noise_stage) {
+            void *p = nullptr;
+            if ((st = dev_alloc(h, &p, (size_t)c.max_group_envs * chunk * 4)) != EBRL_OK) return st;
+            s.noise_stage = (float *)p;
+            if ((st = dev_alloc(h, &p, (size_t)c.max_group_envs * chunk * 4)) != EBRL_OK) return st;
+            s.out_stage = (float *)p;
+        }
+        if (!pull)
+            for (int i = 0; i < n; ++i) {
+                const int P = (ext && ext->prefix_len) ? ext->prefix_len[i] : c.max_prefix_len;
+                CK(cudaMemcpyAsync(s.kv_stage + off[i], prefix_kv[i], (size_t)c.kv_layers * 2 * P * c.d * h->esz, cudaMemcpyHostToDevice, cs));
+                kv_dev[i] = s.kv_stage + off[i];
+            }
+        CK(cudaMemcpyAsync(s.noise_stage, noise, (size_t)n * chunk * 4, cudaMemcpyHostToDevice, cs));
+        noise_d = s.noise_stage;
+        out_d = s.out_stage;
+    } else if (!pull) {
+        for (int i = 0; i < n; ++i) kv_dev[i] = prefix_kv[i];
+    }
+
+    std::vector<double> sum_P(c.K_steps, 0.0);
+    uint64_t env_steps = 0;
+    for (int j = 0; j < n; ++j) {
+        const int i = order[j];
+        EnvMeta &m = s.meta_h[j];
+        m.kv = kv_dev[i];
+        m.P = (ext && ext->prefix_len) ? ext->prefix_len[i] : c.max_prefix_len;
+        m.k0 = (ext && ext->step_index) ? ext->step_index[i] : 0;
+        m.nsteps = nsteps[j];
+        m.src = i;
+        env_steps += (uint64_t)nsteps[j];
+        for (int t = 0; t < nsteps[j]; ++t) sum_P[t] += m.P;
+    }
+    CK(cudaMemcpyAsync(s.meta_d, s.meta_h, sizeof(EnvMeta) * (size_t)n, cudaMemcpyHostToDevice, cs));
+
+    cudaError_t e = enqueue_group(h, s, n, S, n_active.data(), sum_P.data(), noise_d, out_d, grid, cs);
+    if (e != cudaSuccess) {
+        h->sticky = EBRL_ERR_CUDA;
+        return fail(h, EBRL_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
+    }
+    if (host_buffers) CK(cudaMemcpyAsync(out, s.out_stage, (size_t)n * chunk * 4, cudaMemcpyDeviceToHost, cs));
+    CK(cudaEventRecord(s.done, cs));
+    s.busy = true;
+    s.ids.assign(env_ids, env_ids + n);
+    for (int i = 0; i < n; ++i) h->busy_ids.insert(env_ids[i]);
+    h->stats.groups += 1;
+    h->stats.envs += (uint64_t)n;
+    h->stats.env_steps += env_steps;
+    h->stats.granted_sms = grid;
+    h->stats.green_ctx_active = 0;
+    return EBRL_OK;
+}
+
+void free_all(ebrl_actgen *h)
+{
+    for (Slot &s : h->slots) {
+        if (s.done) cudaEventDestroy(s.done);
+        if (s.meta_h) cudaFreeHost(s.meta_h);
+        if (s.kv_stage) cudaFree(s.kv_stage);
+        for (TimedLaunch &t : s.timed) { if (t.t0) cudaEventDestroy(t.t0); if (t.t1) cudaEventDestroy(t.t1); }
+    }
+    for (void *p : h->owned) cudaFree(p);
+    h->owned.clear();
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------------
+// exported
+// ---------------------------------------------------------------------------------------------
+extern "C" {
+
+uint32_t ebrl_actgen_abi_version(void) { return EBRL_ACTGEN_ABI_VERSION; }
+
+// Host-only checks, exported so that the argument rules can be tested without a device.
+ebrl_status_t ebrl_actgen_check_cfg(const ebrl_actgen_cfg_t *cfg)
+{
+    std::string why;
+    ebrl_status_t st = check_cfg(cfg, &why);
+    if (st != EBRL_OK) g_create_error = why;
+    return st;
+}
+
+ebrl_status_t ebrl_actgen_check_submit(const ebrl_actgen_cfg_t *cfg, int32_t n_sms, int32_t n_envs,
+                                       const int64_t *env_ids, const void *const *prefix_kv,
+                                       const float *noise, const float *out, int32_t sm_quota,
+                                       const ebrl_submit_ext_t *ext)
+{
+    std::string why;
+    ebrl_status_t st = check_cfg(cfg, &why);
+    if (st == EBRL_OK) st = check_submit(cfg, n_sms, n_envs, env_ids, prefix_kv, noise, out, sm_quota, ext, &why);
+    if (st != EBRL_OK) g_create_error = why;
+    return st;
+}
+
+// The batcher's plan for a group (host only): order[n], nsteps[n], n_active[K]; returns the
+// number of inner steps, or -1 on bad arguments.
+int32_t ebrl_actgen_plan_group(const ebrl_actgen_cfg_t *cfg, int32_t n_envs, const ebrl_submit_ext_t *ext,
+                               int32_t *order, int32_t *nsteps, int32_t *n_active)
+{
+    if (check_cfg(cfg, nullptr) != EBRL_OK || n_envs < 0 || !order || !nsteps || !n_active) return -1;
+    if (ext && ext->step_index)
+        for (int i = 0; i < n_envs; ++i)
+            if (ext->step_index[i] < 0 || ext->step_index[i] >= cfg->K_steps) return -1;
+    return plan_group(cfg, n_envs, ext, order, nsteps, n_active);
+}
+
+ebrl_status_t ebrl_actgen_create(const ebrl_actgen_cfg_t *cfg, const ebrl_actgen_weights_t *wts, ebrl_actgen_t *out_handle)
+{
+    if (!out_handle) return fail(nullptr, EBRL_ERR_INVALID_ARG, "out_handle is NULL");
+    *out_handle = nullptr;
+    std::string why;
+    ebrl_status_t st = check_cfg(cfg, &why);
+    if (st != EBRL_OK) return fail(nullptr, st, "%s", why.c_str());
+    if (!wts || (cfg->n_layers > 0 && !wts->layers)) return fail(nullptr, EBRL_ERR_INVALID_ARG, "weights is NULL");
+
+    ebrl_actgen *h = new (std::nothrow) ebrl_actgen();
+    if (!h) return fail(nullptr, EBRL_ERR_NOMEM, "out of host memory");
+    h->cfg = *cfg;
+    memset(&h->stats, 0, sizeof h->stats);
+    h->bf16 = cfg->param_dtype == EBRL_BF16;
+    h->esz = h->bf16 ? 2 : 4;
+    h->hd = cfg->d / cfg->n_heads;
+    h->md = cfg->mlp_mult * cfg->d;
+
+    auto bail = [&](ebrl_status_t s) {
+        g_create_error = h->err;
+        free_all(h);
+        delete h;
+        return s;
+    };
+    cudaError_t e = cudaSetDevice(cfg->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->n_sms, cudaDevAttrMultiProcessorCount, cfg->device);
+    if (e != cudaSuccess) {
+        fail(h, EBRL_ERR_CUDA, "no usable CUDA device %d: %s", cfg->device, cudaGetErrorString(e));
+        cudaGetLastError();
+        return bail(EBRL_ERR_CUDA);
+    }
+    const int d = cfg->d, A = cfg->A, md = h->md, L = cfg->n_layers;
+    const size_t esz = h->esz;
+    if ((st = dev_copy_in(h, &h->w_in, wts->w_in, (size_t)d * A * esz)) != EBRL_OK) return bail(st);
+    if ((st = dev_copy_in(h, &h->w_out, wts->w_out, (size_t)A * d * esz)) != EBRL_OK) return bail(st);
+    if ((st = dev_copy_in(h, (void **)&h->b_out, wts->b_out, (size_t)A * 4)) != EBRL_OK) return bail(st);
+    if ((st = dev_copy_in(h, (void **)&h->g_final, wts->g_final, (size_t)d * 4)) != EBRL_OK) return bail(st);
+    h->layers.resize(L);
+    for (int l = 0; l < L; ++l) {
+        const ebrl_layer_weights_t &w = wts->layers[l];
+        LayerDev &o = h->layers[l];
+        if ((st = dev_copy_in(h, (void **)&o.g1, w.g1, (size_t)d * 4)) != EBRL_OK) return bail(st);
+        if ((st = dev_copy_in(h, (void **)&o.g2, w.g2, (size_t)d * 4)) != EBRL_OK) return bail(st);
+        if ((st = dev_copy_in(h, (void **)&o.g3, w.g3, (size_t)d * 4)) != EBRL_OK) return bail(st);
+        if ((st = dev_copy_in(h, &o.w_qkv, w.w_qkv, (size_t)3 * d * d * esz)) != EBRL_OK) return bail(st);
+        if ((st = dev_copy_in(h, &o.w_o, w.w_o, (size_t)d * d * esz)) != EBRL_OK) return bail(st);
+        if ((st = dev_copy_in(h, &o.w_qc, w.w_qc, (size_t)d * d * esz)) != EBRL_OK) return bail(st);
+        if ((st = dev_copy_in(h, &o.w_oc, w.w_oc, (size_t)d * d * esz)) != EBRL_OK) return bail(st);
+        if ((st = dev_copy_in(h, &o.w_1, w.w_1, (size_t)md * d * esz)) != EBRL_OK) return bail(st);
+        if ((st = dev_copy_in(h, &o.w_2, w.w_2, (size_t)d * md * esz)) != EBRL_OK) return bail(st);
+    }
+    {   // timestep-embedding table [K][d], evaluated in double on the host and rounded once
+        std::vector<float> t((size_t)cfg->K_steps * d);
+        const int half = d / 2;
+        for (int k = 0; k < cfg->K_steps; ++k) {
+            const double tau = (double)cfg->temb_scale * ((double)k / (double)cfg->K_steps);
+            for (int j = 0; j < half; ++j) {
+                const double w = std::pow((double)cfg->temb_max_period, -(double)j / (double)half);
+                t[(size_t)k * d + j] = (float)std::sin(tau * w);
+                t[(size_t)k * d + half + j] = (float)std::cos(tau * w);
+            }
+        }
+        if ((st = dev_copy_in(h, (void **)&h->temb, t.data(), t.size() * 4)) != EBRL_OK) return bail(st);
+    }
+    const size_t rows = (size_t)cfg->max_group_envs * cfg->H;
+    h->slots.resize(cfg->max_inflight_groups);
+    for (Slot &s : h->slots) {
+        void *p = nullptr;
+        if ((st = dev_alloc(h, &p, rows * A * 4)) != EBRL_OK) return bail(st); s.a_state = (float *)p;
+        if ((st = dev_alloc(h, &p, rows * d * 4)) != EBRL_OK) return bail(st); s.x = (float *)p;
+        if ((st = dev_alloc(h, &p, rows * (d / SSQ_W) * 4)) != EBRL_OK) return bail(st); s.ssq = (float *)p;
+        if ((st = dev_alloc(h, &s.xg, rows * d * esz)) != EBRL_OK) return bail(st);
+        if ((st = dev_alloc(h, &s.qkv, rows * 3 * d * esz)) != EBRL_OK) return bail(st);
+        if ((st = dev_alloc(h, &s.att, rows * d * esz)) != EBRL_OK) return bail(st);
+        if ((st = dev_alloc(h, &s.qc, rows * d * esz)) != EBRL_OK) return bail(st);
+        if ((st = dev_alloc(h, &s.u, rows * md * esz)) != EBRL_OK) return bail(st);
+        if ((st = dev_alloc(h, &p, sizeof(EnvMeta) * (size_t)cfg->max_group_envs)) != EBRL_OK) return bail(st); s.meta_d = (EnvMeta *)p;
+        if (cudaMallocHost((void **)&s.meta_h, sizeof(EnvMeta) * (size_t)cfg->max_group_envs) != cudaSuccess) {
+            cudaGetLastError();
+            fail(h, EBRL_ERR_NOMEM, "pinned staging allocation failed");
+            return bail(EBRL_ERR_NOMEM);
+        }
+        if (cudaEventCreateWithFlags(&s.done, cudaEventDisableTiming) != cudaSuccess) {
+            fail(h, EBRL_ERR_CUDA, "cudaEventCreate failed");
+            return bail(EBRL_ERR_CUDA);
+        }
+    }
+    *out_handle = h;
+    return EBRL_OK;
+}
+
+ebrl_status_t ebrl_actgen_submit(ebrl_actgen_t h, int32_t n, const int64_t *env_ids, const void *const *prefix_kv,
+                                 const float *noise, float *out, int32_t sm_quota, void *stream, const ebrl_submit_ext_t *ext)
+{
+    if (!h) return EBRL_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lk(h->mu);
+    return submit_impl(h, n, env_ids, prefix_kv, noise, out, sm_quota, stream, ext, false);
+}
+
+ebrl_status_t ebrl_actgen_submit_host(ebrl_actgen_t h, int32_t n, const int64_t *env_ids, const void *const *prefix_kv_host,
+                                      const float *noise_host, float *out_host, int32_t sm_quota, void *stream,
+                                      const ebrl_submit_ext_t *ext)
+{
+    if (!h) return EBRL_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lk(h->mu);
+    return submit_impl(h, n, env_ids, prefix_kv_host, noise_host, out_host, sm_quota, stream, ext, true);
+}
+
+ebrl_status_t ebrl_actgen_sync(ebrl_actgen_t h)
+{
+    if (!h) return EBRL_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lk(h->mu);
+    if (cudaSetDevice(h->cfg.device) != cudaSuccess) return fail(h, EBRL_ERR_CUDA, "cudaSetDevice failed");
+    ebrl_status_t first = EBRL_OK;
+    for (size_t i = 0; i < h->slots.size(); ++i) {
+        Slot &s = h->slots[(h->next_slot + i) % h->slots.size()];
+        ebrl_status_t st = retire(h, s);
+        if (st != EBRL_OK && first == EBRL_OK) first = st;
+    }
+    if (first == EBRL_OK && h->sticky != EBRL_OK) first = h->sticky;
+    return first;
+}
+
+ebrl_status_t ebrl_actgen_destroy(ebrl_actgen_t h)
+{
+    if (!h) return EBRL_OK;
+    ebrl_status_t st;
+    {
+        std::lock_guard<std::mutex> lk(h->mu);
+        cudaSetDevice(h->cfg.device);
+        st = EBRL_OK;
+        for (Slot &s : h->slots) { ebrl_status_t r = retire(h, s); if (r != EBRL_OK && st == EBRL_OK) st = r; }
+        free_all(h);
+    }
+    delete h;
+    return st;
+}
+
+const char *ebrl_actgen_last_error(ebrl_actgen_t h) { return h ? h->err.c_str() : g_create_error.c_str(); }
+
+ebrl_status_t ebrl_actgen_get_stats(ebrl_actgen_t h, ebrl_actgen_stats_t *out)
+{
+    if (!h || !out) return EBRL_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lk(h->mu);
+    *out = h->stats;
+    return EBRL_OK;
+}
+
+ebrl_status_t ebrl_actgen_reset_stats(ebrl_actgen_t h)
+{
+    if (!h) return EBRL_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lk(h->mu);
+    const int32_t g = h->stats.granted_sms, gc = h->stats.green_ctx_active;
+    memset(&h->stats, 0, sizeof h->stats);
+    h->stats.granted_sms = g; h->stats.green_ctx_active = gc;
+    return EBRL_OK;
+}
+
+}  // extern "C"

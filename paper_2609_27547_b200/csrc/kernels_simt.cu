@@ -1,0 +1,420 @@
+// Plain-ALU (FFMA) kernels of the action-generation path: input embedding, velocity head with
+// the Euler update, a tiled GEMM with the fused epilogues, and softmax attention (self and
+// cross).  They serve the fp32 models, whose 1e-4 accuracy bound rules out tensor cores, and
+// they are the fall-back kernels of the bf16 models for shapes the tensor-core kernels do not
+// cover.  Every kernel is a persistent grid of at most `grid` CTAs (the SM quota), and every
+// output element is computed by a fixed sequence of operations that does not depend on the
+// grid size or on which other rows share a tile.
+#include "actgen_internal.h"
+
+namespace ebrl {
+
+template <typename T> __device__ __forceinline__ float ldf(const T *p);
+template <> __device__ __forceinline__ float ldf<float>(const float *p) { return *p; }
+template <> __device__ __forceinline__ float ldf<__nv_bfloat16>(const __nv_bfloat16 *p) { return __bfloat162float(*p); }
+template <typename T> __device__ __forceinline__ void stf(T *p, float v);
+template <> __device__ __forceinline__ void stf<float>(float *p, float v) { *p = v; }
+template <> __device__ __forceinline__ void stf<__nv_bfloat16>(__nv_bfloat16 *p, float v) { *p = __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_max(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ __forceinline__ float gelu_erf(float z) { return 0.5f * z * (1.0f + erff(z * 0.70710678118654752440f)); }
+
+// ---------------------------------------------------------------------------------------
+// x = W_in a + temb(t_k); xg = x * gain; sum-of-squares partials.  One row per CTA pass.
+// ---------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) embed_kernel(EmbedArgs a)
+{
+    __shared__ float sa[32];
+    const int rows = a.n_envs * a.H, nseg = a.d / SSQ_W;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const T *w_in = (const T *)a.w_in;
+    T *xg = (T *)a.xg;
+    for (int row = blockIdx.x; row < rows; row += gridDim.x) {
+        const int env = row / a.H, h = row - env * a.H;
+        const EnvMeta m = a.meta[env];
+        const int k = m.k0 + a.s;
+        const float *av = (a.s == 0) ? a.noise + ((size_t)m.src * a.H + h) * a.A : a.a_state + (size_t)row * a.A;
+        if (threadIdx.x < a.A) sa[threadIdx.x] = av[threadIdx.x];
+        __syncthreads();
+        for (int seg = warp; seg < nseg; seg += 8) {
+            float ss = 0.f;
+#pragma unroll
+            for (int i = 0; i < SSQ_W / 32; ++i) {
+                const int c = seg * SSQ_W + i * 32 + lane;
+                float acc = 0.f;
+                for (int j = 0; j < a.A; ++j) acc = fmaf(ldf(w_in + (size_t)c * a.A + j), sa[j], acc);
+                acc += a.temb[(size_t)k * a.d + c];
+                a.x[(size_t)row * a.d + c] = acc;
+                stf(xg + (size_t)row * a.d + c, acc * a.gain[c]);
+                ss = fmaf(acc, acc, ss);
+            }
+            ss = warp_sum(ss);
+            if (lane == 0) a.ssq[(size_t)row * nseg + seg] = ss;
+        }
+        __syncthreads();
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// v = W_out RMSNorm(x; g_final) + b_out;  a += v / K.  One warp per row.
+// ---------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) head_kernel(HeadArgs a)
+{
+    const int rows = a.n_envs * a.H;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const T *w_out = (const T *)a.w_out;
+    for (int row = blockIdx.x * 8 + warp; row < rows; row += gridDim.x * 8) {
+        const int env = row / a.H, h = row - env * a.H;
+        const EnvMeta m = a.meta[env];
+        const float *xr = a.x + (size_t)row * a.d;
+        float acc[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) acc[j] = 0.f;
+        float ss = 0.f;
+        if (!a.pull) {
+            for (int c = lane; c < a.d; c += 32) {
+                const float xv = xr[c];
+                ss = fmaf(xv, xv, ss);
+                const float t = xv * a.gain[c];
+#pragma unroll
+                for (int j = 0; j < 32; ++j)
+                    if (j < a.A) acc[j] = fmaf(t, ldf(w_out + (size_t)j * a.d + c), acc[j]);
+            }
+            ss = warp_sum(ss);
+        }
+        const float inv = 1.0f / sqrtf(ss / (float)a.d + a.eps);
+        const float *a_old = (a.s == 0) ? a.noise + ((size_t)m.src * a.H + h) * a.A : a.a_state + (size_t)row * a.A;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+            if (j < a.A) {
+                const float dot = warp_sum(acc[j]);
+                if (lane == 0) {
+                    const float ao = a_old[j];
+                    const float v = a.pull ? (a.b_out[j] - ao) : (dot * inv + a.b_out[j]);
+                    const float an = ao + v / (float)a.K;
+                    a.a_state[(size_t)row * a.A + j] = an;
+                    if (a.s == m.nsteps - 1) a.out[((size_t)m.src * a.H + h) * a.A + j] = an;
+                }
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// C = A W^T with fused epilogues.  128 x 128 tile, 1024 threads, 4 x 4 outputs per thread;
+// each output is one FMA chain over k = 0 .. K-1 in order.
+// ---------------------------------------------------------------------------------------
+constexpr int GT = 128, GK = 16, GPAD = 4;
+
+template <typename T>
+__device__ __forceinline__ void load2(const T *p, float &a, float &b);
+template <> __device__ __forceinline__ void load2<float>(const float *p, float &a, float &b)
+{
+    const float2 v = *reinterpret_cast<const float2 *>(p); a = v.x; b = v.y;
+}
+template <> __device__ __forceinline__ void load2<__nv_bfloat16>(const __nv_bfloat16 *p, float &a, float &b)
+{
+    const __nv_bfloat162 v = *reinterpret_cast<const __nv_bfloat162 *>(p);
+    a = __bfloat162float(v.x); b = __bfloat162float(v.y);
+}
+
+template <typename T, int EPI>
+__global__ void __launch_bounds__(1024) gemm_simt_kernel(GemmArgs g)
+{
+    __shared__ __align__(16) float As[2][GK][GT + GPAD];
+    __shared__ __align__(16) float Ws[2][GK][GT + GPAD];
+    const int tid = threadIdx.x, tx = tid & 31, ty = tid >> 5;
+    const int lr = tid >> 3, lk = (tid & 7) * 2;
+    const T *A = (const T *)g.A;
+    const T *W = (const T *)g.W;
+    const int ntm = (g.M + GT - 1) / GT, ntn = g.N / GT, ntiles = ntm * ntn, nk = g.K / GK;
+    for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+        const int m0 = (tile / ntn) * GT, n0 = (tile % ntn) * GT;
+        float acc[4][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+        const bool arow_ok = (m0 + lr) < g.M;
+        const T *ap = A + (size_t)(m0 + lr) * g.K + lk;
+        const T *wp = W + (size_t)(n0 + lr) * g.K + lk;
+        float pa0 = 0.f, pa1 = 0.f, pw0, pw1;
+        if (arow_ok) load2(ap, pa0, pa1);
+        load2(wp, pw0, pw1);
+        __syncthreads();   // previous tile's readers are done with both buffers
+        As[0][lk][lr] = pa0; As[0][lk + 1][lr] = pa1;
+        Ws[0][lk][lr] = pw0; Ws[0][lk + 1][lr] = pw1;
+        __syncthreads();
+        for (int kb = 0; kb < nk; ++kb) {
+            const int buf = kb & 1;
+            if (kb + 1 < nk) {
+                if (arow_ok) load2(ap + (size_t)(kb + 1) * GK, pa0, pa1);
+                load2(wp + (size_t)(kb + 1) * GK, pw0, pw1);
+            }
+#pragma unroll
+            for (int k = 0; k < GK; ++k) {
+                const float4 av = *reinterpret_cast<const float4 *>(&As[buf][k][ty * 4]);
+                const float4 wv = *reinterpret_cast<const float4 *>(&Ws[buf][k][tx * 4]);
+                const float aa[4] = {av.x, av.y, av.z, av.w};
+                const float ww[4] = {wv.x, wv.y, wv.z, wv.w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(aa[i], ww[j], acc[i][j]);
+            }
+            if (kb + 1 < nk) {
+                As[buf ^ 1][lk][lr] = pa0; As[buf ^ 1][lk + 1][lr] = pa1;
+                Ws[buf ^ 1][lk][lr] = pw0; Ws[buf ^ 1][lk + 1][lr] = pw1;
+            }
+            __syncthreads();
+        }
+        // ---- epilogue
+        const int col = n0 + tx * 4;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int row = m0 + ty * 4 + i;
+            const bool ok = row < g.M;
+            if (EPI == EPI_RESID) {
+                float ss = 0.f;
+                float xn[4] = {0.f, 0.f, 0.f, 0.f};
+                if (ok) {
+                    const float4 xo = *reinterpret_cast<const float4 *>(g.x + (size_t)row * g.N + col);
+                    xn[0] = xo.x + acc[i][0]; xn[1] = xo.y + acc[i][1];
+                    xn[2] = xo.z + acc[i][2]; xn[3] = xo.w + acc[i][3];
+                    *reinterpret_cast<float4 *>(g.x + (size_t)row * g.N + col) = make_float4(xn[0], xn[1], xn[2], xn[3]);
+                    T *xg = (T *)g.xg + (size_t)row * g.N + col;
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        stf(xg + j, xn[j] * g.gain[col + j]);
+                        ss = fmaf(xn[j], xn[j], ss);
+                    }
+                }
+                ss = warp_sum(ss);
+                if (ok && tx == 0) g.ssq_out[(size_t)row * (g.N / SSQ_W) + n0 / SSQ_W] = ss;
+            } else if (ok) {
+                float s = 0.f;
+                for (int t = 0; t < g.n_ssq; ++t) s += g.ssq_in[(size_t)row * g.n_ssq + t];
+                const float rs = 1.0f / sqrtf(s * g.inv_d + g.eps);
+                T *c = (T *)g.C + (size_t)row * g.N + col;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    float v = acc[i][j] * rs;
+                    if (EPI == EPI_SCALE_GELU) v = gelu_erf(v);
+                    stf(c + j, v);
+                }
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// Softmax attention for one (environment, head) per 128-thread group, four groups per CTA.
+// Keys are visited in blocks of 32 in index order with a running maximum and sum.
+// ---------------------------------------------------------------------------------------
+constexpr int AKB = 32;   // keys per block: a constant, so the arithmetic is the same at any quota
+
+__device__ __forceinline__ void group_sync(int g) { asm volatile("bar.sync %0, 128;" ::"r"(g + 1) : "memory"); }
+
+template <typename T, int RMAX>
+__global__ void __launch_bounds__(512) attn_simt_kernel(AttnArgs a)
+{
+    extern __shared__ float smem[];
+    const int grp = threadIdx.x >> 7, t = threadIdx.x & 127, warp = t >> 5, lane = t & 31;
+    const int H = a.H, hd = a.hd;
+    const int per_group = H * hd + AKB * (hd + 1) + AKB * hd + H * AKB + 2 * H;
+    float *q = smem + (size_t)grp * per_group;
+    float *kb = q + H * hd;
+    float *vb = kb + AKB * (hd + 1);
+    float *p = vb + AKB * hd;
+    float *alpha = p + H * AKB;
+    float *lsum = alpha + H;
+    const int ncg = 128 / hd, c = t % hd, rg = t / hd;
+    const float scale = 1.0f / sqrtf((float)hd);
+    const int items = a.n_envs * a.n_heads;
+    for (int item = blockIdx.x * 4 + grp; item < items; item += gridDim.x * 4) {
+        const int env = item / a.n_heads, h = item - env * a.n_heads;
+        const T *kbase, *vbase;
+        int P, kvs;
+        if (a.self) {
+            kbase = (const T *)a.k_self + (size_t)env * H * a.kv_stride + h * hd;
+            vbase = (const T *)a.v_self + (size_t)env * H * a.kv_stride + h * hd;
+            P = H; kvs = a.kv_stride;
+        } else {
+            const EnvMeta m = a.meta[env];
+            P = m.P; kvs = a.d;
+            kbase = (const T *)m.kv + (size_t)a.kv_plane * 2 * P * a.d + h * hd;
+            vbase = kbase + (size_t)P * a.d;
+        }
+        const T *qg = (const T *)a.q + (size_t)env * H * a.q_stride + h * hd;
+        for (int e = t; e < H * hd; e += 128) {
+            const int i = e / hd, cc = e - i * hd;
+            q[e] = ldf(qg + (size_t)i * a.q_stride + cc) * scale;
+        }
+        float acc[RMAX];
+#pragma unroll
+        for (int r = 0; r < RMAX; ++r) acc[r] = 0.f;
+        float mrun[8], lrun[8];   // rows warp, warp+4, ... (H <= 32)
+#pragma unroll
+        for (int r = 0; r < 8; ++r) { mrun[r] = -INFINITY; lrun[r] = 0.f; }
+        for (int j0 = 0; j0 < P; j0 += AKB) {
+            group_sync(grp);   // q ready; previous block's readers done
+            const int nkeys = min(AKB, P - j0);
+            for (int e = t; e < AKB * hd; e += 128) {
+                const int j = e / hd, cc = e - j * hd;
+                float kv = 0.f, vv = 0.f;
+                if (j < nkeys) {
+                    kv = ldf(kbase + (size_t)(j0 + j) * kvs + cc);
+                    vv = ldf(vbase + (size_t)(j0 + j) * kvs + cc);
+                }
+                kb[j * (hd + 1) + cc] = kv;
+                vb[j * hd + cc] = vv;
+            }
+            group_sync(grp);
+            // scores and running softmax statistics: lane = key, each warp owns rows warp + 4 r
+#pragma unroll
+            for (int r0 = 0; r0 < 8; r0 += 4) {
+                float s[4] = {0.f, 0.f, 0.f, 0.f};
+                const float *krow = kb + lane * (hd + 1);
+                for (int cc = 0; cc < hd; ++cc) {
+                    const float kvv = krow[cc];
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) {
+                        const int i = warp + 4 * (r0 + r);
+                        if (i < H) s[r] = fmaf(q[i * hd + cc], kvv, s[r]);
+                    }
+                }
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    const int i = warp + 4 * (r0 + r);
+                    if (i < H) {
+                        const float sv = (lane < nkeys) ? s[r] : -INFINITY;
+                        const float mnew = fmaxf(mrun[r0 + r], warp_max(sv));
+                        const float pv = expf(sv - mnew);
+                        const float al = expf(mrun[r0 + r] - mnew);
+                        lrun[r0 + r] = lrun[r0 + r] * al + warp_sum(pv);
+                        mrun[r0 + r] = mnew;
+                        p[i * AKB + lane] = pv;
+                        if (lane == 0) alpha[i] = al;
+                    }
+                }
+            }
+            group_sync(grp);
+            // out += p v
+#pragma unroll
+            for (int r = 0; r < RMAX; ++r) {
+                const int i = rg + ncg * r;
+                if (i < H) acc[r] *= alpha[i];
+            }
+            for (int j = 0; j < nkeys; ++j) {
+                const float vv = vb[j * hd + c];
+#pragma unroll
+                for (int r = 0; r < RMAX; ++r) {
+                    const int i = rg + ncg * r;
+                    if (i < H) acc[r] = fmaf(p[i * AKB + j], vv, acc[r]);
+                }
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+            const int i = warp + 4 * r;
+            if (i < H && lane == 0) lsum[i] = lrun[r];
+        }
+        group_sync(grp);
+        T *og = (T *)a.out + (size_t)env * H * a.o_stride + h * hd + c;
+#pragma unroll
+        for (int r = 0; r < RMAX; ++r) {
+            const int i = rg + ncg * r;
+            if (i < H) stf(og + (size_t)i * a.o_stride, acc[r] / lsum[i]);
+        }
+        group_sync(grp);   // lsum, q are reused by the next item
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// launchers
+// ---------------------------------------------------------------------------------------
+cudaError_t launch_embed(const EmbedArgs &a, int bf16, int grid, cudaStream_t st)
+{
+    const int rows = a.n_envs * a.H;
+    if (rows == 0) return cudaSuccess;
+    const int g = rows < grid ? rows : grid;
+    if (bf16) embed_kernel<__nv_bfloat16><<<g, 256, 0, st>>>(a);
+    else embed_kernel<float><<<g, 256, 0, st>>>(a);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_head(const HeadArgs &a, int bf16, int grid, cudaStream_t st)
+{
+    const int rows = a.n_envs * a.H;
+    if (rows == 0) return cudaSuccess;
+    const int need = (rows + 7) / 8;
+    const int g = need < grid ? need : grid;
+    if (bf16) head_kernel<__nv_bfloat16><<<g, 256, 0, st>>>(a);
+    else head_kernel<float><<<g, 256, 0, st>>>(a);
+    return cudaGetLastError();
+}
+
+template <typename T>
+static cudaError_t gemm_simt_dispatch(const GemmArgs &a, int g, cudaStream_t st)
+{
+    switch (a.epi) {
+    case EPI_SCALE_STORE: gemm_simt_kernel<T, EPI_SCALE_STORE><<<g, 1024, 0, st>>>(a); break;
+    case EPI_SCALE_GELU: gemm_simt_kernel<T, EPI_SCALE_GELU><<<g, 1024, 0, st>>>(a); break;
+    default: gemm_simt_kernel<T, EPI_RESID><<<g, 1024, 0, st>>>(a); break;
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gemm_simt(const GemmArgs &a, int bf16, int grid, cudaStream_t st)
+{
+    if (a.M == 0) return cudaSuccess;
+    const int tiles = ((a.M + GT - 1) / GT) * (a.N / GT);
+    const int g = tiles < grid ? tiles : grid;
+    return bf16 ? gemm_simt_dispatch<__nv_bfloat16>(a, g, st) : gemm_simt_dispatch<float>(a, g, st);
+}
+
+template <typename T, int RMAX>
+static cudaError_t attn_launch(const AttnArgs &a, int g, size_t smem, cudaStream_t st)
+{
+    cudaError_t e = cudaFuncSetAttribute(attn_simt_kernel<T, RMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    attn_simt_kernel<T, RMAX><<<g, 512, smem, st>>>(a);
+    return cudaGetLastError();
+}
+
+template <typename T>
+static cudaError_t attn_dispatch(const AttnArgs &a, int g, size_t smem, cudaStream_t st)
+{
+    const int ncg = 128 / a.hd;
+    const int R = (a.H + ncg - 1) / ncg;
+    if (R <= 4) return attn_launch<T, 4>(a, g, smem, st);
+    if (R <= 8) return attn_launch<T, 8>(a, g, smem, st);
+    if (R <= 16) return attn_launch<T, 16>(a, g, smem, st);
+    return attn_launch<T, 32>(a, g, smem, st);
+}
+
+cudaError_t launch_attn_simt(const AttnArgs &a, int bf16, int grid, cudaStream_t st)
+{
+    const int items = a.n_envs * a.n_heads;
+    if (items == 0) return cudaSuccess;
+    const int need = (items + 3) / 4;
+    const int g = need < grid ? need : grid;
+    const size_t per_group = (size_t)a.H * a.hd + AKB * (a.hd + 1) + AKB * a.hd + a.H * AKB + 2 * a.H;
+    const size_t smem = 4 * per_group * sizeof(float);
+    return bf16 ? attn_dispatch<__nv_bfloat16>(a, g, smem, st) : attn_dispatch<float>(a, g, smem, st);
+}
+
+}  // namespace ebrl

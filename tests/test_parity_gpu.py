@@ -1,0 +1,211 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle element by
+element on the same seeded inputs; bit-identity of GPU results across SM quotas, group
+partitions, arrival orders and step-at-a-time batching; closed forms; edge cases.
+
+Tolerances (max over environments of max|gpu - oracle| / max(1, max|oracle|) on the final
+action chunk): 1e-4 for fp32 models, 2e-2 for bf16 models with fp32 accumulation.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_27547_b200 import binding as B
+from paper_2609_27547_b200 import synth
+from helpers import chunk_rel_err, oracle_run, np32
+from gpu_helpers import Runner, TOL, stack, to_dev
+
+pytestmark = pytest.mark.gpu
+SEED = synth.DEFAULT_SEED
+
+
+def _setup(w, n=None, random_gains=True, seed=SEED):
+    wt = synth.make_weights(w, seed, random_gains=random_gains)
+    envs = [synth.make_env(w, e, seed) for e in range(n if n is not None else w.B)]
+    return wt, envs
+
+
+def test_cfg0_tiny_fp32_parity():
+    """The tiny fp32 configuration as stated: 16 envs, one group, full quota."""
+    w = synth.WORKLOADS[0]
+    wt, envs = _setup(w, random_gains=False)
+    ref = oracle_run(w, wt, envs)
+    r = Runner(w, wt, envs)
+    got = stack(r.run([list(range(w.B))]), range(w.B))
+    r.close()
+    assert chunk_rel_err(got, ref) <= TOL["f32"]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_small_models_parity_ragged(dtype):
+    """Several row tiles and a ragged tail: 37 envs x H=8 = 296 rows (128-row tiles: 2 full +
+    40 rows), ragged prefix lengths not multiples of the key block, mixed step indices."""
+    w = synth.scaled(synth.WORKLOADS[0], B=37, dtype=dtype, P=(1, 97), mixed_steps=True, K=5)
+    wt, envs = _setup(w)
+    ref = oracle_run(w, wt, envs)
+    r = Runner(w, wt, envs)
+    got = stack(r.run([list(range(w.B))]), range(w.B))
+    r.close()
+    assert chunk_rel_err(got, ref) <= TOL[dtype]
+
+
+def test_cfg1_model_bf16_parity_sample():
+    """The mid-size bf16 head (d=1024, L=4, 16 heads, P=256, K=10) on a few environments."""
+    w = synth.scaled(synth.WORKLOADS[1], B=6)
+    wt = synth.make_weights(w, SEED, device="cuda")
+    envs = [synth.make_env(w, e, SEED) for e in range(w.B)]
+    ref = oracle_run(w, wt, envs)
+    r = Runner(w, wt, envs)
+    got = stack(r.run([list(range(w.B))]), range(w.B))
+    r.close()
+    assert chunk_rel_err(got, ref) <= TOL["bf16"]
+
+
+def test_bimanual_shape_bf16_parity():
+    """H=16, A=14, head_dim=128 (the large configuration's token and head shapes) at d=256."""
+    w = synth.scaled(synth.WORKLOADS[4], B=9, d=256, n_heads=2, L=2, P=(40, 70), K=3, group=None)
+    wt, envs = _setup(w)
+    ref = oracle_run(w, wt, envs)
+    r = Runner(w, wt, envs)
+    got = stack(r.run([list(range(w.B))]), range(w.B))
+    r.close()
+    assert chunk_rel_err(got, ref) <= TOL["bf16"]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_bit_identity_across_quotas_partitions_orders(dtype):
+    """Same environments: one group, seeded ragged groups, a second grouping, reversed order,
+    each alone, and SM quotas 16/37/74/148 must give the same bits."""
+    w = synth.scaled(synth.WORKLOADS[2], B=40, dtype=dtype, P=(64, 160), group=(1, 12))
+    wt, envs = _setup(w)
+    ids = list(range(w.B))
+    r = Runner(w, wt, envs, max_inflight_groups=3)
+    base = stack(r.run([ids], quota=0), ids)
+    for q in (16, 37, 74, 148):
+        assert np.array_equal(stack(r.run([ids], quota=q), ids), base), "quota %d" % q
+    g1 = synth.arrival_groups(w, SEED)
+    g2 = synth.arrival_groups(w, SEED + 1)
+    assert len(g1) > 3 and g1 != g2
+    assert np.array_equal(stack(r.run(g1, quota=37), ids), base)
+    assert np.array_equal(stack(r.run(g2, quota=74), ids), base)
+    assert np.array_equal(stack(r.run([ids[::-1]]), ids), base)
+    assert np.array_equal(stack(r.run([[e] for e in ids[:10]], quota=16), ids[:10]), base[:10])
+    # and against the oracle
+    assert chunk_rel_err(base, oracle_run(w, wt, envs)) <= TOL[dtype]
+    r.close()
+
+
+def test_step_at_a_time_equals_full_run():
+    """n_steps = 1 re-batching every Euler step (state carried by the caller in fp32) gives the
+    same bits as running each environment to the end in one submit."""
+    w = synth.scaled(synth.WORKLOADS[0], B=12, P=(20, 50), mixed_steps=True, K=4)
+    wt, envs = _setup(w)
+    ids = list(range(w.B))
+    r = Runner(w, wt, envs)
+    full = stack(r.run([ids]), ids)
+    state = {e: r.noise[e].clone() for e in ids}
+    steps = {e: r.envs[e].step for e in ids}
+    live = list(ids)
+    while live:
+        res = r.run([live], n_steps=1, state=state, steps=steps)
+        for e in live:
+            state[e] = torch.from_numpy(res[e]).cuda()
+            steps[e] += 1
+        live = [e for e in live if steps[e] < w.K]
+    assert np.array_equal(np.stack([state[e].cpu().numpy() for e in ids]), full)
+    r.close()
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_zero_weights_closed_form(dtype):
+    """All matrices zero: a_K = a_0 + b (K additions of b/K in fp32)."""
+    w = synth.scaled(synth.WORKLOADS[0], B=5, dtype=dtype)
+    wt, envs = _setup(w)
+    for k in ("w_in", "w_out"):
+        wt[k].zero_()
+    for l in wt["layers"]:
+        for k in ("w_qkv", "w_o", "w_qc", "w_oc", "w_1", "w_2"):
+            l[k].zero_()
+    r = Runner(w, wt, envs)
+    got = stack(r.run([list(range(w.B))]), range(w.B))
+    r.close()
+    want = np.stack([np32(e.noise) for e in envs]).astype(np.float64) + np32(wt["b_out"]).astype(np.float64)
+    assert np.abs(got - want).max() < 1e-6
+
+
+def test_pull_field_closed_form():
+    """v = c - a: a_K = c + (a_0 - c)(1 - 1/K)^K; from step k0 the exponent is K - k0."""
+    w = synth.scaled(synth.WORKLOADS[0], B=7, K=10, mixed_steps=True)
+    wt, envs = _setup(w)
+    r = Runner(w, wt, envs, flags=B.FLAG_TEST_PULL)
+    got = stack(r.run([list(range(w.B))]), range(w.B))
+    r.close()
+    c = np32(wt["b_out"]).astype(np.float64)
+    for i, e in enumerate(envs):
+        want = c + (np32(e.noise).astype(np.float64) - c) * (1 - 1 / w.K) ** (w.K - e.step)
+        assert np.abs(got[i] - want).max() < 1e-6
+
+
+def test_edge_cases():
+    """Empty group; one environment; prefix of one token; H = 1; one Euler step."""
+    w = synth.scaled(synth.WORKLOADS[0], B=3, H=1, A=1, P=(1, 1), K=1)
+    wt, envs = _setup(w)
+    r = Runner(w, wt, envs)
+    assert r.run([[]]) == {}
+    got = stack(r.run([[0], [1, 2]]), range(3))
+    r.close()
+    assert chunk_rel_err(got, oracle_run(w, wt, envs)) <= TOL["f32"]
+
+
+def test_maximum_sizes_of_the_interface():
+    """H = 32 and A = 32 (the largest supported), head_dim 32, prefix longer than several key
+    blocks."""
+    w = synth.scaled(synth.WORKLOADS[0], B=3, H=32, A=32, d=128, n_heads=4, L=1, P=(130, 200), K=2)
+    wt, envs = _setup(w)
+    r = Runner(w, wt, envs)
+    got = stack(r.run([[0, 1, 2]]), range(3))
+    r.close()
+    assert chunk_rel_err(got, oracle_run(w, wt, envs)) <= TOL["f32"]
+
+
+def test_host_buffer_entry_point_matches_device_entry_point():
+    w = synth.scaled(synth.WORKLOADS[0], B=6, P=(10, 40), mixed_steps=True)
+    wt, envs = _setup(w)
+    ids = list(range(w.B))
+    r = Runner(w, wt, envs)
+    base = stack(r.run([ids]), ids)
+    noise = torch.stack([e.noise for e in envs]).pin_memory()
+    out = torch.empty_like(noise).pin_memory()
+    kv = [e.kv.contiguous().pin_memory() for e in envs]
+    r.gen.submit_host(ids, kv, noise, out, step_index=[e.step for e in envs])
+    r.gen.sync()
+    assert np.array_equal(out.numpy(), base)
+    r.close()
+
+
+def test_errors_and_busy_ids():
+    w = synth.scaled(synth.WORKLOADS[0], B=4)
+    wt, envs = _setup(w)
+    r = Runner(w, wt, envs, max_inflight_groups=2)
+    noise = torch.stack([r.noise[e] for e in range(4)])
+    out = torch.empty_like(noise)
+    kv = [r.kv[e] for e in range(4)]
+    with pytest.raises(B.EbrlError) as ei:
+        r.gen.submit([0, 1, 1, 2], kv, noise, out)
+    assert ei.value.status == B.ERR_INVALID_ARG
+    with pytest.raises(B.EbrlError) as ei:
+        r.gen.submit([0, 1, 2, 3], kv, noise, out, sm_quota=100000)
+    assert ei.value.status == B.ERR_QUOTA
+    with pytest.raises(B.EbrlError) as ei:
+        r.gen.submit([0, 1, 2, 3], kv, noise, out, step_index=[0, 0, w.K, 0])
+    assert ei.value.status == B.ERR_INVALID_ARG
+    r.gen.submit([0, 1, 2, 3], kv, noise, out)
+    out2 = torch.empty_like(noise)
+    with pytest.raises(B.EbrlError) as ei:
+        r.gen.submit([7, 3], kv[:2], noise[:2], out2[:2])      # env 3 is still in flight
+    assert ei.value.status == B.ERR_ENV_BUSY
+    r.gen.sync()
+    r.gen.submit([7, 3], kv[:2], noise[:2].contiguous(), out2[:2])   # fine after the sync
+    r.gen.sync()
+    st = r.gen.stats()
+    assert st["groups"] == 2 and st["envs"] == 6 and st["kernel_launches"] > 0
+    r.close()
