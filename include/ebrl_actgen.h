@@ -187,6 +187,9 @@ const char *ebrl_actgen_last_error(ebrl_actgen_t h);
 ebrl_status_t ebrl_actgen_get_stats(ebrl_actgen_t h, ebrl_actgen_stats_t *out_stats);
 ebrl_status_t ebrl_actgen_reset_stats(ebrl_actgen_t h);
 
+/* Switches the per-kernel-class timing (EBRL_FLAG_TIMING) on or off for later submits. */
+ebrl_status_t ebrl_actgen_set_timing(ebrl_actgen_t h, int32_t on);
+
 uint32_t ebrl_actgen_abi_version(void);
 
 /* ---- host-only helpers (no device needed): the argument rules and the batcher's plan ------

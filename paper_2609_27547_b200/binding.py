@@ -86,6 +86,7 @@ def lib():
         L.ebrl_actgen_destroy.argtypes = [C.c_void_p]
         L.ebrl_actgen_get_stats.argtypes = [C.c_void_p, C.POINTER(Stats)]
         L.ebrl_actgen_reset_stats.argtypes = [C.c_void_p]
+        L.ebrl_actgen_set_timing.argtypes = [C.c_void_p, C.c_int32]
         L.ebrl_actgen_check_cfg.argtypes = [C.POINTER(Cfg)]
         L.ebrl_actgen_check_submit.argtypes = [C.POINTER(Cfg), C.c_int32, C.c_int32, C.POINTER(C.c_int64),
                                                C.POINTER(C.c_void_p), C.c_void_p, C.c_void_p, C.c_int32,
@@ -217,6 +218,9 @@ class ActGen:
 
     def reset_stats(self):
         self._check(self._L.ebrl_actgen_reset_stats(self._h))
+
+    def set_timing(self, on: bool):
+        self._check(self._L.ebrl_actgen_set_timing(self._h, 1 if on else 0))
 
     def destroy(self):
         if self._h:

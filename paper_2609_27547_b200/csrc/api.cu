@@ -626,4 +626,12 @@ ebrl_status_t ebrl_actgen_reset_stats(ebrl_actgen_t h)
     return EBRL_OK;
 }
 
+ebrl_status_t ebrl_actgen_set_timing(ebrl_actgen_t h, int32_t on)
+{
+    if (!h) return EBRL_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lk(h->mu);
+    if (on) h->cfg.flags |= EBRL_FLAG_TIMING; else h->cfg.flags &= ~EBRL_FLAG_TIMING;
+    return EBRL_OK;
+}
+
 }  // extern "C"
