@@ -91,6 +91,17 @@ struct HeadArgs {
     int pull;                      // v = b_out - a
 };
 
+// Opaque storage of a CUtensorMap (the driver's 128-byte TMA descriptor).
+struct alignas(64) TensorMap128 { uint64_t opaque[16]; };
+
+// Tensor-core GEMM (bf16 operands, fp32 accumulation in tensor memory).
+int make_tmap_bf16(TensorMap128 *out, const void *base, uint64_t inner, uint64_t rows, uint32_t box_rows);
+bool gemm_tc_supported(int N, int K);
+int gemm_tc_box_rows_a();
+int gemm_tc_box_rows_w();
+cudaError_t launch_gemm_tc(const TensorMap128 &ta, const TensorMap128 &tw, const GemmArgs &a, int grid,
+                           unsigned long long limit_ns, int *status, cudaStream_t st);
+
 // Launchers (plain-ALU kernels).  bf16 != 0 selects bf16 activations/weights/planes.
 // grid = number of persistent CTAs (the SM quota).
 cudaError_t launch_embed(const EmbedArgs &a, int bf16, int grid, cudaStream_t st);

@@ -23,6 +23,7 @@ namespace {
 struct LayerDev {
     float *g1 = nullptr, *g2 = nullptr, *g3 = nullptr;
     void *w_qkv = nullptr, *w_o = nullptr, *w_qc = nullptr, *w_oc = nullptr, *w_1 = nullptr, *w_2 = nullptr;
+    TensorMap128 t_qkv, t_o, t_qc, t_oc, t_1, t_2;   // TMA descriptors of the matrices (tensor-core path)
 };
 
 struct TimedLaunch {
@@ -35,6 +36,7 @@ struct Slot {
     float *a_state = nullptr, *x = nullptr, *ssq = nullptr;
     void *xg = nullptr, *qkv = nullptr, *att = nullptr, *qc = nullptr, *u = nullptr;
     EnvMeta *meta_d = nullptr, *meta_h = nullptr;
+    TensorMap128 t_xg, t_att, t_u;                    // TMA descriptors of the A operands
     cudaEvent_t done = nullptr;
     bool busy = false;
     std::vector<int64_t> ids;
@@ -53,6 +55,9 @@ thread_local std::string g_create_error;
 struct ebrl_actgen {
     ebrl_actgen_cfg_t cfg;
     int bf16 = 0, n_sms = 0, hd = 0, md = 0;
+    bool use_tc = false;          // tensor-core GEMMs (bf16, d a multiple of 256)
+    int *status_d = nullptr;      // device status word written by kernels whose waits ran out
+    unsigned long long wait_ns = 0;
     size_t esz = 4;   // bytes per element of matrices / activations / planes
     void *w_in = nullptr, *w_out = nullptr;
     float *b_out = nullptr, *g_final = nullptr, *temb = nullptr;
@@ -269,16 +274,20 @@ cudaError_t enqueue_group(ebrl_actgen *h, Slot &s, int n, int S, const int32_t *
             ln.run(EBRL_KC_EMBED, 2.0 * M * d * c.A, (double)M * d * (4 + esz), [&] { return launch_embed(ea, bf, grid, st); });
             for (int l = 0; l < L; ++l) {
                 const LayerDev &w = h->layers[l];
-                auto gemm = [&](const void *A, const void *W, int N, int K, int epi, void *C, const float *gain) {
+                auto gemm = [&](const void *A, const TensorMap128 &tA, const void *W, const TensorMap128 &tW, int N, int K, int epi,
+                                void *C, const float *gain) {
                     GemmArgs g{};
                     g.A = A; g.W = W; g.M = M; g.N = N; g.K = K; g.epi = epi;
                     g.ssq_in = s.ssq; g.n_ssq = nseg; g.inv_d = 1.0f / (float)d; g.eps = c.rms_eps;
                     g.C = C; g.x = s.x; g.gain = gain; g.xg = s.xg; g.ssq_out = s.ssq;
                     const double bytes = ((double)M * K + (double)N * K + (double)M * N) * esz + (epi == EPI_RESID ? 8.0 * M * N : 0.0);
-                    ln.run(EBRL_KC_GEMM, 2.0 * M * N * K, bytes, [&] { return launch_gemm_simt(g, bf, grid, st); });
+                    if (h->use_tc)
+                        ln.run(EBRL_KC_GEMM, 2.0 * M * N * K, bytes, [&] { return launch_gemm_tc(tA, tW, g, grid, h->wait_ns, h->status_d, st); });
+                    else
+                        ln.run(EBRL_KC_GEMM, 2.0 * M * N * K, bytes, [&] { return launch_gemm_simt(g, bf, grid, st); });
                 };
                 // self-attention block
-                gemm(s.xg, w.w_qkv, 3 * d, d, EPI_SCALE_STORE, s.qkv, nullptr);
+                gemm(s.xg, s.t_xg, w.w_qkv, w.t_qkv, 3 * d, d, EPI_SCALE_STORE, s.qkv, nullptr);
                 {
                     AttnArgs a{};
                     a.q = s.qkv; a.q_stride = 3 * d; a.out = s.att; a.o_stride = d;
@@ -289,9 +298,9 @@ cudaError_t enqueue_group(ebrl_actgen *h, Slot &s, int n, int S, const int32_t *
                     a.kv_stride = 3 * d;
                     ln.run(EBRL_KC_SELF_ATTN, 4.0 * M * H * d, 4.0 * M * d * esz, [&] { return launch_attn_simt(a, bf, grid, st); });
                 }
-                gemm(s.att, w.w_o, d, d, EPI_RESID, nullptr, w.g2);
+                gemm(s.att, s.t_att, w.w_o, w.t_o, d, d, EPI_RESID, nullptr, w.g2);
                 // cross-attention block
-                gemm(s.xg, w.w_qc, d, d, EPI_SCALE_STORE, s.qc, nullptr);
+                gemm(s.xg, s.t_xg, w.w_qc, w.t_qc, d, d, EPI_SCALE_STORE, s.qc, nullptr);
                 {
                     AttnArgs a{};
                     a.q = s.qc; a.q_stride = d; a.out = s.att; a.o_stride = d;
@@ -301,10 +310,10 @@ cudaError_t enqueue_group(ebrl_actgen *h, Slot &s, int n, int S, const int32_t *
                            2.0 * sum_P_active[step] * d * esz + 2.0 * M * d * esz,
                            [&] { return launch_attn_simt(a, bf, grid, st); });
                 }
-                gemm(s.att, w.w_oc, d, d, EPI_RESID, nullptr, w.g3);
+                gemm(s.att, s.t_att, w.w_oc, w.t_oc, d, d, EPI_RESID, nullptr, w.g3);
                 // MLP block
-                gemm(s.xg, w.w_1, md, d, EPI_SCALE_GELU, s.u, nullptr);
-                gemm(s.u, w.w_2, d, md, EPI_RESID, nullptr, (l + 1 < L) ? h->layers[l + 1].g1 : h->g_final);
+                gemm(s.xg, s.t_xg, w.w_1, w.t_1, md, d, EPI_SCALE_GELU, s.u, nullptr);
+                gemm(s.u, s.t_u, w.w_2, w.t_2, d, md, EPI_RESID, nullptr, (l + 1 < L) ? h->layers[l + 1].g1 : h->g_final);
             }
         }
         HeadArgs ha{s.meta_d, ne, H, c.A, d, step, c.K_steps, noise, s.a_state, out, s.x, h->g_final,
@@ -533,6 +542,29 @@ ebrl_status_t ebrl_actgen_create(const ebrl_actgen_cfg_t *cfg, const ebrl_actgen
         if ((st = dev_copy_in(h, (void **)&h->temb, t.data(), t.size() * 4)) != EBRL_OK) return bail(st);
     }
     const size_t rows = (size_t)cfg->max_group_envs * cfg->H;
+    h->wait_ns = cfg->wait_limit_ns ? cfg->wait_limit_ns : 4000000000ull;
+    {
+        void *p = nullptr;
+        if ((st = dev_alloc(h, &p, 16)) != EBRL_OK) return bail(st);
+        h->status_d = (int *)p;
+        if (cudaMemset(h->status_d, 0, 16) != cudaSuccess) { fail(h, EBRL_ERR_CUDA, "cudaMemset failed"); return bail(EBRL_ERR_CUDA); }
+    }
+    h->use_tc = h->bf16 && !(cfg->flags & EBRL_FLAG_FORCE_SIMT) && gemm_tc_supported(d, d) && gemm_tc_supported(md, d) &&
+                gemm_tc_supported(d, md) && gemm_tc_supported(3 * d, d);
+    if (h->use_tc) {
+        const uint32_t bw = (uint32_t)gemm_tc_box_rows_w();
+        int bad = 0;
+        for (int l = 0; l < L; ++l) {
+            LayerDev &o = h->layers[l];
+            bad |= make_tmap_bf16(&o.t_qkv, o.w_qkv, d, 3 * (uint64_t)d, bw);
+            bad |= make_tmap_bf16(&o.t_o, o.w_o, d, d, bw);
+            bad |= make_tmap_bf16(&o.t_qc, o.w_qc, d, d, bw);
+            bad |= make_tmap_bf16(&o.t_oc, o.w_oc, d, d, bw);
+            bad |= make_tmap_bf16(&o.t_1, o.w_1, d, md, bw);
+            bad |= make_tmap_bf16(&o.t_2, o.w_2, md, d, bw);
+        }
+        if (bad) { fail(h, EBRL_ERR_CUDA, "cuTensorMapEncodeTiled failed for a weight matrix"); return bail(EBRL_ERR_CUDA); }
+    }
     h->slots.resize(cfg->max_inflight_groups);
     for (Slot &s : h->slots) {
         void *p = nullptr;
@@ -549,6 +581,14 @@ ebrl_status_t ebrl_actgen_create(const ebrl_actgen_cfg_t *cfg, const ebrl_actgen
             cudaGetLastError();
             fail(h, EBRL_ERR_NOMEM, "pinned staging allocation failed");
             return bail(EBRL_ERR_NOMEM);
+        }
+        if (h->use_tc) {
+            // the row extent is the workspace capacity: rows past a group's M hold stale data
+            // that only ever reaches output rows that are never stored (rows are independent)
+            const uint32_t ba = (uint32_t)gemm_tc_box_rows_a();
+            int bad = make_tmap_bf16(&s.t_xg, s.xg, d, rows, ba) | make_tmap_bf16(&s.t_att, s.att, d, rows, ba) |
+                      make_tmap_bf16(&s.t_u, s.u, md, rows, ba);
+            if (bad) { fail(h, EBRL_ERR_CUDA, "cuTensorMapEncodeTiled failed for a workspace"); return bail(EBRL_ERR_CUDA); }
         }
         if (cudaEventCreateWithFlags(&s.done, cudaEventDisableTiming) != cudaSuccess) {
             fail(h, EBRL_ERR_CUDA, "cudaEventCreate failed");
@@ -586,6 +626,13 @@ ebrl_status_t ebrl_actgen_sync(ebrl_actgen_t h)
         Slot &s = h->slots[(h->next_slot + i) % h->slots.size()];
         ebrl_status_t st = retire(h, s);
         if (st != EBRL_OK && first == EBRL_OK) first = st;
+    }
+    if (first == EBRL_OK && h->status_d) {
+        int word = 0;
+        if (cudaMemcpy(&word, h->status_d, sizeof word, cudaMemcpyDeviceToHost) == cudaSuccess && word != 0) {
+            h->sticky = (ebrl_status_t)word;
+            fail(h, h->sticky, "a device-side wait ran out of time (status %d)", word);
+        }
     }
     if (first == EBRL_OK && h->sticky != EBRL_OK) first = h->sticky;
     return first;

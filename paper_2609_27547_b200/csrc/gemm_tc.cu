@@ -1,0 +1,369 @@
+// bf16 x bf16 -> fp32 GEMM on the 5th-generation tensor cores (tcgen05.mma, accumulators in
+// tensor memory), operands staged in shared memory by TMA, with the path's fused epilogues:
+// RMSNorm row scale, GELU, residual add, gain multiply for the next norm, and the fixed-width
+// sum-of-squares partials.  C[M][N] = A[M][K] W[N][K]^T, both operands K-major.
+//
+// One persistent CTA per SM of the quota walks a static tile list (tile = blockIdx.x + i *
+// gridDim.x).  Roles: warp 0 issues TMA loads into a 4-stage ring, warp 1 issues the MMAs and
+// owns tensor memory, warps 2..5 run the epilogue of tile i from one 256-column accumulator
+// while tile i+1 accumulates into the other.  Every output element is the sum over k in order
+// in its own accumulator, so results do not depend on the grid size, on the tile a row falls
+// in, or on which rows share it.  Every wait is bounded: on a time-out the CTA records
+// EBRL_ERR_TIMEOUT in the status word, lets its copies land, frees tensor memory and returns.
+#include "actgen_internal.h"
+
+#include <cuda.h>
+
+namespace ebrl {
+
+namespace tc {
+
+constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4, UMMA_K = 16;
+constexpr int THREADS = 192;
+constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2;
+constexpr int SMEM_BYTES = STAGES * (A_BYTES + B_BYTES) + 256 + 1024;   // + barriers + alignment slack
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ unsigned long long gtimer()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try(uint32_t bar, uint32_t parity)
+{
+    uint32_t done;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.b32 %0, 1, 0, p;\n\t}"
+                 : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    return done;
+}
+// Bounded wait: false when the limit ran out or another role of this CTA gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned long long limit_ns, volatile int *abort_flag)
+{
+    for (int i = 0; i < 128; ++i)
+        if (mbar_try(bar, parity)) return true;
+    const unsigned long long t0 = gtimer();
+    for (;;) {
+        for (int i = 0; i < 256; ++i)
+            if (mbar_try(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (gtimer() - t0 > limit_ns) return false;
+    }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tm, uint32_t bar, int c0, int c1)
+{
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                 "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes (64 bf16) with the
+// 128-byte swizzle TMA wrote: 8-row groups are 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr)
+{
+    uint64_t d = (uint64_t)((addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)1 << 16;               // leading byte offset (unused for swizzled K-major)
+    d |= (uint64_t)(1024 >> 4) << 32;     // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;               // descriptor version of sm_100
+    d |= (uint64_t)2 << 61;               // 128-byte swizzle
+    return d;
+}
+// kind::f16 instruction descriptor: fp32 accumulate, bf16 A and B, both K-major, M x N.
+__host__ __device__ constexpr uint32_t instr_desc(int M, int N)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+__device__ __forceinline__ float gelu_erf(float z) { return 0.5f * z * (1.0f + erff(z * 0.70710678118654752440f)); }
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+
+template <int EPI>
+__global__ void __launch_bounds__(THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmArgs g,
+               unsigned long long limit_ns, int *status)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const uint32_t sA = smem_u32(smem), sB = sA + STAGES * A_BYTES;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + STAGES * (A_BYTES + B_BYTES));
+    const uint32_t bar0 = smem_u32(bars);
+    auto full = [&](int s) { return bar0 + 8u * s; };
+    auto empty = [&](int s) { return bar0 + 8u * (STAGES + s); };
+    auto tfull = [&](int b) { return bar0 + 8u * (2 * STAGES + b); };
+    auto tempty = [&](int b) { return bar0 + 8u * (2 * STAGES + 2 + b); };
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(bars + 2 * STAGES + 4);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 2 * STAGES + 5);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int ntm = (g.M + BM - 1) / BM, ntn = g.N / BN, ntiles = ntm * ntn, nkb = g.K / BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(tfull(b), 1); mbar_init(tempty(b), 4); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmA)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmB)) : "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void *)tmem_slot)), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    bool ok = true;
+
+    if (warp == 0) {
+        // ---- TMA producer
+        int stage = 0;
+        uint32_t phase = 0;
+        for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
+            const int m0 = (tile / ntn) * BM, n0 = (tile % ntn) * BN;
+            for (int kb = 0; kb < nkb; ++kb) {
+                if (!__all_sync(0xffffffffu, mbar_wait(empty(stage), phase ^ 1u, limit_ns, abort_flag))) { ok = false; break; }
+                if (lane == 0) {
+                    mbar_expect_tx(full(stage), A_BYTES + B_BYTES);
+                    tma_load_2d(sA + stage * A_BYTES, &tmA, full(stage), kb * BK, m0);
+                    tma_load_2d(sB + stage * B_BYTES, &tmB, full(stage), kb * BK, n0);
+                }
+                __syncwarp();
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
+        }
+    } else if (warp == 1) {
+        // ---- MMA issuer
+        constexpr uint32_t idesc = instr_desc(BM, BN);
+        int stage = 0, it = 0;
+        uint32_t phase = 0;
+        for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++it) {
+            const int buf = it & 1;
+            const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+            if (!__all_sync(0xffffffffu, mbar_wait(tempty(buf), acc_phase ^ 1u, limit_ns, abort_flag))) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + (uint32_t)buf * BN;
+            for (int kb = 0; kb < nkb; ++kb) {
+                if (!__all_sync(0xffffffffu, mbar_wait(full(stage), phase, limit_ns, abort_flag))) { ok = false; break; }
+                tc_fence_after();
+                if (lane == 0) {
+                    const uint64_t ad = smem_desc(sA + stage * A_BYTES), bd = smem_desc(sB + stage * B_BYTES);
+#pragma unroll
+                    for (int k = 0; k < BK / UMMA_K; ++k)
+                        tc_mma(d_tmem, ad + (uint64_t)(k * UMMA_K * 2 / 16), bd + (uint64_t)(k * UMMA_K * 2 / 16), idesc,
+                               (kb | k) != 0 ? 1u : 0u);
+                    tc_commit(empty(stage));
+                }
+                __syncwarp();
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
+            if (!ok) break;
+            if (lane == 0) tc_commit(tfull(buf));
+            __syncwarp();
+        }
+    } else {
+        // ---- epilogue: warp w reads TMEM lanes 32 (w % 4) .. +31; one thread per output row
+        const int q = warp & 3;
+        int it = 0;
+        for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++it) {
+            const int buf = it & 1;
+            const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+            const int m0 = (tile / ntn) * BM, n0 = (tile % ntn) * BN;
+            const int row = m0 + q * 32 + lane;
+            const bool valid = row < g.M;
+            float rs = 0.f;
+            if (EPI != EPI_RESID && valid) {
+                float s = 0.f;
+                for (int t = 0; t < g.n_ssq; ++t) s += g.ssq_in[(size_t)row * g.n_ssq + t];
+                rs = 1.0f / sqrtf(s * g.inv_d + g.eps);
+            }
+            if (!__all_sync(0xffffffffu, mbar_wait(tfull(buf), acc_phase, limit_ns, abort_flag))) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * BN;
+            float ss = 0.f;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t r[32];
+                tc_ld32(taddr + (uint32_t)c * 32, r);
+                const int col = n0 + c * 32;
+                if (EPI == EPI_RESID) {
+                    float4 xo[8];
+                    float *xp = g.x + (size_t)row * g.N + col;
+                    if (valid) {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) xo[j] = *reinterpret_cast<const float4 *>(xp + 4 * j);
+                    }
+                    tc_wait_ld();
+                    if (valid) {
+                        uint32_t pk[16];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            const float4 gn = *reinterpret_cast<const float4 *>(g.gain + col + 4 * j);
+                            float4 xn;
+                            xn.x = xo[j].x + __uint_as_float(r[4 * j + 0]);
+                            xn.y = xo[j].y + __uint_as_float(r[4 * j + 1]);
+                            xn.z = xo[j].z + __uint_as_float(r[4 * j + 2]);
+                            xn.w = xo[j].w + __uint_as_float(r[4 * j + 3]);
+                            *reinterpret_cast<float4 *>(xp + 4 * j) = xn;
+                            ss = fmaf(xn.x, xn.x, ss); ss = fmaf(xn.y, xn.y, ss);
+                            ss = fmaf(xn.z, xn.z, ss); ss = fmaf(xn.w, xn.w, ss);
+                            pk[2 * j] = pack_bf16(xn.x * gn.x, xn.y * gn.y);
+                            pk[2 * j + 1] = pack_bf16(xn.z * gn.z, xn.w * gn.w);
+                        }
+                        uint4 *xg = reinterpret_cast<uint4 *>((__nv_bfloat16 *)g.xg + (size_t)row * g.N + col);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) xg[j] = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
+                        if ((c & 3) == 3) {
+                            g.ssq_out[(size_t)row * (g.N / SSQ_W) + (col + 32 - SSQ_W) / SSQ_W] = ss;
+                            ss = 0.f;
+                        }
+                    }
+                } else {
+                    tc_wait_ld();
+                    if (valid) {
+                        uint32_t pk[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            float a = __uint_as_float(r[2 * j]) * rs, b = __uint_as_float(r[2 * j + 1]) * rs;
+                            if (EPI == EPI_SCALE_GELU) { a = gelu_erf(a); b = gelu_erf(b); }
+                            pk[j] = pack_bf16(a, b);
+                        }
+                        uint4 *cp = reinterpret_cast<uint4 *>((__nv_bfloat16 *)g.C + (size_t)row * g.N + col);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) cp[j] = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty(buf));
+        }
+    }
+
+    // ---- teardown
+    if (!ok) {
+        *abort_flag = 1;
+        if (lane == 0) atomicExch(status, (int)7 /* EBRL_ERR_TIMEOUT */);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag && threadIdx.x == 0) {
+        // give copies that were still in flight time to land before shared memory is released
+        const unsigned long long t0 = gtimer();
+        while (gtimer() - t0 < 200000ull) { }
+    }
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    }
+}
+
+}  // namespace tc
+
+// ---- host side -------------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// 2-D bf16 tensor map of a row-major [rows][inner] matrix, box = 64 x box_rows, 128-byte swizzle.
+int make_tmap_bf16(TensorMap128 *out, const void *base, uint64_t inner, uint64_t rows, uint32_t box_rows)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return 1;
+    static_assert(sizeof(TensorMap128) == sizeof(CUtensorMap), "tensor map size");
+    const cuuint64_t dims[2] = {inner, rows};
+    const cuuint64_t strides[1] = {inner * 2};
+    const cuuint32_t box[2] = {64, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(reinterpret_cast<CUtensorMap *>(out), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides,
+                    box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? 0 : 2;
+}
+
+bool gemm_tc_supported(int N, int K) { return N % tc::BN == 0 && K % tc::BK == 0; }
+int gemm_tc_box_rows_a() { return tc::BM; }
+int gemm_tc_box_rows_w() { return tc::BN; }
+
+template <int EPI>
+static cudaError_t tc_launch(const TensorMap128 &ta, const TensorMap128 &tw, const GemmArgs &a, int g, unsigned long long limit_ns,
+                             int *status, cudaStream_t st)
+{
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(tc::gemm_tc_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    tc::gemm_tc_kernel<EPI><<<g, tc::THREADS, tc::SMEM_BYTES, st>>>(*reinterpret_cast<const CUtensorMap *>(&ta),
+                                                                    *reinterpret_cast<const CUtensorMap *>(&tw), a, limit_ns, status);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gemm_tc(const TensorMap128 &ta, const TensorMap128 &tw, const GemmArgs &a, int grid, unsigned long long limit_ns,
+                           int *status, cudaStream_t st)
+{
+    if (a.M == 0) return cudaSuccess;
+    const int tiles = ((a.M + tc::BM - 1) / tc::BM) * (a.N / tc::BN);
+    const int g = tiles < grid ? tiles : grid;
+    switch (a.epi) {
+    case EPI_SCALE_STORE: return tc_launch<EPI_SCALE_STORE>(ta, tw, a, g, limit_ns, status, st);
+    case EPI_SCALE_GELU: return tc_launch<EPI_SCALE_GELU>(ta, tw, a, g, limit_ns, status, st);
+    default: return tc_launch<EPI_RESID>(ta, tw, a, g, limit_ns, status, st);
+    }
+}
+
+}  // namespace ebrl

@@ -48,6 +48,24 @@ def test_small_models_parity_ragged(dtype):
     assert chunk_rel_err(got, ref) <= TOL[dtype]
 
 
+def test_bf16_plain_alu_kernels_parity():
+    """The bf16 model on the plain-ALU kernels (the path taken when d is not a multiple of 256,
+    and on request)."""
+    w = synth.scaled(synth.WORKLOADS[0], B=19, dtype="bf16", d=128, n_heads=4, P=(3, 70), mixed_steps=True)
+    wt, envs = _setup(w)
+    ref = oracle_run(w, wt, envs)
+    r = Runner(w, wt, envs)
+    got = stack(r.run([list(range(w.B))]), range(w.B))
+    r.close()
+    assert chunk_rel_err(got, ref) <= TOL["bf16"]
+    w = synth.scaled(w, d=256)
+    wt, envs = _setup(w)
+    r = Runner(w, wt, envs, flags=B.FLAG_FORCE_SIMT)
+    got = stack(r.run([list(range(w.B))]), range(w.B))
+    r.close()
+    assert chunk_rel_err(got, oracle_run(w, wt, envs)) <= TOL["bf16"]
+
+
 def test_cfg1_model_bf16_parity_sample():
     """The mid-size bf16 head (d=1024, L=4, 16 heads, P=256, K=10) on a few environments."""
     w = synth.scaled(synth.WORKLOADS[1], B=6)
