@@ -226,7 +226,7 @@ def run_ours(args):
     noise = torch.stack([envs[e].noise for e in order]).contiguous()
     out = torch.empty_like(noise)
     kv_bytes = sum(envs[e].kv.numel() * envs[e].kv.element_size() for e in ids)
-    inflight = 4
+    inflight = 8
     flags = B.FLAG_FORCE_SIMT if args.simt else 0
     cfg = B.cfg_for(w, max_group_envs=max(len(g) for g in groups), max_inflight_groups=inflight, flags=flags, device=local)
     gen = B.ActGen(cfg, wt)

@@ -153,28 +153,37 @@ ebrl_status_t ebrl_actgen_create(const ebrl_actgen_cfg_t *cfg, const ebrl_actgen
  *   sm_quota   1..#SMs; 0 = all SMs.  Every kernel of this group runs as a persistent grid of
  *              at most sm_quota CTAs (at most one CTA's worth of SMs each), inside a green
  *              context of that many SMs when EBRL_FLAG_GREEN_CTX is set and available.
- *   stream     cudaStream_t of the caller (NULL = the legacy default stream).  The work is
- *              ordered after everything already on the stream; `out` is ready for work
- *              enqueued on the stream afterwards.
+ *   stream     cudaStream_t of the caller (NULL = the legacy default stream).
+ * Queueing (the bounded queue between simulation and generation, section 4.2.2): a submitted
+ * group waits in the handle until max_inflight_groups groups are queued, or a group for a
+ * different stream or quota arrives, or ebrl_actgen_flush / ebrl_actgen_sync is called; the
+ * queued groups are then launched on `stream` as ONE packed batch (their environments share
+ * the row space, so the weights stream once per Euler step for all of them).  The batch is
+ * ordered after everything on the stream at launch time, and every `out` of the batch is ready
+ * for work enqueued on the stream after the launch.  With max_inflight_groups = 1 every submit
+ * launches at once.  At most two batches are in flight; a further launch first waits for the
+ * older one.  Batching never changes an environment's result.
  * Host arrays are copied before the call returns.  Device buffers must stay valid and
- * unmodified until the group has completed (ebrl_actgen_sync, or a stream synchronisation).
- * If max_inflight_groups groups are already in flight the call first waits for the oldest
- * (the bounded queue between simulation and generation, section 4.2.2).  n_envs = 0 is a
- * no-op returning EBRL_OK. */
+ * unmodified until the group has completed (ebrl_actgen_sync, or ebrl_actgen_flush followed by
+ * a stream synchronisation).  n_envs = 0 is a no-op returning EBRL_OK. */
 ebrl_status_t ebrl_actgen_submit(ebrl_actgen_t h, int32_t n_envs, const int64_t *env_ids,
                                  const void *const *prefix_kv, const float *noise, float *out,
                                  int32_t sm_quota, void *stream, const ebrl_submit_ext_t *ext);
 
 /* The same with HOST buffers: prefix_kv[i], noise and out point to host memory (pinned memory
  * makes the copies asynchronous).  The planes and the noise are copied to device staging
- * owned by the handle, the group runs, and `out` is copied back, all on `stream`; `out` is
- * valid after ebrl_actgen_sync.  Needs prefix_len in ext, or every P_e = max_prefix_len. */
+ * owned by the handle when the call is made, the group runs with its batch, and `out` is
+ * copied back after the batch, all on `stream`; `out` is valid after ebrl_actgen_sync.  Needs prefix_len in ext, or every P_e = max_prefix_len. */
 ebrl_status_t ebrl_actgen_submit_host(ebrl_actgen_t h, int32_t n_envs, const int64_t *env_ids,
                                       const void *const *prefix_kv_host, const float *noise_host,
                                       float *out_host, int32_t sm_quota, void *stream,
                                       const ebrl_submit_ext_t *ext);
 
-/* Blocks until every submitted group has completed; returns the first sticky error. */
+/* Launches the queued groups now, without blocking. */
+ebrl_status_t ebrl_actgen_flush(ebrl_actgen_t h);
+
+/* Launches the queued groups, then blocks until every submitted group has completed; returns
+ * the first sticky error. */
 ebrl_status_t ebrl_actgen_sync(ebrl_actgen_t h);
 
 /* Syncs, then frees everything the handle owns. */

@@ -83,6 +83,7 @@ def lib():
         L.ebrl_actgen_submit.argtypes = sub
         L.ebrl_actgen_submit_host.argtypes = sub
         L.ebrl_actgen_sync.argtypes = [C.c_void_p]
+        L.ebrl_actgen_flush.argtypes = [C.c_void_p]
         L.ebrl_actgen_destroy.argtypes = [C.c_void_p]
         L.ebrl_actgen_get_stats.argtypes = [C.c_void_p, C.POINTER(Stats)]
         L.ebrl_actgen_reset_stats.argtypes = [C.c_void_p]
@@ -204,6 +205,9 @@ class ActGen:
         s = stream if stream is not None else torch.cuda.current_stream(self.cfg.device)
         self._submit(self._L.ebrl_actgen_submit_host, env_ids, kv_ptrs, noise.data_ptr(), out.data_ptr(), sm_quota,
                      s.cuda_stream, prefix_len, step_index, n_steps)
+
+    def flush(self):
+        self._check(self._L.ebrl_actgen_flush(self._h))
 
     def sync(self):
         self._check(self._L.ebrl_actgen_sync(self._h))

@@ -20,7 +20,9 @@ struct EnvMeta {
     int32_t P;         // prefix length
     int32_t k0;        // Euler step index the environment starts from
     int32_t nsteps;    // steps to run in this submit
-    int32_t src;       // index of the environment in the caller's noise/out arrays
+    int32_t pad_;
+    const float *noise;  // device: the environment's [H][A] state on entry
+    float *out;          // device: where its [H][A] result goes
 };
 
 enum Epilogue : int {
@@ -66,8 +68,7 @@ struct AttnArgs {
 
 struct EmbedArgs {
     const EnvMeta *meta;
-    int n_envs, H, A, d, s;        // s = inner step of this submit
-    const float *noise;            // caller's [n][H][A]
+    int n_envs, H, A, d, s;        // s = inner step of this batch
     const float *a_state;          // [rows][A]
     const void *w_in;              // [d][A] (TW)
     const float *temb;             // [K][d]
@@ -80,9 +81,7 @@ struct EmbedArgs {
 struct HeadArgs {
     const EnvMeta *meta;
     int n_envs, H, A, d, s, K;
-    const float *noise;
     float *a_state;
-    float *out;                    // caller's [n][H][A]
     const float *x;                // [rows][d]
     const float *gain;             // g_final
     const void *w_out;             // [A][d] (TW)
@@ -101,6 +100,10 @@ int gemm_tc_box_rows_a();
 int gemm_tc_box_rows_w();
 cudaError_t launch_gemm_tc(const TensorMap128 &ta, const TensorMap128 &tw, const GemmArgs &a, int grid,
                            unsigned long long limit_ns, int *status, cudaStream_t st);
+
+// Tensor-core (mma.sync) attention over bulk-copied K/V rows, bf16 models.
+bool attn_mma_supported(int H, int n_heads, int hd);
+cudaError_t launch_attn_mma(const AttnArgs &a, int grid, unsigned long long limit_ns, int *status, cudaStream_t st);
 
 // Launchers (plain-ALU kernels).  bf16 != 0 selects bf16 activations/weights/planes.
 // grid = number of persistent CTAs (the SM quota).

@@ -32,6 +32,12 @@ struct TimedLaunch {
     double flops, bytes;
 };
 
+struct HostCopy {
+    void *dst;
+    const void *src;
+    size_t bytes;
+};
+
 struct Slot {
     float *a_state = nullptr, *x = nullptr, *ssq = nullptr;
     void *xg = nullptr, *qkv = nullptr, *att = nullptr, *qc = nullptr, *u = nullptr;
@@ -46,6 +52,12 @@ struct Slot {
     float *noise_stage = nullptr, *out_stage = nullptr;
     std::vector<TimedLaunch> timed;
     size_t timed_used = 0;
+    // groups queued in this slot and not yet launched
+    std::vector<EnvMeta> pending;
+    std::vector<HostCopy> copies_out;
+    cudaStream_t stream = nullptr;
+    int grid = 0, groups_pending = 0;
+    size_t stage_used = 0, chunks_used = 0;
 };
 
 thread_local std::string g_create_error;
@@ -56,6 +68,7 @@ struct ebrl_actgen {
     ebrl_actgen_cfg_t cfg;
     int bf16 = 0, n_sms = 0, hd = 0, md = 0;
     bool use_tc = false;          // tensor-core GEMMs (bf16, d a multiple of 256)
+    bool use_attn_mma = false;    // tensor-core attention (bf16, H <= 16, head_dim 64/128)
     int *status_d = nullptr;      // device status word written by kernels whose waits ran out
     unsigned long long wait_ns = 0;
     size_t esz = 4;   // bytes per element of matrices / activations / planes
@@ -63,7 +76,7 @@ struct ebrl_actgen {
     float *b_out = nullptr, *g_final = nullptr, *temb = nullptr;
     std::vector<LayerDev> layers;
     std::vector<Slot> slots;
-    size_t next_slot = 0;
+    size_t fill = 0;              // slot collecting groups for the next batch
     std::unordered_set<int64_t> busy_ids;
     std::mutex mu;
     std::string err;
@@ -107,7 +120,8 @@ ebrl_status_t check_cfg(const ebrl_actgen_cfg_t *c, std::string *why)
     const int hd = c->d / c->n_heads;
     if (hd != 32 && hd != 64 && hd != 128) return bad(EBRL_ERR_UNSUPPORTED, "head_dim must be 32, 64 or 128");
     if (c->param_dtype != c->kv_dtype) return bad(EBRL_ERR_UNSUPPORTED, "param_dtype and kv_dtype must match");
-    if ((int64_t)c->max_group_envs * c->H > (int64_t)1 << 24) return bad(EBRL_ERR_UNSUPPORTED, "max_group_envs * H too large");
+    if ((int64_t)c->max_group_envs * c->max_inflight_groups * c->H > (int64_t)1 << 22)
+        return bad(EBRL_ERR_UNSUPPORTED, "max_group_envs * max_inflight_groups * H is limited to 4M rows");
     return EBRL_OK;
 }
 
@@ -254,9 +268,15 @@ struct Launcher {
     }
 };
 
-// Enqueues every kernel of one group on the stream.
-cudaError_t enqueue_group(ebrl_actgen *h, Slot &s, int n, int S, const int32_t *n_active, double sum_P_active[],
-                          const float *noise, float *out, int grid, cudaStream_t st)
+cudaError_t launch_attn(ebrl_actgen *h, const AttnArgs &a, int grid, cudaStream_t st)
+{
+    if (h->use_attn_mma) return launch_attn_mma(a, grid, h->wait_ns, h->status_d, st);
+    return launch_attn_simt(a, h->bf16, grid, st);
+}
+
+// Enqueues every kernel of one batch (the groups coalesced in one slot) on the stream.
+cudaError_t enqueue_batch(ebrl_actgen *h, Slot &s, int S, const int32_t *n_active, const double *sum_P_active, int grid,
+                          cudaStream_t st)
 {
     const ebrl_actgen_cfg_t &c = h->cfg;
     const int d = c.d, H = c.H, L = c.n_layers, md = h->md, bf = h->bf16;
@@ -264,12 +284,11 @@ cudaError_t enqueue_group(ebrl_actgen *h, Slot &s, int n, int S, const int32_t *
     const bool pull = (c.flags & EBRL_FLAG_TEST_PULL) != 0;
     const double esz = (double)h->esz;
     Launcher ln{h, &s, st, grid, (c.flags & EBRL_FLAG_TIMING) != 0};
-    (void)n;
     for (int step = 0; step < S; ++step) {
         const int ne = n_active[step], M = ne * H;
         if (ne == 0) break;
         if (!pull) {
-            EmbedArgs ea{s.meta_d, ne, H, c.A, d, step, noise, s.a_state, h->w_in, h->temb,
+            EmbedArgs ea{s.meta_d, ne, H, c.A, d, step, s.a_state, h->w_in, h->temb,
                          L > 0 ? h->layers[0].g1 : h->g_final, s.x, s.xg, s.ssq};
             ln.run(EBRL_KC_EMBED, 2.0 * M * d * c.A, (double)M * d * (4 + esz), [&] { return launch_embed(ea, bf, grid, st); });
             for (int l = 0; l < L; ++l) {
@@ -296,7 +315,7 @@ cudaError_t enqueue_group(ebrl_actgen *h, Slot &s, int n, int S, const int32_t *
                     a.k_self = (const char *)s.qkv + (size_t)d * h->esz;
                     a.v_self = (const char *)s.qkv + (size_t)2 * d * h->esz;
                     a.kv_stride = 3 * d;
-                    ln.run(EBRL_KC_SELF_ATTN, 4.0 * M * H * d, 4.0 * M * d * esz, [&] { return launch_attn_simt(a, bf, grid, st); });
+                    ln.run(EBRL_KC_SELF_ATTN, 4.0 * M * H * d, 4.0 * M * d * esz, [&] { return launch_attn(h, a, grid, st); });
                 }
                 gemm(s.att, s.t_att, w.w_o, w.t_o, d, d, EPI_RESID, nullptr, w.g2);
                 // cross-attention block
@@ -307,8 +326,7 @@ cudaError_t enqueue_group(ebrl_actgen *h, Slot &s, int n, int S, const int32_t *
                     a.H = H; a.n_heads = c.n_heads; a.hd = h->hd; a.n_envs = ne; a.d = d;
                     a.meta = s.meta_d; a.kv_plane = (c.kv_layers == 1) ? 0 : l; a.self = 0;
                     ln.run(EBRL_KC_CROSS_ATTN, 4.0 * H * sum_P_active[step] * d,
-                           2.0 * sum_P_active[step] * d * esz + 2.0 * M * d * esz,
-                           [&] { return launch_attn_simt(a, bf, grid, st); });
+                           2.0 * sum_P_active[step] * d * esz + 2.0 * M * d * esz, [&] { return launch_attn(h, a, grid, st); });
                 }
                 gemm(s.att, s.t_att, w.w_oc, w.t_oc, d, d, EPI_RESID, nullptr, w.g3);
                 // MLP block
@@ -316,11 +334,47 @@ cudaError_t enqueue_group(ebrl_actgen *h, Slot &s, int n, int S, const int32_t *
                 gemm(s.u, s.t_u, w.w_2, w.t_2, d, md, EPI_RESID, nullptr, (l + 1 < L) ? h->layers[l + 1].g1 : h->g_final);
             }
         }
-        HeadArgs ha{s.meta_d, ne, H, c.A, d, step, c.K_steps, noise, s.a_state, out, s.x, h->g_final,
-                    h->w_out, h->b_out, c.rms_eps, pull ? 1 : 0};
+        HeadArgs ha{s.meta_d, ne, H, c.A, d, step, c.K_steps, s.a_state, s.x, h->g_final, h->w_out, h->b_out, c.rms_eps, pull ? 1 : 0};
         ln.run(EBRL_KC_HEAD, 2.0 * M * d * c.A, (double)M * d * 4, [&] { return launch_head(ha, bf, grid, st); });
     }
     return ln.err;
+}
+
+// Launches the groups waiting in a slot as ONE packed batch: their environments share the row
+// space, so weights stream once per step for all of them.  Rows are independent in every
+// kernel, hence the result of an environment does not depend on what it is batched with.
+ebrl_status_t flush_slot(ebrl_actgen *h, Slot &s)
+{
+    if (s.pending.empty()) return EBRL_OK;
+    const ebrl_actgen_cfg_t &c = h->cfg;
+    const int n = (int)s.pending.size();
+    cudaStream_t cs = s.stream;
+    // the batcher's plan over the whole batch: longest-running environments first
+    std::vector<int32_t> order(n);
+    for (int i = 0; i < n; ++i) order[i] = i;
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return s.pending[a].nsteps > s.pending[b].nsteps; });
+    std::vector<int32_t> n_active(c.K_steps, 0);
+    std::vector<double> sum_P(c.K_steps, 0.0);
+    int S = 0;
+    for (int j = 0; j < n; ++j) {
+        const EnvMeta &m = s.pending[order[j]];
+        s.meta_h[j] = m;
+        S = std::max(S, (int)m.nsteps);
+        for (int t = 0; t < m.nsteps; ++t) { n_active[t] += 1; sum_P[t] += m.P; }
+    }
+    s.pending.clear();
+    CK(cudaMemcpyAsync(s.meta_d, s.meta_h, sizeof(EnvMeta) * (size_t)n, cudaMemcpyHostToDevice, cs));
+    cudaError_t e = enqueue_batch(h, s, S, n_active.data(), sum_P.data(), s.grid, cs);
+    if (e != cudaSuccess) {
+        h->sticky = EBRL_ERR_CUDA;
+        return fail(h, EBRL_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
+    }
+    for (const HostCopy &hc : s.copies_out) CK(cudaMemcpyAsync(hc.dst, hc.src, hc.bytes, cudaMemcpyDeviceToHost, cs));
+    s.copies_out.clear();
+    CK(cudaEventRecord(s.done, cs));
+    s.busy = true;
+    h->fill = (h->fill + 1) % h->slots.size();
+    return EBRL_OK;
 }
 
 ebrl_status_t submit_impl(ebrl_actgen *h, int32_t n, const int64_t *env_ids, const void *const *prefix_kv,
@@ -338,43 +392,57 @@ ebrl_status_t submit_impl(ebrl_actgen *h, int32_t n, const int64_t *env_ids, con
     CK(cudaSetDevice(h->cfg.device));
 
     const ebrl_actgen_cfg_t &c = h->cfg;
-    Slot &s = h->slots[h->next_slot];
-    h->next_slot = (h->next_slot + 1) % h->slots.size();
-    st = retire(h, s);   // bounded queue: wait for the oldest group when every slot is taken
-    if (st != EBRL_OK) return st;
-
     cudaStream_t cs = (cudaStream_t)stream;
     const int grid = sm_quota == 0 ? h->n_sms : sm_quota;
+    // groups queue in the slot being filled; a group for another stream or quota closes the batch
+    if (!h->slots[h->fill].pending.empty() && (h->slots[h->fill].stream != cs || h->slots[h->fill].grid != grid))
+        if ((st = flush_slot(h, h->slots[h->fill])) != EBRL_OK) return st;
+    Slot &s = h->slots[h->fill];
+    if (s.pending.empty()) {
+        // bounded queue: a slot is reused only after its previous batch has completed
+        if ((st = retire(h, s)) != EBRL_OK) return st;
+        s.stream = cs; s.grid = grid; s.groups_pending = 0; s.stage_used = 0; s.chunks_used = 0;
+    }
     const bool pull = (c.flags & EBRL_FLAG_TEST_PULL) != 0;
     const size_t chunk = (size_t)c.H * c.A;
+    const int K = c.K_steps;
 
-    std::vector<int32_t> order(n), nsteps(n), n_active(c.K_steps);
-    const int S = plan_group(&c, n, ext, order.data(), nsteps.data(), n_active.data());
-
-    // host-buffer variant: stage planes, noise and out on the device
     const float *noise_d = noise;
     float *out_d = out;
     std::vector<const void *> kv_dev(n, nullptr);
     if (host_buffers) {
-        size_t total = 0;
+        // stage planes, noise and out on the device (staging belongs to the slot)
+        size_t need = s.stage_used;
         std::vector<size_t> off(n);
         for (int i = 0; i < n; ++i) {
             const int P = (ext && ext->prefix_len) ? ext->prefix_len[i] : c.max_prefix_len;
-            off[i] = total;
-            total += ((size_t)c.kv_layers * 2 * P * c.d * h->esz + 255) & ~(size_t)255;
+            off[i] = need;
+            need += ((size_t)c.kv_layers * 2 * P * c.d * h->esz + 255) & ~(size_t)255;
         }
-        if (!pull && s.kv_stage_bytes < total) {
+        if (!pull && s.kv_stage_bytes < need) {
+            if (s.stage_used != 0) {   // staging already referenced by queued groups: close the batch first
+                if ((st = flush_slot(h, s)) != EBRL_OK) return st;
+                return submit_impl(h, n, env_ids, prefix_kv, noise, out, sm_quota, stream, ext, host_buffers);
+            }
             if (s.kv_stage) cudaFree(s.kv_stage);
             s.kv_stage = nullptr; s.kv_stage_bytes = 0;
-            cudaError_t e = cudaMalloc((void **)&s.kv_stage, total);
-            if (e != cudaSuccess) { cudaGetLastError(); return fail(h, EBRL_ERR_NOMEM, "staging of %zu bytes: %s", total, cudaGetErrorString(e)); }
-            s.kv_stage_bytes = total;
+            const size_t want = (size_t)c.max_inflight_groups * need;   // room for a whole batch of such groups
+            cudaError_t e = cudaMalloc((void **)&s.kv_stage, want);
+            if (e != cudaSuccess) {
+                cudaGetLastError();
+                e = cudaMalloc((void **)&s.kv_stage, need);
+                if (e != cudaSuccess) { cudaGetLastError(); return fail(h, EBRL_ERR_NOMEM, "staging of %zu bytes: %s", need, cudaGetErrorString(e)); }
+                s.kv_stage_bytes = need;
+            } else {
+                s.kv_stage_bytes = want;
+            }
         }
         if (!s.noise_stage) {
             void *p = nullptr;
-            if ((st = dev_alloc(h, &p, (size_t)c.max_group_envs * chunk * 4)) != EBRL_OK) return st;
+            const size_t cap = (size_t)c.max_inflight_groups * c.max_group_envs * chunk * 4;
+            if ((st = dev_alloc(h, &p, cap)) != EBRL_OK) return st;
             s.noise_stage = (float *)p;
-            if ((st = dev_alloc(h, &p, (size_t)c.max_group_envs * chunk * 4)) != EBRL_OK) return st;
+            if ((st = dev_alloc(h, &p, cap)) != EBRL_OK) return st;
             s.out_stage = (float *)p;
         }
         if (!pull)
@@ -383,43 +451,39 @@ ebrl_status_t submit_impl(ebrl_actgen *h, int32_t n, const int64_t *env_ids, con
                 CK(cudaMemcpyAsync(s.kv_stage + off[i], prefix_kv[i], (size_t)c.kv_layers * 2 * P * c.d * h->esz, cudaMemcpyHostToDevice, cs));
                 kv_dev[i] = s.kv_stage + off[i];
             }
-        CK(cudaMemcpyAsync(s.noise_stage, noise, (size_t)n * chunk * 4, cudaMemcpyHostToDevice, cs));
-        noise_d = s.noise_stage;
-        out_d = s.out_stage;
+        s.stage_used = need;
+        noise_d = s.noise_stage + s.chunks_used * chunk;
+        out_d = s.out_stage + s.chunks_used * chunk;
+        CK(cudaMemcpyAsync((void *)noise_d, noise, (size_t)n * chunk * 4, cudaMemcpyHostToDevice, cs));
+        s.copies_out.push_back(HostCopy{out, out_d, (size_t)n * chunk * 4});
+        s.chunks_used += (size_t)n;
     } else if (!pull) {
         for (int i = 0; i < n; ++i) kv_dev[i] = prefix_kv[i];
     }
 
-    std::vector<double> sum_P(c.K_steps, 0.0);
     uint64_t env_steps = 0;
-    for (int j = 0; j < n; ++j) {
-        const int i = order[j];
-        EnvMeta &m = s.meta_h[j];
+    for (int i = 0; i < n; ++i) {
+        EnvMeta m{};
         m.kv = kv_dev[i];
         m.P = (ext && ext->prefix_len) ? ext->prefix_len[i] : c.max_prefix_len;
         m.k0 = (ext && ext->step_index) ? ext->step_index[i] : 0;
-        m.nsteps = nsteps[j];
-        m.src = i;
-        env_steps += (uint64_t)nsteps[j];
-        for (int t = 0; t < nsteps[j]; ++t) sum_P[t] += m.P;
+        int ns = K - m.k0;
+        if (ext && ext->n_steps > 0 && ext->n_steps < ns) ns = ext->n_steps;
+        m.nsteps = ns;
+        m.noise = noise_d + (size_t)i * chunk;
+        m.out = out_d + (size_t)i * chunk;
+        s.pending.push_back(m);
+        env_steps += (uint64_t)ns;
+        s.ids.push_back(env_ids[i]);
+        h->busy_ids.insert(env_ids[i]);
     }
-    CK(cudaMemcpyAsync(s.meta_d, s.meta_h, sizeof(EnvMeta) * (size_t)n, cudaMemcpyHostToDevice, cs));
-
-    cudaError_t e = enqueue_group(h, s, n, S, n_active.data(), sum_P.data(), noise_d, out_d, grid, cs);
-    if (e != cudaSuccess) {
-        h->sticky = EBRL_ERR_CUDA;
-        return fail(h, EBRL_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
-    }
-    if (host_buffers) CK(cudaMemcpyAsync(out, s.out_stage, (size_t)n * chunk * 4, cudaMemcpyDeviceToHost, cs));
-    CK(cudaEventRecord(s.done, cs));
-    s.busy = true;
-    s.ids.assign(env_ids, env_ids + n);
-    for (int i = 0; i < n; ++i) h->busy_ids.insert(env_ids[i]);
+    s.groups_pending += 1;
     h->stats.groups += 1;
     h->stats.envs += (uint64_t)n;
     h->stats.env_steps += env_steps;
     h->stats.granted_sms = grid;
     h->stats.green_ctx_active = 0;
+    if (s.groups_pending >= c.max_inflight_groups) return flush_slot(h, s);
     return EBRL_OK;
 }
 
@@ -541,7 +605,10 @@ ebrl_status_t ebrl_actgen_create(const ebrl_actgen_cfg_t *cfg, const ebrl_actgen
         }
         if ((st = dev_copy_in(h, (void **)&h->temb, t.data(), t.size() * 4)) != EBRL_OK) return bail(st);
     }
-    const size_t rows = (size_t)cfg->max_group_envs * cfg->H;
+    // a batch holds up to max_inflight_groups groups; two batch slots let the host queue the
+    // next batch while the previous one runs
+    const size_t batch_envs = (size_t)cfg->max_inflight_groups * cfg->max_group_envs;
+    const size_t rows = batch_envs * cfg->H;
     h->wait_ns = cfg->wait_limit_ns ? cfg->wait_limit_ns : 4000000000ull;
     {
         void *p = nullptr;
@@ -551,6 +618,7 @@ ebrl_status_t ebrl_actgen_create(const ebrl_actgen_cfg_t *cfg, const ebrl_actgen
     }
     h->use_tc = h->bf16 && !(cfg->flags & EBRL_FLAG_FORCE_SIMT) && gemm_tc_supported(d, d) && gemm_tc_supported(md, d) &&
                 gemm_tc_supported(d, md) && gemm_tc_supported(3 * d, d);
+    h->use_attn_mma = h->bf16 && !(cfg->flags & EBRL_FLAG_FORCE_SIMT) && attn_mma_supported(cfg->H, cfg->n_heads, h->hd);
     if (h->use_tc) {
         const uint32_t bw = (uint32_t)gemm_tc_box_rows_w();
         int bad = 0;
@@ -565,7 +633,7 @@ ebrl_status_t ebrl_actgen_create(const ebrl_actgen_cfg_t *cfg, const ebrl_actgen
         }
         if (bad) { fail(h, EBRL_ERR_CUDA, "cuTensorMapEncodeTiled failed for a weight matrix"); return bail(EBRL_ERR_CUDA); }
     }
-    h->slots.resize(cfg->max_inflight_groups);
+    h->slots.resize(2);
     for (Slot &s : h->slots) {
         void *p = nullptr;
         if ((st = dev_alloc(h, &p, rows * A * 4)) != EBRL_OK) return bail(st); s.a_state = (float *)p;
@@ -576,8 +644,8 @@ ebrl_status_t ebrl_actgen_create(const ebrl_actgen_cfg_t *cfg, const ebrl_actgen
         if ((st = dev_alloc(h, &s.att, rows * d * esz)) != EBRL_OK) return bail(st);
         if ((st = dev_alloc(h, &s.qc, rows * d * esz)) != EBRL_OK) return bail(st);
         if ((st = dev_alloc(h, &s.u, rows * md * esz)) != EBRL_OK) return bail(st);
-        if ((st = dev_alloc(h, &p, sizeof(EnvMeta) * (size_t)cfg->max_group_envs)) != EBRL_OK) return bail(st); s.meta_d = (EnvMeta *)p;
-        if (cudaMallocHost((void **)&s.meta_h, sizeof(EnvMeta) * (size_t)cfg->max_group_envs) != cudaSuccess) {
+        if ((st = dev_alloc(h, &p, sizeof(EnvMeta) * batch_envs)) != EBRL_OK) return bail(st); s.meta_d = (EnvMeta *)p;
+        if (cudaMallocHost((void **)&s.meta_h, sizeof(EnvMeta) * batch_envs) != cudaSuccess) {
             cudaGetLastError();
             fail(h, EBRL_ERR_NOMEM, "pinned staging allocation failed");
             return bail(EBRL_ERR_NOMEM);
@@ -616,14 +684,22 @@ ebrl_status_t ebrl_actgen_submit_host(ebrl_actgen_t h, int32_t n, const int64_t 
     return submit_impl(h, n, env_ids, prefix_kv_host, noise_host, out_host, sm_quota, stream, ext, true);
 }
 
+ebrl_status_t ebrl_actgen_flush(ebrl_actgen_t h)
+{
+    if (!h) return EBRL_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lk(h->mu);
+    if (cudaSetDevice(h->cfg.device) != cudaSuccess) return fail(h, EBRL_ERR_CUDA, "cudaSetDevice failed");
+    return flush_slot(h, h->slots[h->fill]);
+}
+
 ebrl_status_t ebrl_actgen_sync(ebrl_actgen_t h)
 {
     if (!h) return EBRL_ERR_INVALID_ARG;
     std::lock_guard<std::mutex> lk(h->mu);
     if (cudaSetDevice(h->cfg.device) != cudaSuccess) return fail(h, EBRL_ERR_CUDA, "cudaSetDevice failed");
-    ebrl_status_t first = EBRL_OK;
+    ebrl_status_t first = flush_slot(h, h->slots[h->fill]);
     for (size_t i = 0; i < h->slots.size(); ++i) {
-        Slot &s = h->slots[(h->next_slot + i) % h->slots.size()];
+        Slot &s = h->slots[(h->fill + i) % h->slots.size()];
         ebrl_status_t st = retire(h, s);
         if (st != EBRL_OK && first == EBRL_OK) first = st;
     }
@@ -645,7 +721,7 @@ ebrl_status_t ebrl_actgen_destroy(ebrl_actgen_t h)
     {
         std::lock_guard<std::mutex> lk(h->mu);
         cudaSetDevice(h->cfg.device);
-        st = EBRL_OK;
+        st = flush_slot(h, h->slots[h->fill]);
         for (Slot &s : h->slots) { ebrl_status_t r = retire(h, s); if (r != EBRL_OK && st == EBRL_OK) st = r; }
         free_all(h);
     }

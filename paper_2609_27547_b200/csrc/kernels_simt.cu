@@ -31,46 +31,43 @@ __device__ __forceinline__ float warp_max(float v)
 __device__ __forceinline__ float gelu_erf(float z) { return 0.5f * z * (1.0f + erff(z * 0.70710678118654752440f)); }
 
 // ---------------------------------------------------------------------------------------
-// x = W_in a + temb(t_k); xg = x * gain; sum-of-squares partials.  One row per CTA pass.
+// x = W_in a + temb(t_k); xg = x * gain; sum-of-squares partials.  One warp per (row, 128-column
+// segment); the row's action vector lives in the lanes and is broadcast by shuffles.
 // ---------------------------------------------------------------------------------------
 template <typename T>
-__global__ void __launch_bounds__(256) embed_kernel(EmbedArgs a)
+__global__ void __launch_bounds__(1024) embed_kernel(EmbedArgs a)
 {
-    __shared__ float sa[32];
-    const int rows = a.n_envs * a.H, nseg = a.d / SSQ_W;
+    const int rows = a.n_envs * a.H, nseg = a.d / SSQ_W, units = rows * nseg;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const T *w_in = (const T *)a.w_in;
     T *xg = (T *)a.xg;
-    for (int row = blockIdx.x; row < rows; row += gridDim.x) {
+    for (int u = blockIdx.x * 32 + warp; u < units; u += gridDim.x * 32) {
+        const int row = u / nseg, seg = u - row * nseg;
         const int env = row / a.H, h = row - env * a.H;
         const EnvMeta m = a.meta[env];
         const int k = m.k0 + a.s;
-        const float *av = (a.s == 0) ? a.noise + ((size_t)m.src * a.H + h) * a.A : a.a_state + (size_t)row * a.A;
-        if (threadIdx.x < a.A) sa[threadIdx.x] = av[threadIdx.x];
-        __syncthreads();
-        for (int seg = warp; seg < nseg; seg += 8) {
-            float ss = 0.f;
+        const float *av = (a.s == 0) ? m.noise + (size_t)h * a.A : a.a_state + (size_t)row * a.A;
+        const float mine = lane < a.A ? av[lane] : 0.f;
+        float ss = 0.f;
 #pragma unroll
-            for (int i = 0; i < SSQ_W / 32; ++i) {
-                const int c = seg * SSQ_W + i * 32 + lane;
-                float acc = 0.f;
-                for (int j = 0; j < a.A; ++j) acc = fmaf(ldf(w_in + (size_t)c * a.A + j), sa[j], acc);
-                acc += a.temb[(size_t)k * a.d + c];
-                a.x[(size_t)row * a.d + c] = acc;
-                stf(xg + (size_t)row * a.d + c, acc * a.gain[c]);
-                ss = fmaf(acc, acc, ss);
-            }
-            ss = warp_sum(ss);
-            if (lane == 0) a.ssq[(size_t)row * nseg + seg] = ss;
+        for (int i = 0; i < SSQ_W / 32; ++i) {
+            const int c = seg * SSQ_W + i * 32 + lane;
+            float acc = 0.f;
+            for (int j = 0; j < a.A; ++j) acc = fmaf(ldf(w_in + (size_t)c * a.A + j), __shfl_sync(0xffffffffu, mine, j), acc);
+            acc += a.temb[(size_t)k * a.d + c];
+            a.x[(size_t)row * a.d + c] = acc;
+            stf(xg + (size_t)row * a.d + c, acc * a.gain[c]);
+            ss = fmaf(acc, acc, ss);
         }
-        __syncthreads();
+        ss = warp_sum(ss);
+        if (lane == 0) a.ssq[(size_t)row * nseg + seg] = ss;
     }
 }
 
 // ---------------------------------------------------------------------------------------
 // v = W_out RMSNorm(x; g_final) + b_out;  a += v / K.  One warp per row.
 // ---------------------------------------------------------------------------------------
-template <typename T>
+template <typename T, int AMAX>
 __global__ void __launch_bounds__(256) head_kernel(HeadArgs a)
 {
     const int rows = a.n_envs * a.H;
@@ -80,9 +77,9 @@ __global__ void __launch_bounds__(256) head_kernel(HeadArgs a)
         const int env = row / a.H, h = row - env * a.H;
         const EnvMeta m = a.meta[env];
         const float *xr = a.x + (size_t)row * a.d;
-        float acc[32];
+        float acc[AMAX];
 #pragma unroll
-        for (int j = 0; j < 32; ++j) acc[j] = 0.f;
+        for (int j = 0; j < AMAX; ++j) acc[j] = 0.f;
         float ss = 0.f;
         if (!a.pull) {
             for (int c = lane; c < a.d; c += 32) {
@@ -90,15 +87,15 @@ __global__ void __launch_bounds__(256) head_kernel(HeadArgs a)
                 ss = fmaf(xv, xv, ss);
                 const float t = xv * a.gain[c];
 #pragma unroll
-                for (int j = 0; j < 32; ++j)
+                for (int j = 0; j < AMAX; ++j)
                     if (j < a.A) acc[j] = fmaf(t, ldf(w_out + (size_t)j * a.d + c), acc[j]);
             }
             ss = warp_sum(ss);
         }
         const float inv = 1.0f / sqrtf(ss / (float)a.d + a.eps);
-        const float *a_old = (a.s == 0) ? a.noise + ((size_t)m.src * a.H + h) * a.A : a.a_state + (size_t)row * a.A;
+        const float *a_old = (a.s == 0) ? m.noise + (size_t)h * a.A : a.a_state + (size_t)row * a.A;
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
+        for (int j = 0; j < AMAX; ++j) {
             if (j < a.A) {
                 const float dot = warp_sum(acc[j]);
                 if (lane == 0) {
@@ -106,7 +103,7 @@ __global__ void __launch_bounds__(256) head_kernel(HeadArgs a)
                     const float v = a.pull ? (a.b_out[j] - ao) : (dot * inv + a.b_out[j]);
                     const float an = ao + v / (float)a.K;
                     a.a_state[(size_t)row * a.A + j] = an;
-                    if (a.s == m.nsteps - 1) a.out[((size_t)m.src * a.H + h) * a.A + j] = an;
+                    if (a.s == m.nsteps - 1) m.out[(size_t)h * a.A + j] = an;
                 }
             }
         }
@@ -348,12 +345,21 @@ __global__ void __launch_bounds__(512) attn_simt_kernel(AttnArgs a)
 // ---------------------------------------------------------------------------------------
 cudaError_t launch_embed(const EmbedArgs &a, int bf16, int grid, cudaStream_t st)
 {
-    const int rows = a.n_envs * a.H;
-    if (rows == 0) return cudaSuccess;
-    const int g = rows < grid ? rows : grid;
-    if (bf16) embed_kernel<__nv_bfloat16><<<g, 256, 0, st>>>(a);
-    else embed_kernel<float><<<g, 256, 0, st>>>(a);
+    const int units = a.n_envs * a.H * (a.d / SSQ_W);
+    if (units == 0) return cudaSuccess;
+    const int need = (units + 31) / 32;
+    const int g = need < grid ? need : grid;
+    if (bf16) embed_kernel<__nv_bfloat16><<<g, 1024, 0, st>>>(a);
+    else embed_kernel<float><<<g, 1024, 0, st>>>(a);
     return cudaGetLastError();
+}
+
+template <typename T>
+static void head_dispatch(const HeadArgs &a, int g, cudaStream_t st)
+{
+    if (a.A <= 8) head_kernel<T, 8><<<g, 256, 0, st>>>(a);
+    else if (a.A <= 16) head_kernel<T, 16><<<g, 256, 0, st>>>(a);
+    else head_kernel<T, 32><<<g, 256, 0, st>>>(a);
 }
 
 cudaError_t launch_head(const HeadArgs &a, int bf16, int grid, cudaStream_t st)
@@ -362,8 +368,8 @@ cudaError_t launch_head(const HeadArgs &a, int bf16, int grid, cudaStream_t st)
     if (rows == 0) return cudaSuccess;
     const int need = (rows + 7) / 8;
     const int g = need < grid ? need : grid;
-    if (bf16) head_kernel<__nv_bfloat16><<<g, 256, 0, st>>>(a);
-    else head_kernel<float><<<g, 256, 0, st>>>(a);
+    if (bf16) head_dispatch<__nv_bfloat16>(a, g, st);
+    else head_dispatch<float>(a, g, st);
     return cudaGetLastError();
 }
 
