@@ -201,6 +201,31 @@ ebrl_status_t ebrl_actgen_set_timing(ebrl_actgen_t h, int32_t on);
 
 uint32_t ebrl_actgen_abi_version(void);
 
+/* ---- an entry point that allocates nothing ---------------------------------------------
+ * (The paper has no counterpart; this serves callers that cannot call cudaMalloc.)
+ * One Euler step of a layer-less action head on n_rows action tokens:
+ *     x = W_in a + temb_row;  v = W_out RMSNorm(x; g_final) + b_out;  a_out = a_in + v / K_steps
+ * -- what ebrl_actgen_submit computes for an n_layers = 0, fp32 model advanced by one step --
+ * for callers that may not allocate device memory at this point: a control loop that must not
+ * take the allocator's lock or risk its implicit synchronisation, a worker whose whole memory
+ * budget was handed out at start-up, a plug-in that is only given pointers and a stream.
+ * All pointers are DEVICE memory owned by the caller, fp32: a_in/a_out [n_rows][A] (may be the
+ * same buffer), w_in [d][A], w_out [A][d], b_out [A], g_final [d], temb_row [d] (the timestep
+ * embedding of this step).  The intermediate x is kept in a fixed 2 MiB array that is part of
+ * the library image on every GPU that loads it, so the call never calls cudaMalloc, cudaFree
+ * or any allocating routine.  Limits: n_rows <= 512, d <= 1024 and a multiple of 128, A <= 32;
+ * larger sizes return EBRL_ERR_UNSUPPORTED.  sm_quota as in submit (0 = all SMs).
+ * The first call on a device looks up the array's device address (with that device current,
+ * which must be the device of `stream`); make that first call outside any stream capture.
+ * All calls share the one array and it keeps the previous call's contents: nothing in it needs
+ * clearing (every row used is written before it is read), but two calls whose kernels overlap
+ * on the GPU (different streams) race on it -- order them on one stream or with events.
+ * The work is asynchronous on `stream`. */
+ebrl_status_t ebrl_actgen_l0_step_noalloc(const float *a_in, float *a_out, const float *w_in, const float *w_out,
+                                          const float *b_out, const float *g_final, const float *temb_row,
+                                          int32_t n_rows, int32_t A, int32_t d, int32_t K_steps, float rms_eps,
+                                          int32_t sm_quota, void *stream);
+
 /* ---- host-only helpers (no device needed): the argument rules and the batcher's plan ------
  * ebrl_actgen_check_cfg / check_submit apply exactly the checks create / submit apply before
  * touching the device (n_sms = the SM count to check the quota against) and return the same

@@ -95,6 +95,7 @@ def lib():
         L.ebrl_actgen_plan_group.argtypes = [C.POINTER(Cfg), C.c_int32, C.POINTER(SubmitExt),
                                              C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         L.ebrl_actgen_plan_group.restype = C.c_int32
+        L.ebrl_actgen_l0_step_noalloc.argtypes = [C.c_void_p] * 7 + [C.c_int32] * 4 + [C.c_float, C.c_int32, C.c_void_p]
         L.ebrl_sim_corunner_launch.argtypes = [C.c_void_p, C.c_uint64, C.c_int32, C.c_int32, C.c_void_p]
         _lib = L
     return _lib
@@ -238,6 +239,24 @@ class ActGen:
             self.destroy()
         except Exception:
             pass
+
+
+def l0_step_noalloc(a_in: torch.Tensor, a_out: torch.Tensor, w_in: torch.Tensor, w_out: torch.Tensor,
+                    b_out: torch.Tensor, g_final: torch.Tensor, temb_row: torch.Tensor, K_steps: int,
+                    rms_eps: float = 1e-6, sm_quota: int = 0, stream: Optional[torch.cuda.Stream] = None) -> int:
+    """``ebrl_actgen_l0_step_noalloc``: one Euler step of a layer-less fp32 head for callers that
+    cannot allocate device memory; all tensors are the caller's CUDA fp32 tensors.  Returns the
+    status code (0 = OK) instead of raising so that a caller can test the size limits."""
+    ts = (a_in, a_out, w_in, w_out, b_out, g_final, temb_row)
+    for t in ts:
+        if t.device.type != "cuda" or t.dtype != torch.float32 or not t.is_contiguous():
+            raise ValueError("contiguous CUDA fp32 tensors required")
+    n_rows, A = a_in.shape[-2] * (a_in.shape[0] if a_in.dim() == 3 else 1), a_in.shape[-1]
+    d = w_in.shape[0]
+    s = stream if stream is not None else torch.cuda.current_stream(a_in.device)
+    with torch.cuda.device(a_in.device):
+        return int(lib().ebrl_actgen_l0_step_noalloc(*[t.data_ptr() for t in ts], n_rows, A, d, K_steps, rms_eps,
+                                                     sm_quota, s.cuda_stream))
 
 
 def sim_corunner_launch(buf: torch.Tensor, n_steps: int, n_ctas: int, stream: torch.cuda.Stream):
