@@ -66,6 +66,8 @@ def parse_args():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--corunner", action="store_true", help="run the streaming co-runner on the other SMs")
     ap.add_argument("--simt", action="store_true", help="force the plain-ALU kernels")
+    ap.add_argument("--min-warmup", type=int, default=3, help="lower bound on warm-up steps (profiling captures use 1)")
+    ap.add_argument("--inflight", type=int, default=8, help="groups queued before a batch is launched")
     return ap.parse_args()
 
 
@@ -226,7 +228,7 @@ def run_ours(args):
     noise = torch.stack([envs[e].noise for e in order]).contiguous()
     out = torch.empty_like(noise)
     kv_bytes = sum(envs[e].kv.numel() * envs[e].kv.element_size() for e in ids)
-    inflight = 8
+    inflight = args.inflight
     flags = B.FLAG_FORCE_SIMT if args.simt else 0
     cfg = B.cfg_for(w, max_group_envs=max(len(g) for g in groups), max_inflight_groups=inflight, flags=flags, device=local)
     gen = B.ActGen(cfg, wt)
@@ -249,7 +251,8 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize(dev)
 
-    for _ in range(max(3, args.warmup)):
+    n_warm = max(args.min_warmup, args.warmup)
+    for _ in range(n_warm):
         step()
     gen.reset_stats()
     barrier()
@@ -354,7 +357,7 @@ def run_ours(args):
     gen.destroy()
     if rank == 0:
         line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": n_warm,
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16" if bf16 else "f32", "data": "synthetic",
             "config": {"workload": "configs[%d] %s" % (args.config, w.name), "envs_per_gpu": w.B, "H": w.H, "A": w.A, "d": w.d,

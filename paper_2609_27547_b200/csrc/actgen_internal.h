@@ -25,6 +25,9 @@ struct EnvMeta {
     float *out;          // device: where its [H][A] result goes
 };
 
+// Opaque storage of a CUtensorMap (the driver's 128-byte TMA descriptor).
+struct alignas(64) TensorMap128 { uint64_t opaque[16]; };
+
 enum Epilogue : int {
     EPI_SCALE_STORE = 0,   // C = acc * rowscale
     EPI_SCALE_GELU = 1,    // C = gelu(acc * rowscale)
@@ -64,6 +67,9 @@ struct AttnArgs {
     const void *k_self;    // [rows][kv_stride]
     const void *v_self;
     int kv_stride;
+    // tensor-core kernel: TMA descriptors (device memory)
+    const TensorMap128 *kv_maps;   // [n_envs]: the environment's planes as [kv_layers*2*P][d]
+    const TensorMap128 *self_map;  // the QKV buffer as [rows][3d]
 };
 
 struct EmbedArgs {
@@ -90,9 +96,6 @@ struct HeadArgs {
     int pull;                      // v = b_out - a
 };
 
-// Opaque storage of a CUtensorMap (the driver's 128-byte TMA descriptor).
-struct alignas(64) TensorMap128 { uint64_t opaque[16]; };
-
 // Tensor-core GEMM (bf16 operands, fp32 accumulation in tensor memory).
 int make_tmap_bf16(TensorMap128 *out, const void *base, uint64_t inner, uint64_t rows, uint32_t box_rows);
 bool gemm_tc_supported(int N, int K);
@@ -103,6 +106,7 @@ cudaError_t launch_gemm_tc(const TensorMap128 &ta, const TensorMap128 &tw, const
 
 // Tensor-core (mma.sync) attention over bulk-copied K/V rows, bf16 models.
 bool attn_mma_supported(int H, int n_heads, int hd);
+int attn_mma_make_map(TensorMap128 *out, const void *base, uint64_t rows, uint64_t width, int n_heads, int hd);
 cudaError_t launch_attn_mma(const AttnArgs &a, int grid, unsigned long long limit_ns, int *status, cudaStream_t st);
 
 // Launchers (plain-ALU kernels).  bf16 != 0 selects bf16 activations/weights/planes.

@@ -43,6 +43,7 @@ struct Slot {
     void *xg = nullptr, *qkv = nullptr, *att = nullptr, *qc = nullptr, *u = nullptr;
     EnvMeta *meta_d = nullptr, *meta_h = nullptr;
     TensorMap128 t_xg, t_att, t_u;                    // TMA descriptors of the A operands
+    TensorMap128 *maps_d = nullptr, *maps_h = nullptr; // attention descriptors: [0] = QKV buffer, [1 + j] = env j's planes
     cudaEvent_t done = nullptr;
     bool busy = false;
     std::vector<int64_t> ids;
@@ -315,6 +316,7 @@ cudaError_t enqueue_batch(ebrl_actgen *h, Slot &s, int S, const int32_t *n_activ
                     a.k_self = (const char *)s.qkv + (size_t)d * h->esz;
                     a.v_self = (const char *)s.qkv + (size_t)2 * d * h->esz;
                     a.kv_stride = 3 * d;
+                    a.self_map = s.maps_d; a.kv_maps = s.maps_d + 1;
                     ln.run(EBRL_KC_SELF_ATTN, 4.0 * M * H * d, 4.0 * M * d * esz, [&] { return launch_attn(h, a, grid, st); });
                 }
                 gemm(s.att, s.t_att, w.w_o, w.t_o, d, d, EPI_RESID, nullptr, w.g2);
@@ -325,6 +327,7 @@ cudaError_t enqueue_batch(ebrl_actgen *h, Slot &s, int S, const int32_t *n_activ
                     a.q = s.qc; a.q_stride = d; a.out = s.att; a.o_stride = d;
                     a.H = H; a.n_heads = c.n_heads; a.hd = h->hd; a.n_envs = ne; a.d = d;
                     a.meta = s.meta_d; a.kv_plane = (c.kv_layers == 1) ? 0 : l; a.self = 0;
+                    a.self_map = s.maps_d; a.kv_maps = s.maps_d + 1;
                     ln.run(EBRL_KC_CROSS_ATTN, 4.0 * H * sum_P_active[step] * d,
                            2.0 * sum_P_active[step] * d * esz + 2.0 * M * d * esz, [&] { return launch_attn(h, a, grid, st); });
                 }
@@ -364,6 +367,13 @@ ebrl_status_t flush_slot(ebrl_actgen *h, Slot &s)
     }
     s.pending.clear();
     CK(cudaMemcpyAsync(s.meta_d, s.meta_h, sizeof(EnvMeta) * (size_t)n, cudaMemcpyHostToDevice, cs));
+    if (h->use_attn_mma && !(c.flags & EBRL_FLAG_TEST_PULL)) {
+        // one TMA descriptor per environment: its planes as a [kv_layers * 2 * P][d] matrix
+        for (int j = 0; j < n; ++j)
+            if (attn_mma_make_map(&s.maps_h[j], s.meta_h[j].kv, (uint64_t)c.kv_layers * 2 * s.meta_h[j].P, c.d, c.n_heads, h->hd))
+                return fail(h, EBRL_ERR_CUDA, "cuTensorMapEncodeTiled failed for the prefix planes of a batch entry");
+        CK(cudaMemcpyAsync(s.maps_d + 1, s.maps_h, sizeof(TensorMap128) * (size_t)n, cudaMemcpyHostToDevice, cs));
+    }
     cudaError_t e = enqueue_batch(h, s, S, n_active.data(), sum_P.data(), s.grid, cs);
     if (e != cudaSuccess) {
         h->sticky = EBRL_ERR_CUDA;
@@ -492,6 +502,7 @@ void free_all(ebrl_actgen *h)
     for (Slot &s : h->slots) {
         if (s.done) cudaEventDestroy(s.done);
         if (s.meta_h) cudaFreeHost(s.meta_h);
+        if (s.maps_h) cudaFreeHost(s.maps_h);
         if (s.kv_stage) cudaFree(s.kv_stage);
         for (TimedLaunch &t : s.timed) { if (t.t0) cudaEventDestroy(t.t0); if (t.t1) cudaEventDestroy(t.t1); }
     }
@@ -649,6 +660,29 @@ ebrl_status_t ebrl_actgen_create(const ebrl_actgen_cfg_t *cfg, const ebrl_actgen
             cudaGetLastError();
             fail(h, EBRL_ERR_NOMEM, "pinned staging allocation failed");
             return bail(EBRL_ERR_NOMEM);
+        }
+        // stale workspace rows are read (never stored) as padding of tiles and boxes: keep them finite
+        if (cudaMemset(s.x, 0, rows * d * 4) != cudaSuccess || cudaMemset(s.xg, 0, rows * d * esz) != cudaSuccess ||
+            cudaMemset(s.qkv, 0, rows * 3 * d * esz) != cudaSuccess || cudaMemset(s.att, 0, rows * d * esz) != cudaSuccess ||
+            cudaMemset(s.qc, 0, rows * d * esz) != cudaSuccess || cudaMemset(s.u, 0, rows * md * esz) != cudaSuccess ||
+            cudaMemset(s.ssq, 0, rows * (d / SSQ_W) * 4) != cudaSuccess) {
+            fail(h, EBRL_ERR_CUDA, "cudaMemset of the workspace failed");
+            return bail(EBRL_ERR_CUDA);
+        }
+        if (h->use_attn_mma) {
+            if ((st = dev_alloc(h, &p, sizeof(TensorMap128) * (batch_envs + 1))) != EBRL_OK) return bail(st);
+            s.maps_d = (TensorMap128 *)p;
+            if (cudaMallocHost((void **)&s.maps_h, sizeof(TensorMap128) * batch_envs) != cudaSuccess) {
+                cudaGetLastError();
+                fail(h, EBRL_ERR_NOMEM, "pinned staging allocation failed");
+                return bail(EBRL_ERR_NOMEM);
+            }
+            TensorMap128 self_map;
+            if (attn_mma_make_map(&self_map, s.qkv, rows, 3 * (uint64_t)d, cfg->n_heads, h->hd) ||
+                cudaMemcpy(s.maps_d, &self_map, sizeof self_map, cudaMemcpyHostToDevice) != cudaSuccess) {
+                fail(h, EBRL_ERR_CUDA, "building the TMA descriptor of the QKV buffer failed");
+                return bail(EBRL_ERR_CUDA);
+            }
         }
         if (h->use_tc) {
             // the row extent is the workspace capacity: rows past a group's M hold stale data

@@ -1,17 +1,21 @@
 // Softmax attention for the bf16 models: the H (<= 16) query tokens of one environment against
 // its keys/values -- the cached prefix planes (cross-attention) or its own H rows of the QKV
 // buffer (self-attention).  The kernel is bandwidth-shaped: every K/V element is used by only H
-// queries, so the planes are streamed once through shared memory by 1-D bulk copies (one per
-// key row, so that rows can be padded against bank conflicts) into a 3-stage ring, and the
+// queries, so the planes are streamed once through shared memory.  Each environment's planes
+// are described by a 3-D TMA descriptor (64-column group, row, group index) whose box covers a
+// whole slab of heads for a block of keys, so one copy instruction moves 32 KB and lands it as
+// [group][key][128 B] tiles with the 128-byte swizzle: ldmatrix reads them conflict-free.  The
 // small contractions run on mma.sync (m16n8k16, bf16 in, fp32 accumulate) with the softmax
 // statistics kept per row by quad shuffles.
 //
 // Work item = (environment, slab of up to 8 heads); one warp per head; a ninth warp issues the
-// copies.  Keys are visited in blocks of 16 in index order with a running maximum and sum, so
-// an environment's result does not depend on the grid size or on what else is in the batch.
-// Every wait is bounded (status word, as in the GEMM).
+// copies into a 3-stage ring.  Keys are visited in blocks of 16 in index order with a running
+// maximum and sum, so an environment's result does not depend on the grid size or on what else
+// is in the batch.  Every wait is bounded (status word, as in the GEMM).
 #include "actgen_internal.h"
 #include "ptx_helpers.cuh"
+
+#include <cuda.h>
 
 namespace ebrl {
 namespace am {
@@ -39,6 +43,12 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], 
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+__device__ __forceinline__ float ex2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 __device__ __forceinline__ uint32_t pack2(float lo, float hi)
 {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -48,15 +58,21 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi)
 // Keys per stage for a slab of W columns: a whole number of 16-key blocks within the stage budget.
 __host__ __device__ inline int stage_keys(int W) { int k = STAGE_ROWS_BYTES / (W * 2); k &= ~15; return k < 16 ? 16 : (k > 64 ? 64 : k); }
 
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const void *tmap, uint32_t bar, int c0, int c1, int c2)
+{
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+
 template <int HD>
 __global__ void __launch_bounds__(THREADS, 1) attn_mma_kernel(AttnArgs a, int hpc, unsigned long long limit_ns, int *status)
 {
     extern __shared__ uint8_t smem_raw[];
-    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~(uintptr_t)127);
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int W = hpc * HD;                       // slab width in columns
-    const int pitch = W * 2 + 16;                 // bytes per staged key row (padded: conflict-free ldmatrix)
-    const int KB = stage_keys(W);
-    const int stage_bytes = KB * pitch;
+    const int G = W / 64;                         // 64-column groups per slab
+    const int KB = stage_keys(W);                 // keys per stage (a multiple of 16)
+    const int stage_bytes = G * KB * 128;         // one box: [G][KB][128 B]
     const uint32_t sK = smem_u32(smem), sV = sK + NSTAGE * stage_bytes;
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + 2 * NSTAGE * stage_bytes);
     const uint32_t bar0 = smem_u32(bars);
@@ -67,46 +83,42 @@ __global__ void __launch_bounds__(THREADS, 1) attn_mma_kernel(AttnArgs a, int hp
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int H = a.H, nslab = a.n_heads / hpc, items = a.n_envs * nslab;
 
-    // zero the ring once: rows past a prefix's end are never copied, and 0 * stale bits must be 0
-    for (int i = threadIdx.x; i < 2 * NSTAGE * stage_bytes / 16; i += blockDim.x)
-        reinterpret_cast<uint4 *>(smem)[i] = make_uint4(0, 0, 0, 0);
     if (threadIdx.x == 0) {
         for (int s = 0; s < NSTAGE; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), hpc); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    fence_proxy_async();
     __syncthreads();
 
     bool ok = true;
-    int stage = 0;
-    uint32_t phase = 0;
 
     if (warp == MAXW) {
-        // ---- producer: one bulk copy per key row of K and of V
+        // ---- producer: per key block one box of K and one of V (rows past the planes' end are
+        // zero-filled by the copy; rows of the V plane read through the K box are masked later)
+        int stage = 0;
+        uint32_t phase = 0;
         for (int item = blockIdx.x; item < items && ok; item += gridDim.x) {
             const int env = item / nslab, slab = item - env * nslab;
-            const __nv_bfloat16 *kbase, *vbase;
-            int P, stride;
+            const void *tm;
+            int P, krow, vrow, kgrp, vgrp;
             if (a.self) {
-                kbase = (const __nv_bfloat16 *)a.k_self + (size_t)env * H * a.kv_stride + slab * W;
-                vbase = (const __nv_bfloat16 *)a.v_self + (size_t)env * H * a.kv_stride + slab * W;
-                P = H; stride = a.kv_stride;
+                tm = a.self_map; P = H;
+                krow = vrow = env * H;
+                kgrp = (a.d + slab * W) / 64; vgrp = (2 * a.d + slab * W) / 64;
             } else {
-                const EnvMeta m = a.meta[env];
-                P = m.P; stride = a.d;
-                kbase = (const __nv_bfloat16 *)m.kv + (size_t)a.kv_plane * 2 * P * a.d + slab * W;
-                vbase = kbase + (size_t)P * a.d;
+                tm = a.kv_maps + env; P = a.meta[env].P;
+                krow = a.kv_plane * 2 * P; vrow = krow + P;
+                kgrp = vgrp = slab * G;
+                // descriptors are rewritten by the host between batches: drop any stale cached copy
+                if (lane == 0) asm volatile("fence.proxy.tensormap::generic.acquire.gpu [%0], 128;" ::"l"(reinterpret_cast<uint64_t>(tm)) : "memory");
+                __syncwarp();
             }
             for (int j0 = 0; j0 < P; j0 += KB) {
-                const int nrows = min(KB, P - j0);
                 if (!__all_sync(0xffffffffu, mbar_wait(empty(stage), phase ^ 1u, limit_ns, abort_flag))) { ok = false; break; }
-                if (lane == 0) mbar_expect_tx(full(stage), (uint32_t)(2 * nrows * W * 2));
-                __syncwarp();
-                for (int r = lane; r < 2 * nrows; r += 32) {
-                    const int isv = r >= nrows, j = isv ? r - nrows : r;
-                    const __nv_bfloat16 *src = (isv ? vbase : kbase) + (size_t)(j0 + j) * stride;
-                    bulk_load((isv ? sV : sK) + stage * stage_bytes + j * pitch, src, (uint32_t)(W * 2), full(stage));
+                if (lane == 0) {
+                    mbar_expect_tx(full(stage), (uint32_t)(2 * stage_bytes));
+                    tma_load_3d(sK + stage * stage_bytes, tm, full(stage), 0, krow + j0, kgrp);
+                    tma_load_3d(sV + stage * stage_bytes, tm, full(stage), 0, vrow + j0, vgrp);
                 }
                 __syncwarp();
                 if (++stage == NSTAGE) { stage = 0; phase ^= 1u; }
@@ -116,6 +128,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_mma_kernel(AttnArgs a, int hp
         // ---- consumers: warp = head within the slab
         const int g = lane >> 2, t = lane & 3;
         const float sc = 1.4426950408889634f / sqrtf((float)HD);   // log2(e) / sqrt(hd): scores in base-2 units
+        int qbase = 0;                                              // stages consumed by earlier items
         for (int item = blockIdx.x; item < items && ok; item += gridDim.x) {
             const int env = item / nslab, slab = item - env * nslab;
             const int P = a.self ? H : a.meta[env].P;
@@ -137,63 +150,95 @@ __global__ void __launch_bounds__(THREADS, 1) attn_mma_kernel(AttnArgs a, int hp
 #pragma unroll
             for (int n = 0; n < HD / 8; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
             float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;   // rows g and g + 8
-            const uint32_t kcol = (uint32_t)(warp * HD * 2);
-            for (int j0 = 0; j0 < P; j0 += KB) {
-                if (!__all_sync(0xffffffffu, mbar_wait(full(stage), phase, limit_ns, abort_flag))) { ok = false; break; }
-                const int nrows = min(KB, P - j0);
-                const uint32_t kst = sK + stage * stage_bytes + kcol, vst = sV + stage * stage_bytes + kcol;
-                for (int jb = 0; jb < nrows; jb += 16) {
-                    // S = Q K^T for 16 keys: two n-tiles of 8 keys
-                    float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
-                    {
-                        const uint32_t addr = kst + (uint32_t)((jb + (lane >> 4) * 8 + (lane & 7)) * pitch + ((lane >> 3) & 1) * 16);
+            const int g0 = warp * (HD / 64);   // first 64-column group of this warp's head
+            const int BPS = KB / 16, nblk = (P + 15) / 16;               // 16-key blocks per stage / in this item
+            // stage of block b: ring slot (qbase + b / BPS) % NSTAGE, parity ((qbase + b / BPS) / NSTAGE) & 1
+            auto qk = [&](int b, float (&s0)[4], float (&s1)[4]) {
+                const int qs = qbase + b / BPS;
+                const uint32_t kst = sK + (uint32_t)(qs % NSTAGE) * stage_bytes;
+                const int r = (b % BPS) * 16 + (lane >> 4) * 8 + (lane & 7);   // key row within the stage; r & 7 == lane & 7
+                const int ch = (lane >> 3) & 1;                                  // 16-byte chunk within the k-step
+                auto kaddr = [&](int ks) {   // tile [group][KB rows][128 B], chunk index XOR (row & 7)
+                    return kst + (uint32_t)(((g0 + (ks >> 2)) * KB + r) * 128 + (((((ks & 3) << 1) | ch) ^ (lane & 7)) << 4));
+                };
+                // two accumulation chains per n-tile (even / odd k-steps), added at the end
+                float e0[4] = {0.f, 0.f, 0.f, 0.f}, e1[4] = {0.f, 0.f, 0.f, 0.f}, d0[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                        for (int ks = 0; ks < HD / 16; ++ks) {
-                            uint32_t b0, b1, b2, b3;
-                            ldsm_x4(addr + ks * 32, b0, b1, b2, b3);
-                            mma_bf16(s0, qf[ks], b0, b1);
-                            mma_bf16(s1, qf[ks], b2, b3);
-                        }
-                    }
-                    // mask keys past the prefix, running max / sum per row
-                    const int kleft = nrows - jb;   // valid keys in this block (may exceed 16)
-                    const int c0 = 2 * t, c1 = 2 * t + 1;
-                    float v[8] = {s0[0], s0[1], s0[2], s0[3], s1[0], s1[1], s1[2], s1[3]};
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        const int key = (e >> 2) * 8 + ((e & 1) ? c1 : c0);
-                        v[e] = key < kleft ? v[e] * sc : -INFINITY;
-                    }
-                    float mx0 = fmaxf(fmaxf(v[0], v[1]), fmaxf(v[4], v[5]));
-                    float mx1 = fmaxf(fmaxf(v[2], v[3]), fmaxf(v[6], v[7]));
-                    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1)); mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
-                    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1)); mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-                    const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
-                    const float al0 = exp2f(m0 - mn0), al1 = exp2f(m1 - mn1);
-                    m0 = mn0; m1 = mn1;
-                    float p[8];
-                    p[0] = exp2f(v[0] - mn0); p[1] = exp2f(v[1] - mn0); p[4] = exp2f(v[4] - mn0); p[5] = exp2f(v[5] - mn0);
-                    p[2] = exp2f(v[2] - mn1); p[3] = exp2f(v[3] - mn1); p[6] = exp2f(v[6] - mn1); p[7] = exp2f(v[7] - mn1);
-                    l0 = l0 * al0 + ((p[0] + p[1]) + (p[4] + p[5]));
-                    l1 = l1 * al1 + ((p[2] + p[3]) + (p[6] + p[7]));
-                    uint32_t pf[4];
-                    pf[0] = pack2(p[0], p[1]); pf[1] = pack2(p[2], p[3]); pf[2] = pack2(p[4], p[5]); pf[3] = pack2(p[6], p[7]);
-                    // O = O * alpha + P V
-                    const uint32_t vaddr = vst + (uint32_t)((jb + ((lane >> 3) & 1) * 8 + (lane & 7)) * pitch + (lane >> 4) * 16);
-#pragma unroll
-                    for (int n = 0; n < HD / 8; n += 2) {
-                        uint32_t b0, b1, b2, b3;
-                        ldsm_x4_t(vaddr + n * 16, b0, b1, b2, b3);
-                        o[n][0] *= al0; o[n][1] *= al0; o[n][2] *= al1; o[n][3] *= al1;
-                        o[n + 1][0] *= al0; o[n + 1][1] *= al0; o[n + 1][2] *= al1; o[n + 1][3] *= al1;
-                        mma_bf16(o[n], pf, b0, b1);
-                        mma_bf16(o[n + 1], pf, b2, b3);
-                    }
+                for (int ks = 0; ks < HD / 16; ks += 2) {
+                    uint32_t b0, b1, b2, b3, c0, c1, c2, c3;
+                    ldsm_x4(kaddr(ks), b0, b1, b2, b3);
+                    ldsm_x4(kaddr(ks + 1), c0, c1, c2, c3);
+                    mma_bf16(e0, qf[ks], b0, b1);
+                    mma_bf16(e1, qf[ks], b2, b3);
+                    mma_bf16(d0, qf[ks + 1], c0, c1);
+                    mma_bf16(d1, qf[ks + 1], c2, c3);
                 }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(empty(stage));
-                if (++stage == NSTAGE) { stage = 0; phase ^= 1u; }
+#pragma unroll
+                for (int i = 0; i < 4; ++i) { s0[i] = e0[i] + d0[i]; s1[i] = e1[i] + d1[i]; }
+            };
+            auto wait_block = [&](int b) -> bool {   // first block of a stage: wait until the copies have landed
+                if (b % BPS) return true;
+                const int qs = qbase + b / BPS;
+                return __all_sync(0xffffffffu, mbar_wait(full(qs % NSTAGE), (uint32_t)(qs / NSTAGE) & 1u, limit_ns, abort_flag));
+            };
+            float s0[4], s1[4];
+            if (!wait_block(0)) { ok = false; break; }
+            qk(0, s0, s1);
+            for (int b = 0; b < nblk; ++b) {
+                // issue the next block's Q K^T before this block's softmax, so that the tensor pipe
+                // works while the softmax chain of this block resolves
+                float n0[4] = {0.f, 0.f, 0.f, 0.f}, n1[4] = {0.f, 0.f, 0.f, 0.f};
+                if (b + 1 < nblk) {
+                    if (!wait_block(b + 1)) { ok = false; break; }
+                    qk(b + 1, n0, n1);
+                }
+                // mask keys past the prefix, running max / sum per row
+                const int kleft = P - b * 16;
+                float v[8] = {s0[0], s0[1], s0[2], s0[3], s1[0], s1[1], s1[2], s1[3]};
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const int key = (e >> 2) * 8 + 2 * t + (e & 1);
+                    v[e] = key < kleft ? v[e] * sc : -INFINITY;
+                }
+                float mx0 = fmaxf(fmaxf(v[0], v[1]), fmaxf(v[4], v[5]));
+                float mx1 = fmaxf(fmaxf(v[2], v[3]), fmaxf(v[6], v[7]));
+                mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1)); mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1)); mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+                const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
+                const float al0 = ex2(m0 - mn0), al1 = ex2(m1 - mn1);
+                const bool rescale = __any_sync(0xffffffffu, (mn0 != m0) || (mn1 != m1));   // warp-uniform
+                m0 = mn0; m1 = mn1;
+                float p[8];
+                p[0] = ex2(v[0] - mn0); p[1] = ex2(v[1] - mn0); p[4] = ex2(v[4] - mn0); p[5] = ex2(v[5] - mn0);
+                p[2] = ex2(v[2] - mn1); p[3] = ex2(v[3] - mn1); p[6] = ex2(v[6] - mn1); p[7] = ex2(v[7] - mn1);
+                l0 = l0 * al0 + ((p[0] + p[1]) + (p[4] + p[5]));
+                l1 = l1 * al1 + ((p[2] + p[3]) + (p[6] + p[7]));
+                uint32_t pf[4];
+                pf[0] = pack2(p[0], p[1]); pf[1] = pack2(p[2], p[3]); pf[2] = pack2(p[4], p[5]); pf[3] = pack2(p[6], p[7]);
+                // O = O * alpha + P V   (alpha is exactly 1 in every lane when no row maximum moved)
+                const int qs = qbase + b / BPS;
+                const uint32_t vst = sV + (uint32_t)(qs % NSTAGE) * stage_bytes;
+                const int vr = (b % BPS) * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
+                if (rescale) {
+#pragma unroll
+                    for (int n = 0; n < HD / 8; ++n) { o[n][0] *= al0; o[n][1] *= al0; o[n][2] *= al1; o[n][3] *= al1; }
+                }
+#pragma unroll
+                for (int n = 0; n < HD / 8; n += 2) {
+                    uint32_t b0, b1, b2, b3;
+                    const int col0 = n * 8 + (lane >> 4) * 8;   // first column of this lane's 8x8 matrix within the head
+                    ldsm_x4_t(vst + (uint32_t)(((g0 + (col0 >> 6)) * KB + vr) * 128 + ((((col0 & 63) >> 3) ^ (lane & 7)) << 4)), b0, b1, b2, b3);
+                    mma_bf16(o[n], pf, b0, b1);
+                    mma_bf16(o[n + 1], pf, b2, b3);
+                }
+                if ((b % BPS) == BPS - 1 || b == nblk - 1) {   // last block of its stage: hand the stage back
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(empty(qs % NSTAGE));
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i) { s0[i] = n0[i]; s1[i] = n1[i]; }
             }
+            qbase += (P + KB - 1) / KB;
             if (!ok) break;
             // row sums across the quad, normalise, store
             l0 += __shfl_xor_sync(0xffffffffu, l0, 1); l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
@@ -230,6 +275,33 @@ bool attn_mma_supported(int H, int n_heads, int hd)
     return n_heads % hpc == 0;
 }
 
+typedef CUresult (*EncodeTiledFn3)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                   const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// 3-D descriptor of a row-major bf16 matrix [rows][width] seen as (64-column group, row, group
+// index): box = one slab of heads x one stage of keys, 128-byte swizzle, zero fill out of range.
+int attn_mma_make_map(TensorMap128 *out, const void *base, uint64_t rows, uint64_t width, int n_heads, int hd)
+{
+    static EncodeTiledFn3 fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess) return 1;
+        fn = reinterpret_cast<EncodeTiledFn3>(p);
+    }
+    const int hpc = n_heads < am::MAXW ? n_heads : am::MAXW;
+    const int W = hpc * hd;
+    const cuuint64_t dims[3] = {64, rows, width / 64};
+    const cuuint64_t strides[2] = {width * 2, 128};
+    const cuuint32_t box[3] = {64, (cuuint32_t)am::stage_keys(W), (cuuint32_t)(W / 64)};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(reinterpret_cast<CUtensorMap *>(out), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box,
+                    estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? 0 : 2;
+}
+
 cudaError_t launch_attn_mma(const AttnArgs &a, int grid, unsigned long long limit_ns, int *status, cudaStream_t st)
 {
     const int hpc = a.n_heads < am::MAXW ? a.n_heads : am::MAXW;
@@ -237,7 +309,7 @@ cudaError_t launch_attn_mma(const AttnArgs &a, int grid, unsigned long long limi
     if (items == 0) return cudaSuccess;
     const int g = items < grid ? items : grid;
     const int W = hpc * a.hd;
-    const size_t smem = (size_t)2 * am::NSTAGE * am::stage_keys(W) * (W * 2 + 16) + 64 + 128;
+    const size_t smem = (size_t)2 * am::NSTAGE * am::stage_keys(W) * (W / 64) * 128 + 64 + 1024;
     cudaError_t e;
     if (a.hd == 128) {
         e = cudaFuncSetAttribute(am::attn_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

@@ -67,13 +67,29 @@ __global__ void __launch_bounds__(1024) embed_kernel(EmbedArgs a)
 // ---------------------------------------------------------------------------------------
 // v = W_out RMSNorm(x; g_final) + b_out;  a += v / K.  One warp per row.
 // ---------------------------------------------------------------------------------------
+template <typename T> __device__ __forceinline__ void load8(const T *p, float (&v)[8]);
+template <> __device__ __forceinline__ void load8<float>(const float *p, float (&v)[8])
+{
+    const float4 a = *reinterpret_cast<const float4 *>(p), b = *reinterpret_cast<const float4 *>(p + 4);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
+template <> __device__ __forceinline__ void load8<__nv_bfloat16>(const __nv_bfloat16 *p, float (&v)[8])
+{
+    const uint4 u = *reinterpret_cast<const uint4 *>(p);
+    const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&u);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { v[2 * i] = __bfloat162float(h[i].x); v[2 * i + 1] = __bfloat162float(h[i].y); }
+}
+
+constexpr int HEAD_WARPS = 16;
+
 template <typename T, int AMAX>
-__global__ void __launch_bounds__(256) head_kernel(HeadArgs a)
+__global__ void __launch_bounds__(HEAD_WARPS * 32) head_kernel(HeadArgs a)
 {
     const int rows = a.n_envs * a.H;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const T *w_out = (const T *)a.w_out;
-    for (int row = blockIdx.x * 8 + warp; row < rows; row += gridDim.x * 8) {
+    for (int row = blockIdx.x * HEAD_WARPS + warp; row < rows; row += gridDim.x * HEAD_WARPS) {
         const int env = row / a.H, h = row - env * a.H;
         const EnvMeta m = a.meta[env];
         const float *xr = a.x + (size_t)row * a.d;
@@ -82,13 +98,22 @@ __global__ void __launch_bounds__(256) head_kernel(HeadArgs a)
         for (int j = 0; j < AMAX; ++j) acc[j] = 0.f;
         float ss = 0.f;
         if (!a.pull) {
-            for (int c = lane; c < a.d; c += 32) {
-                const float xv = xr[c];
-                ss = fmaf(xv, xv, ss);
-                const float t = xv * a.gain[c];
+            // each lane takes 8 consecutive columns per pass (d is a multiple of 128)
+            for (int c = lane * 8; c < a.d; c += 256) {
+                float xv[8], gv[8], t[8];
+                load8<float>(xr + c, xv);
+                load8<float>(a.gain + c, gv);
 #pragma unroll
-                for (int j = 0; j < AMAX; ++j)
-                    if (j < a.A) acc[j] = fmaf(t, ldf(w_out + (size_t)j * a.d + c), acc[j]);
+                for (int i = 0; i < 8; ++i) { ss = fmaf(xv[i], xv[i], ss); t[i] = xv[i] * gv[i]; }
+#pragma unroll
+                for (int j = 0; j < AMAX; ++j) {
+                    if (j < a.A) {
+                        float wv[8];
+                        load8<T>(w_out + (size_t)j * a.d + c, wv);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) acc[j] = fmaf(t[i], wv[i], acc[j]);
+                    }
+                }
             }
             ss = warp_sum(ss);
         }
@@ -357,16 +382,16 @@ cudaError_t launch_embed(const EmbedArgs &a, int bf16, int grid, cudaStream_t st
 template <typename T>
 static void head_dispatch(const HeadArgs &a, int g, cudaStream_t st)
 {
-    if (a.A <= 8) head_kernel<T, 8><<<g, 256, 0, st>>>(a);
-    else if (a.A <= 16) head_kernel<T, 16><<<g, 256, 0, st>>>(a);
-    else head_kernel<T, 32><<<g, 256, 0, st>>>(a);
+    if (a.A <= 8) head_kernel<T, 8><<<g, HEAD_WARPS * 32, 0, st>>>(a);
+    else if (a.A <= 16) head_kernel<T, 16><<<g, HEAD_WARPS * 32, 0, st>>>(a);
+    else head_kernel<T, 32><<<g, HEAD_WARPS * 32, 0, st>>>(a);
 }
 
 cudaError_t launch_head(const HeadArgs &a, int bf16, int grid, cudaStream_t st)
 {
     const int rows = a.n_envs * a.H;
     if (rows == 0) return cudaSuccess;
-    const int need = (rows + 7) / 8;
+    const int need = (rows + HEAD_WARPS - 1) / HEAD_WARPS;
     const int g = need < grid ? need : grid;
     if (bf16) head_dispatch<__nv_bfloat16>(a, g, st);
     else head_dispatch<float>(a, g, st);
