@@ -104,6 +104,10 @@ int gemm_tc_box_rows_w();
 cudaError_t launch_gemm_tc(const TensorMap128 &ta, const TensorMap128 &tw, const GemmArgs &a, int grid,
                            unsigned long long limit_ns, int *status, cudaStream_t st);
 
+// The same GEMM on CTA pairs (tcgen05 cta_group::2, 256 x 256 tiles); needs grid >= 2.
+cudaError_t launch_gemm_tc2(const TensorMap128 &ta, const TensorMap128 &tw, const GemmArgs &a, int grid,
+                            unsigned long long limit_ns, int *status, cudaStream_t st);
+
 // Tensor-core (mma.sync) attention over bulk-copied K/V rows, bf16 models.
 bool attn_mma_supported(int H, int n_heads, int hd);
 int attn_mma_make_map(TensorMap128 *out, const void *base, uint64_t rows, uint64_t width, int n_heads, int hd);

@@ -9,6 +9,7 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -69,6 +70,7 @@ struct ebrl_actgen {
     ebrl_actgen_cfg_t cfg;
     int bf16 = 0, n_sms = 0, hd = 0, md = 0;
     bool use_tc = false;          // tensor-core GEMMs (bf16, d a multiple of 256)
+    bool use_pairs = true;        // CTA-pair GEMM (EBRL_GEMM_PAIR=0 selects one CTA per tile)
     bool use_attn_mma = false;    // tensor-core attention (bf16, H <= 16, head_dim 64/128)
     int *status_d = nullptr;      // device status word written by kernels whose waits ran out
     unsigned long long wait_ns = 0;
@@ -301,7 +303,9 @@ cudaError_t enqueue_batch(ebrl_actgen *h, Slot &s, int S, const int32_t *n_activ
                     g.ssq_in = s.ssq; g.n_ssq = nseg; g.inv_d = 1.0f / (float)d; g.eps = c.rms_eps;
                     g.C = C; g.x = s.x; g.gain = gain; g.xg = s.xg; g.ssq_out = s.ssq;
                     const double bytes = ((double)M * K + (double)N * K + (double)M * N) * esz + (epi == EPI_RESID ? 8.0 * M * N : 0.0);
-                    if (h->use_tc)
+                    if (h->use_tc && h->use_pairs && grid >= 2)
+                        ln.run(EBRL_KC_GEMM, 2.0 * M * N * K, bytes, [&] { return launch_gemm_tc2(tA, tW, g, grid, h->wait_ns, h->status_d, st); });
+                    else if (h->use_tc)
                         ln.run(EBRL_KC_GEMM, 2.0 * M * N * K, bytes, [&] { return launch_gemm_tc(tA, tW, g, grid, h->wait_ns, h->status_d, st); });
                     else
                         ln.run(EBRL_KC_GEMM, 2.0 * M * N * K, bytes, [&] { return launch_gemm_simt(g, bf, grid, st); });
@@ -629,6 +633,7 @@ ebrl_status_t ebrl_actgen_create(const ebrl_actgen_cfg_t *cfg, const ebrl_actgen
     }
     h->use_tc = h->bf16 && !(cfg->flags & EBRL_FLAG_FORCE_SIMT) && gemm_tc_supported(d, d) && gemm_tc_supported(md, d) &&
                 gemm_tc_supported(d, md) && gemm_tc_supported(3 * d, d);
+    if (const char *e = getenv("EBRL_GEMM_PAIR")) h->use_pairs = atoi(e) != 0;
     h->use_attn_mma = h->bf16 && !(cfg->flags & EBRL_FLAG_FORCE_SIMT) && attn_mma_supported(cfg->H, cfg->n_heads, h->hd);
     if (h->use_tc) {
         const uint32_t bw = (uint32_t)gemm_tc_box_rows_w();

@@ -12,6 +12,7 @@
 // EBRL_ERR_TIMEOUT in the status word, lets its copies land, frees tensor memory and returns.
 #include "actgen_internal.h"
 #include "ptx_helpers.cuh"
+#include "gemm_epilogue.cuh"
 
 #include <cuda.h>
 
@@ -31,8 +32,6 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tm,
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
                  ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar), "r"(c0), "r"(c1) : "memory");
 }
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -43,19 +42,6 @@ __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t
                  "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
                  ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32])
-{
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-                 "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-                 "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-                 : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
 // Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes (64 bf16) with the
 // 128-byte swizzle TMA wrote: 8-row groups are 1024 bytes apart.
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr)
@@ -71,13 +57,6 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr)
 __host__ __device__ constexpr uint32_t instr_desc(int M, int N)
 {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
-}
-
-__device__ __forceinline__ float gelu_erf(float z) { return 0.5f * z * (1.0f + erff(z * 0.70710678118654752440f)); }
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
-{
-    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<uint32_t *>(&v);
 }
 
 template <int EPI>
@@ -129,7 +108,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 if (lane == 0) {
                     mbar_expect_tx(full(stage), A_BYTES + B_BYTES);
                     tma_load_2d(sA + stage * A_BYTES, &tmA, full(stage), kb * BK, m0);
-                    tma_load_2d(sB + stage * B_BYTES, &tmB, full(stage), kb * BK, n0);
+                    tma_load_2d(sB + stage * B_BYTES, &tmB, full(stage), kb * BK, n0);                      // weight rows n0 .. n0+127
+                    tma_load_2d(sB + stage * B_BYTES + B_BYTES / 2, &tmB, full(stage), kb * BK, n0 + BN / 2);   // and n0+128 .. n0+255
                 }
                 __syncwarp();
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -174,69 +154,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const int m0 = (tile / ntn) * BM, n0 = (tile % ntn) * BN;
             const int row = m0 + q * 32 + lane;
             const bool valid = row < g.M;
-            float rs = 0.f;
-            if (EPI != EPI_RESID && valid) {
-                float s = 0.f;
-                for (int t = 0; t < g.n_ssq; ++t) s += g.ssq_in[(size_t)row * g.n_ssq + t];
-                rs = 1.0f / sqrtf(s * g.inv_d + g.eps);
-            }
             if (!__all_sync(0xffffffffu, mbar_wait(tfull(buf), acc_phase, limit_ns, abort_flag))) { ok = false; break; }
             tc_fence_after();
-            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * BN;
-            float ss = 0.f;
-#pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
-                uint32_t r[32];
-                tc_ld32(taddr + (uint32_t)c * 32, r);
-                const int col = n0 + c * 32;
-                if (EPI == EPI_RESID) {
-                    float4 xo[8];
-                    float *xp = g.x + (size_t)row * g.N + col;
-                    if (valid) {
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) xo[j] = *reinterpret_cast<const float4 *>(xp + 4 * j);
-                    }
-                    tc_wait_ld();
-                    if (valid) {
-                        uint32_t pk[16];
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            const float4 gn = *reinterpret_cast<const float4 *>(g.gain + col + 4 * j);
-                            float4 xn;
-                            xn.x = xo[j].x + __uint_as_float(r[4 * j + 0]);
-                            xn.y = xo[j].y + __uint_as_float(r[4 * j + 1]);
-                            xn.z = xo[j].z + __uint_as_float(r[4 * j + 2]);
-                            xn.w = xo[j].w + __uint_as_float(r[4 * j + 3]);
-                            *reinterpret_cast<float4 *>(xp + 4 * j) = xn;
-                            ss = fmaf(xn.x, xn.x, ss); ss = fmaf(xn.y, xn.y, ss);
-                            ss = fmaf(xn.z, xn.z, ss); ss = fmaf(xn.w, xn.w, ss);
-                            pk[2 * j] = pack_bf16(xn.x * gn.x, xn.y * gn.y);
-                            pk[2 * j + 1] = pack_bf16(xn.z * gn.z, xn.w * gn.w);
-                        }
-                        uint4 *xg = reinterpret_cast<uint4 *>((__nv_bfloat16 *)g.xg + (size_t)row * g.N + col);
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) xg[j] = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
-                        if ((c & 3) == 3) {
-                            g.ssq_out[(size_t)row * (g.N / SSQ_W) + (col + 32 - SSQ_W) / SSQ_W] = ss;
-                            ss = 0.f;
-                        }
-                    }
-                } else {
-                    tc_wait_ld();
-                    if (valid) {
-                        uint32_t pk[16];
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            float a = __uint_as_float(r[2 * j]) * rs, b = __uint_as_float(r[2 * j + 1]) * rs;
-                            if (EPI == EPI_SCALE_GELU) { a = gelu_erf(a); b = gelu_erf(b); }
-                            pk[j] = pack_bf16(a, b);
-                        }
-                        uint4 *cp = reinterpret_cast<uint4 *>((__nv_bfloat16 *)g.C + (size_t)row * g.N + col);
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) cp[j] = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
-                    }
-                }
-            }
+            epilogue_row<EPI, BN>(g, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * BN, row, valid, n0);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty(buf));
@@ -300,7 +220,7 @@ int make_tmap_bf16(TensorMap128 *out, const void *base, uint64_t inner, uint64_t
 
 bool gemm_tc_supported(int N, int K) { return N % tc::BN == 0 && K % tc::BK == 0; }
 int gemm_tc_box_rows_a() { return tc::BM; }
-int gemm_tc_box_rows_w() { return tc::BN; }
+int gemm_tc_box_rows_w() { return tc::BN / 2; }   // weight maps serve both kernels: 128-row boxes
 
 template <int EPI>
 static cudaError_t tc_launch(const TensorMap128 &ta, const TensorMap128 &tw, const GemmArgs &a, int g, unsigned long long limit_ns,

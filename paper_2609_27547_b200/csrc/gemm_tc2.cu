@@ -1,0 +1,258 @@
+// The tensor-core GEMM on CTA pairs: two CTAs of a cluster (two SMs) compute one 256 x 256 tile
+// with tcgen05.mma.cta_group::2.  Each CTA stages its own 128 rows of A and only HALF of the
+// weight tile (128 of its 256 rows) per k-block, so the bytes an SM pulls from L2 per FLOP drop
+// by a third compared with one CTA per 128 x 256 tile -- the single-CTA kernel is bound by that
+// L2 -> SM traffic.  The leader CTA (rank 0 of the pair) issues the MMAs for both; each CTA
+// reads its own 128 accumulator rows from its own tensor memory and runs the same epilogue as
+// the single-CTA kernel.  Same arithmetic per output element, same bounded waits.
+//
+// Barriers: full[s] of the LEADER collects the copy bytes of both CTAs; empty[s] and tfull[b]
+// live in each CTA and are signalled by the leader's tcgen05.commit multicast; tempty[b] of the
+// leader counts the epilogue warps of both CTAs (the peer arrives remotely).
+#include "actgen_internal.h"
+#include "ptx_helpers.cuh"
+#include "gemm_epilogue.cuh"
+
+#include <cuda.h>
+
+namespace ebrl {
+namespace tc2 {
+
+using namespace ptx;
+using namespace tc;
+
+constexpr int BM = 128;          // rows per CTA (256 per pair)
+constexpr int BN = 256;          // columns per pair tile
+constexpr int BNH = 128;         // weight rows staged per CTA
+constexpr int BK = 64, UMMA_K = 16, STAGES = 6;
+constexpr int THREADS = 192;
+constexpr int A_BYTES = BM * BK * 2, B_BYTES = BNH * BK * 2;
+constexpr int SMEM_BYTES = STAGES * (A_BYTES + B_BYTES) + 256 + 1024;
+
+__device__ __forceinline__ uint32_t cluster_rank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t mapa(uint32_t addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA tile load whose completion bytes go to an mbarrier that may live in the pair's other CTA.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *tm, uint32_t bar_cluster, int c0, int c1)
+{
+    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tm)), "r"(bar_cluster), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+__device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr)
+{
+    uint64_t d = (uint64_t)((addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+__host__ __device__ constexpr uint32_t instr_desc_bf16(int M, int N)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+template <int EPI>
+__global__ void __launch_bounds__(THREADS, 1)
+gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmArgs g,
+                unsigned long long limit_ns, int *status)
+{
+    extern __shared__ uint8_t smem_raw[];
+    // the same offset in both CTAs of the pair: the dynamic shared window starts at the same
+    // address in every CTA of a kernel, so rounding up gives matching layouts
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const uint32_t sA = smem_u32(smem), sB = sA + STAGES * A_BYTES;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + STAGES * (A_BYTES + B_BYTES));
+    const uint32_t bar0 = smem_u32(bars);
+    auto full = [&](int s) { return bar0 + 8u * s; };
+    auto empty = [&](int s) { return bar0 + 8u * (STAGES + s); };
+    auto tfull = [&](int b) { return bar0 + 8u * (2 * STAGES + b); };
+    auto tempty = [&](int b) { return bar0 + 8u * (2 * STAGES + 2 + b); };
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(bars + 2 * STAGES + 4);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 2 * STAGES + 5);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_rank();          // 0 = leader
+    const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+    const int ntm = (g.M + 2 * BM - 1) / (2 * BM), ntn = g.N / BN, ntiles = ntm * ntn, nkb = g.K / BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(tfull(b), 1); mbar_init(tempty(b), 8); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmA)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmB)) : "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void *)tmem_slot)), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync();      // barriers of both CTAs initialised, tensor memory of both allocated
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    bool ok = true;
+
+    if (warp == 0) {
+        // ---- TMA producer (both CTAs): own A rows, own half of the weight tile; bytes land on the leader's barrier
+        int stage = 0;
+        uint32_t phase = 0;
+        for (int tile = pair; tile < ntiles && ok; tile += npairs) {
+            const int m0 = (tile / ntn) * (2 * BM) + (int)rank * BM, n0 = (tile % ntn) * BN + (int)rank * BNH;
+            for (int kb = 0; kb < nkb; ++kb) {
+                if (!__all_sync(0xffffffffu, mbar_wait(empty(stage), phase ^ 1u, limit_ns, abort_flag))) { ok = false; break; }
+                if (lane == 0) {
+                    if (rank == 0) mbar_expect_tx(full(stage), 2 * (A_BYTES + B_BYTES));
+                    const uint32_t lead_full = mapa(full(stage), 0);
+                    tma_load_2d_pair(sA + stage * A_BYTES, &tmA, lead_full, kb * BK, m0);
+                    tma_load_2d_pair(sB + stage * B_BYTES, &tmB, lead_full, kb * BK, n0);
+                }
+                __syncwarp();
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
+        }
+    } else if (warp == 1) {
+        // ---- MMA issuer: the leader only, for both CTAs
+        if (rank == 0) {
+            constexpr uint32_t idesc = instr_desc_bf16(2 * BM, BN);
+            int stage = 0, it = 0;
+            uint32_t phase = 0;
+            for (int tile = pair; tile < ntiles && ok; tile += npairs, ++it) {
+                const int buf = it & 1;
+                const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+                if (!__all_sync(0xffffffffu, mbar_wait(tempty(buf), acc_phase ^ 1u, limit_ns, abort_flag))) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)buf * BN;
+                for (int kb = 0; kb < nkb; ++kb) {
+                    if (!__all_sync(0xffffffffu, mbar_wait(full(stage), phase, limit_ns, abort_flag))) { ok = false; break; }
+                    tc_fence_after();
+                    if (lane == 0) {
+                        const uint64_t ad = smem_desc_sw128(sA + stage * A_BYTES), bd = smem_desc_sw128(sB + stage * B_BYTES);
+#pragma unroll
+                        for (int k = 0; k < BK / UMMA_K; ++k)
+                            tc_mma_pair(d_tmem, ad + (uint64_t)(k * UMMA_K * 2 / 16), bd + (uint64_t)(k * UMMA_K * 2 / 16), idesc,
+                                        (kb | k) != 0 ? 1u : 0u);
+                        tc_commit_pair(empty(stage));     // frees the stage in both CTAs
+                    }
+                    __syncwarp();
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                if (lane == 0) tc_commit_pair(tfull(buf));  // accumulators of both CTAs are complete
+                __syncwarp();
+            }
+        }
+    } else {
+        // ---- epilogue (both CTAs): own 128 rows of the pair tile
+        const int q = warp & 3;
+        int it = 0;
+        for (int tile = pair; tile < ntiles && ok; tile += npairs, ++it) {
+            const int buf = it & 1;
+            const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+            const int m0 = (tile / ntn) * (2 * BM) + (int)rank * BM, n0 = (tile % ntn) * BN;
+            const int row = m0 + q * 32 + lane;
+            const bool valid = row < g.M;
+            if (!__all_sync(0xffffffffu, mbar_wait(tfull(buf), acc_phase, limit_ns, abort_flag))) { ok = false; break; }
+            tc_fence_after();
+            epilogue_row<EPI, BN>(g, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * BN, row, valid, n0);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(mapa(tempty(buf), 0));
+        }
+    }
+
+    // ---- teardown: nobody leaves while its partner may still touch its memory
+    if (!ok) {
+        *abort_flag = 1;
+        if (lane == 0) atomicExch(status, 7 /* EBRL_ERR_TIMEOUT */);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag && threadIdx.x == 0) {
+        const unsigned long long t0 = gtimer();   // give copies still in flight time to land
+        while (gtimer() - t0 < 200000ull) { }
+    }
+    __syncthreads();
+    cluster_sync();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    }
+}
+
+}  // namespace tc2
+
+template <int EPI>
+static cudaError_t tc2_launch(const TensorMap128 &ta, const TensorMap128 &tw, const GemmArgs &a, int g, unsigned long long limit_ns,
+                              int *status, cudaStream_t st)
+{
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(tc2::gemm_tc2_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc2::SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)g, 1, 1);
+    cfg.blockDim = dim3(tc2::THREADS, 1, 1);
+    cfg.dynamicSmemBytes = tc2::SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, tc2::gemm_tc2_kernel<EPI>, *reinterpret_cast<const CUtensorMap *>(&ta),
+                              *reinterpret_cast<const CUtensorMap *>(&tw), a, limit_ns, status);
+}
+
+// grid = SM quota; the kernel uses floor(grid / 2) CTA pairs.  Needs grid >= 2.
+cudaError_t launch_gemm_tc2(const TensorMap128 &ta, const TensorMap128 &tw, const GemmArgs &a, int grid, unsigned long long limit_ns,
+                            int *status, cudaStream_t st)
+{
+    if (a.M == 0) return cudaSuccess;
+    const int tiles = ((a.M + 2 * tc2::BM - 1) / (2 * tc2::BM)) * (a.N / tc2::BN);
+    int pairs = grid / 2;
+    if (pairs > tiles) pairs = tiles;
+    const int g = 2 * pairs;
+    switch (a.epi) {
+    case EPI_SCALE_STORE: return tc2_launch<EPI_SCALE_STORE>(ta, tw, a, g, limit_ns, status, st);
+    case EPI_SCALE_GELU: return tc2_launch<EPI_SCALE_GELU>(ta, tw, a, g, limit_ns, status, st);
+    default: return tc2_launch<EPI_RESID>(ta, tw, a, g, limit_ns, status, st);
+    }
+}
+
+}  // namespace ebrl
