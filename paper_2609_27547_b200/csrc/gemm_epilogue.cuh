@@ -29,74 +29,125 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 }
 
 
+constexpr int EPI_STAGE_FLOATS = 32 * 32;   // per-warp transpose buffer: 32 rows x 32 fp32 columns, 16-byte chunks swizzled
+
 // EPI_SCALE_STORE: C = acc * rowscale;  EPI_SCALE_GELU: C = gelu(acc * rowscale);
 // EPI_RESID: x += acc, xg = x * gain, one sum-of-squares partial per 128 columns.
-// `taddr` = tensor-memory address of this warp's lane quarter and of the accumulator's first
-// column; NCOLS columns starting at global column n0.  All 32 lanes must call it (tcgen05.ld is
-// warp-collective); lanes with valid == false load and discard.
-template <int EPI, int NCOLS>
-__device__ __forceinline__ void epilogue_row(const GemmArgs &g, uint32_t taddr, int row, bool valid, int n0)
+//
+// Tensor memory hands each thread one ROW of the accumulator (32 columns at a time).  Global
+// memory wants a warp instruction to touch few rows: the L1 handles one 128-byte line per cycle
+// per instruction, so 32 threads x 16 bytes of 32 different rows cost 32 cycles.  Each 32 x 32
+// chunk is therefore turned through shared memory: thread = row writes its 8 16-byte pieces
+// (piece j of row r at position j ^ (r & 7): conflict-free), then lane l reads piece (l & 7) of
+// rows 4 i + (l >> 3), i = 0..7, so that one instruction covers 4 rows x 128 contiguous bytes.
+//
+// `taddr` = tensor-memory address of this warp's lane quarter and of the first of the NCOLS
+// accumulator columns this warp handles; n0 = their global column; row0 = global row of lane 0.
+// All 32 lanes must call it.  `wait` blocks until the accumulator is complete (false on a
+// time-out); the residual values of the first chunk are requested before it and those of each
+// later chunk one chunk ahead.
+template <int EPI, int NCOLS, typename WaitF>
+__device__ __forceinline__ bool epilogue_rows(const GemmArgs &g, uint32_t taddr, int row0, int n0, float *stg_generic, WaitF wait)
 {
+    constexpr int NC = NCOLS / 32;
+    static_assert(NCOLS == SSQ_W, "one sum-of-squares segment per call");
+    const int lane = threadIdx.x & 31;
+    const uint32_t stg = (uint32_t)__cvta_generic_to_shared(stg_generic);
+    const int nrows = g.M - row0;                   // rows of this warp that exist (may be <= 0 or > 32)
+    const int sub = lane >> 3, piece = lane & 7;    // transposed domain: row 4 i + sub, columns 4 piece .. 4 piece + 3
+    float *__restrict__ xg_x = g.x;
     float rs = 0.f;
-    if (EPI != EPI_RESID && valid) {
+    float4 xv[8];
+    if (EPI == EPI_RESID) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            if (4 * i + sub < nrows) xv[i] = *reinterpret_cast<const float4 *>(xg_x + (size_t)(row0 + 4 * i + sub) * g.N + n0 + 4 * piece);
+    } else if (lane < nrows) {
         float s = 0.f;
+        const int row = row0 + lane;
         for (int t = 0; t < g.n_ssq; ++t) s += g.ssq_in[(size_t)row * g.n_ssq + t];
         rs = 1.0f / sqrtf(s * g.inv_d + g.eps);
     }
-    float ss = 0.f;
+    if (!wait()) return false;
+    tc_fence_after();
+    float ssp[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) ssp[i] = 0.f;
 #pragma unroll 1
-    for (int c = 0; c < NCOLS / 32; ++c) {
+    for (int c = 0; c < NC; ++c) {
         uint32_t r[32];
         tc_ld32(taddr + (uint32_t)c * 32, r);
+        tc_wait_ld();
         const int col = n0 + c * 32;
-        if (EPI == EPI_RESID) {
-            float4 xo[8];
-            float *xp = g.x + (size_t)row * g.N + col;
-            if (valid) {
+        // thread = row: 8 pieces of 16 bytes, swizzled
 #pragma unroll
-                for (int j = 0; j < 8; ++j) xo[j] = *reinterpret_cast<const float4 *>(xp + 4 * j);
+        for (int j = 0; j < 8; ++j) {
+            float v[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                v[e] = __uint_as_float(r[4 * j + e]);
+                if (EPI != EPI_RESID) {
+                    v[e] *= rs;
+                    if (EPI == EPI_SCALE_GELU) v[e] = gelu_erf(v[e]);
+                }
             }
-            tc_wait_ld();
-            if (valid) {
-                uint32_t pk[16];
+            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(stg + (uint32_t)(lane * 128 + ((j ^ (lane & 7)) << 4))),
+                         "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]) : "memory");
+        }
+        __syncwarp();
+        float4 acc[8];
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const float4 gn = *reinterpret_cast<const float4 *>(g.gain + col + 4 * j);
+        for (int i = 0; i < 8; ++i) {
+            const int rr = 4 * i + sub;
+            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(acc[i].x), "=f"(acc[i].y), "=f"(acc[i].z), "=f"(acc[i].w)
+                         : "r"(stg + (uint32_t)(rr * 128 + ((piece ^ (rr & 7)) << 4))) : "memory");
+        }
+        __syncwarp();
+        if (EPI == EPI_RESID) {
+            const float4 gn = *reinterpret_cast<const float4 *>(g.gain + col + 4 * piece);
+            __nv_bfloat16 *__restrict__ xg = (__nv_bfloat16 *)g.xg;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int rr = 4 * i + sub;
+                if (rr < nrows) {
+                    const size_t off = (size_t)(row0 + rr) * g.N + col + 4 * piece;
                     float4 xn;
-                    xn.x = xo[j].x + __uint_as_float(r[4 * j + 0]);
-                    xn.y = xo[j].y + __uint_as_float(r[4 * j + 1]);
-                    xn.z = xo[j].z + __uint_as_float(r[4 * j + 2]);
-                    xn.w = xo[j].w + __uint_as_float(r[4 * j + 3]);
-                    *reinterpret_cast<float4 *>(xp + 4 * j) = xn;
-                    ss = fmaf(xn.x, xn.x, ss); ss = fmaf(xn.y, xn.y, ss);
-                    ss = fmaf(xn.z, xn.z, ss); ss = fmaf(xn.w, xn.w, ss);
-                    pk[2 * j] = pack_bf16(xn.x * gn.x, xn.y * gn.y);
-                    pk[2 * j + 1] = pack_bf16(xn.z * gn.z, xn.w * gn.w);
+                    xn.x = xv[i].x + acc[i].x; xn.y = xv[i].y + acc[i].y; xn.z = xv[i].z + acc[i].z; xn.w = xv[i].w + acc[i].w;
+                    *reinterpret_cast<float4 *>(xg_x + off) = xn;
+                    *reinterpret_cast<uint2 *>(xg + off) = make_uint2(pack_bf16(xn.x * gn.x, xn.y * gn.y), pack_bf16(xn.z * gn.z, xn.w * gn.w));
+                    ssp[i] = fmaf(xn.x, xn.x, ssp[i]); ssp[i] = fmaf(xn.y, xn.y, ssp[i]);
+                    ssp[i] = fmaf(xn.z, xn.z, ssp[i]); ssp[i] = fmaf(xn.w, xn.w, ssp[i]);
                 }
-                uint4 *xg = reinterpret_cast<uint4 *>((__nv_bfloat16 *)g.xg + (size_t)row * g.N + col);
+            }
+            if (c + 1 < NC) {
 #pragma unroll
-                for (int j = 0; j < 4; ++j) xg[j] = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
-                if ((c & 3) == 3) {
-                    g.ssq_out[(size_t)row * (g.N / SSQ_W) + (col + 32 - SSQ_W) / SSQ_W] = ss;
-                    ss = 0.f;
-                }
+                for (int i = 0; i < 8; ++i)
+                    if (4 * i + sub < nrows) xv[i] = *reinterpret_cast<const float4 *>(xg_x + (size_t)(row0 + 4 * i + sub) * g.N + col + 32 + 4 * piece);
             }
         } else {
-            tc_wait_ld();
-            if (valid) {
-                uint32_t pk[16];
+            __nv_bfloat16 *__restrict__ cp = (__nv_bfloat16 *)g.C;
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    float a = __uint_as_float(r[2 * j]) * rs, b = __uint_as_float(r[2 * j + 1]) * rs;
-                    if (EPI == EPI_SCALE_GELU) { a = gelu_erf(a); b = gelu_erf(b); }
-                    pk[j] = pack_bf16(a, b);
-                }
-                uint4 *cp = reinterpret_cast<uint4 *>((__nv_bfloat16 *)g.C + (size_t)row * g.N + col);
-#pragma unroll
-                for (int j = 0; j < 4; ++j) cp[j] = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
+            for (int i = 0; i < 8; ++i) {
+                const int rr = 4 * i + sub;
+                if (rr < nrows)
+                    *reinterpret_cast<uint2 *>(cp + (size_t)(row0 + rr) * g.N + col + 4 * piece) =
+                        make_uint2(pack_bf16(acc[i].x, acc[i].y), pack_bf16(acc[i].z, acc[i].w));
             }
         }
     }
+    if (EPI == EPI_RESID) {
+        // a row's sum of squares over the segment: its 8 lanes' partial sums, added across the lanes
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            float t = ssp[i];
+            t += __shfl_xor_sync(0xffffffffu, t, 1);
+            t += __shfl_xor_sync(0xffffffffu, t, 2);
+            t += __shfl_xor_sync(0xffffffffu, t, 4);
+            const int rr = 4 * i + sub;
+            if (piece == 0 && rr < nrows) g.ssq_out[(size_t)(row0 + rr) * (g.N / SSQ_W) + n0 / SSQ_W] = t;
+        }
+    }
+    return true;
 }
 
 }  // namespace tc

@@ -23,9 +23,10 @@ namespace tc {
 using namespace ptx;
 
 constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4, UMMA_K = 16;
-constexpr int THREADS = 192;
+constexpr int THREADS = 320;          // TMA warp, MMA warp, 8 epilogue warps
+constexpr int EPI_WARPS = 8;
 constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2;
-constexpr int SMEM_BYTES = STAGES * (A_BYTES + B_BYTES) + 256 + 1024;   // + barriers + alignment slack
+constexpr int SMEM_BYTES = STAGES * (A_BYTES + B_BYTES) + 256 + 1024 + EPI_WARPS * EPI_STAGE_FLOATS * 4;   // + barriers + alignment slack
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tm, uint32_t bar, int c0, int c1)
 {
@@ -81,7 +82,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(tfull(b), 1); mbar_init(tempty(b), 4); }
+        for (int b = 0; b < 2; ++b) { mbar_init(tfull(b), 1); mbar_init(tempty(b), EPI_WARPS); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmA)) : "memory");
@@ -145,18 +146,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             __syncwarp();
         }
     } else {
-        // ---- epilogue: warp w reads TMEM lanes 32 (w % 4) .. +31; one thread per output row
-        const int q = warp & 3;
+        // ---- epilogue: warp w reads TMEM lanes 32 (w % 4) .. +31 and half of the tile's columns; one thread per row
+        const int q = warp & 3, half = (warp - 2) >> 2;
+        float *stg = reinterpret_cast<float *>(smem + STAGES * (A_BYTES + B_BYTES) + 256) + (warp - 2) * EPI_STAGE_FLOATS;
         int it = 0;
         for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++it) {
             const int buf = it & 1;
             const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
-            const int m0 = (tile / ntn) * BM, n0 = (tile % ntn) * BN;
-            const int row = m0 + q * 32 + lane;
-            const bool valid = row < g.M;
-            if (!__all_sync(0xffffffffu, mbar_wait(tfull(buf), acc_phase, limit_ns, abort_flag))) { ok = false; break; }
-            tc_fence_after();
-            epilogue_row<EPI, BN>(g, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * BN, row, valid, n0);
+            const int m0 = (tile / ntn) * BM, n0 = (tile % ntn) * BN + half * (BN / 2);
+            if (!epilogue_rows<EPI, BN / 2>(g, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + half * (BN / 2)), m0 + q * 32, n0, stg,
+                                            [&] { return __all_sync(0xffffffffu, mbar_wait(tfull(buf), acc_phase, limit_ns, abort_flag)) != 0; })) {
+                ok = false;
+                break;
+            }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty(buf));

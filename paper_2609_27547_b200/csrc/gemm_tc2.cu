@@ -25,9 +25,10 @@ constexpr int BM = 128;          // rows per CTA (256 per pair)
 constexpr int BN = 256;          // columns per pair tile
 constexpr int BNH = 128;         // weight rows staged per CTA
 constexpr int BK = 64, UMMA_K = 16, STAGES = 6;
-constexpr int THREADS = 192;
+constexpr int THREADS = 320;          // TMA warp, MMA warp, 8 epilogue warps
+constexpr int EPI_WARPS = 8;
 constexpr int A_BYTES = BM * BK * 2, B_BYTES = BNH * BK * 2;
-constexpr int SMEM_BYTES = STAGES * (A_BYTES + B_BYTES) + 256 + 1024;
+constexpr int SMEM_BYTES = STAGES * (A_BYTES + B_BYTES) + 256 + 1024 + EPI_WARPS * EPI_STAGE_FLOATS * 4;
 
 __device__ __forceinline__ uint32_t cluster_rank()
 {
@@ -107,7 +108,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(tfull(b), 1); mbar_init(tempty(b), 8); }
+        for (int b = 0; b < 2; ++b) { mbar_init(tfull(b), 1); mbar_init(tempty(b), 2 * EPI_WARPS); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmA)) : "memory");
@@ -174,18 +175,19 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             }
         }
     } else {
-        // ---- epilogue (both CTAs): own 128 rows of the pair tile
-        const int q = warp & 3;
+        // ---- epilogue (both CTAs): own 128 rows of the pair tile; each warp a lane quarter and half of the columns
+        const int q = warp & 3, half = (warp - 2) >> 2;
+        float *stg = reinterpret_cast<float *>(smem + STAGES * (A_BYTES + B_BYTES) + 256) + (warp - 2) * EPI_STAGE_FLOATS;
         int it = 0;
         for (int tile = pair; tile < ntiles && ok; tile += npairs, ++it) {
             const int buf = it & 1;
             const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
-            const int m0 = (tile / ntn) * (2 * BM) + (int)rank * BM, n0 = (tile % ntn) * BN;
-            const int row = m0 + q * 32 + lane;
-            const bool valid = row < g.M;
-            if (!__all_sync(0xffffffffu, mbar_wait(tfull(buf), acc_phase, limit_ns, abort_flag))) { ok = false; break; }
-            tc_fence_after();
-            epilogue_row<EPI, BN>(g, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * BN, row, valid, n0);
+            const int m0 = (tile / ntn) * (2 * BM) + (int)rank * BM, n0 = (tile % ntn) * BN + half * (BN / 2);
+            if (!epilogue_rows<EPI, BN / 2>(g, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + half * (BN / 2)), m0 + q * 32, n0, stg,
+                                            [&] { return __all_sync(0xffffffffu, mbar_wait(tfull(buf), acc_phase, limit_ns, abort_flag)) != 0; })) {
+                ok = false;
+                break;
+            }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(mapa(tempty(buf), 0));
