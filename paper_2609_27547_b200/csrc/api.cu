@@ -123,6 +123,7 @@ ebrl_status_t check_cfg(const ebrl_actgen_cfg_t *c, std::string *why)
     const int hd = c->d / c->n_heads;
     if (hd != 32 && hd != 64 && hd != 128) return bad(EBRL_ERR_UNSUPPORTED, "head_dim must be 32, 64 or 128");
     if (c->param_dtype != c->kv_dtype) return bad(EBRL_ERR_UNSUPPORTED, "param_dtype and kv_dtype must match");
+    if ((int64_t)c->d * c->A * 4 > 200 * 1024) return bad(EBRL_ERR_UNSUPPORTED, "d * A is limited to 51200 (the input embedding is staged in shared memory)");
     if ((int64_t)c->max_group_envs * c->max_inflight_groups * c->H > (int64_t)1 << 22)
         return bad(EBRL_ERR_UNSUPPORTED, "max_group_envs * max_inflight_groups * H is limited to 4M rows");
     return EBRL_OK;

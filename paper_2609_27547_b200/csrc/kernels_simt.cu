@@ -31,36 +31,60 @@ __device__ __forceinline__ float warp_max(float v)
 __device__ __forceinline__ float gelu_erf(float z) { return 0.5f * z * (1.0f + erff(z * 0.70710678118654752440f)); }
 
 // ---------------------------------------------------------------------------------------
-// x = W_in a + temb(t_k); xg = x * gain; sum-of-squares partials.  One warp per (row, 128-column
-// segment); the row's action vector lives in the lanes and is broadcast by shuffles.
+// x = W_in a + temb(t_k); xg = x * gain; sum-of-squares partials.  W_in is staged once per CTA
+// in shared memory as fp32 [A][d]; one warp per row, each lane four consecutive columns of a
+// 128-column segment at a time; the row's action vector lives in the lanes and is broadcast by
+// shuffles.
 // ---------------------------------------------------------------------------------------
+template <typename T> __device__ __forceinline__ void store4(T *p, float a, float b, float c, float d);
+template <> __device__ __forceinline__ void store4<float>(float *p, float a, float b, float c, float d)
+{
+    *reinterpret_cast<float4 *>(p) = make_float4(a, b, c, d);
+}
+template <> __device__ __forceinline__ void store4<__nv_bfloat16>(__nv_bfloat16 *p, float a, float b, float c, float d)
+{
+    __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+    *reinterpret_cast<uint2 *>(p) = make_uint2(*reinterpret_cast<uint32_t *>(&lo), *reinterpret_cast<uint32_t *>(&hi));
+}
+
 template <typename T>
 __global__ void __launch_bounds__(1024) embed_kernel(EmbedArgs a)
 {
-    const int rows = a.n_envs * a.H, nseg = a.d / SSQ_W, units = rows * nseg;
+    extern __shared__ float wT[];   // [A][d]
+    const int rows = a.n_envs * a.H, nseg = a.d / SSQ_W;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const T *w_in = (const T *)a.w_in;
     T *xg = (T *)a.xg;
-    for (int u = blockIdx.x * 32 + warp; u < units; u += gridDim.x * 32) {
-        const int row = u / nseg, seg = u - row * nseg;
+    for (int e = threadIdx.x; e < a.d * a.A; e += blockDim.x) {
+        const int c = e / a.A, j = e - c * a.A;
+        wT[j * a.d + c] = ldf(w_in + e);
+    }
+    __syncthreads();
+    for (int row = blockIdx.x * 32 + warp; row < rows; row += gridDim.x * 32) {
         const int env = row / a.H, h = row - env * a.H;
         const EnvMeta m = a.meta[env];
         const int k = m.k0 + a.s;
         const float *av = (a.s == 0) ? m.noise + (size_t)h * a.A : a.a_state + (size_t)row * a.A;
         const float mine = lane < a.A ? av[lane] : 0.f;
-        float ss = 0.f;
-#pragma unroll
-        for (int i = 0; i < SSQ_W / 32; ++i) {
-            const int c = seg * SSQ_W + i * 32 + lane;
-            float acc = 0.f;
-            for (int j = 0; j < a.A; ++j) acc = fmaf(ldf(w_in + (size_t)c * a.A + j), __shfl_sync(0xffffffffu, mine, j), acc);
-            acc += a.temb[(size_t)k * a.d + c];
-            a.x[(size_t)row * a.d + c] = acc;
-            stf(xg + (size_t)row * a.d + c, acc * a.gain[c]);
-            ss = fmaf(acc, acc, ss);
+        for (int seg = 0; seg < nseg; ++seg) {
+            const int c = seg * SSQ_W + 4 * lane;
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+            for (int j = 0; j < a.A; ++j) {
+                const float aj = __shfl_sync(0xffffffffu, mine, j);
+                const float4 w = *reinterpret_cast<const float4 *>(wT + j * a.d + c);
+                acc[0] = fmaf(w.x, aj, acc[0]); acc[1] = fmaf(w.y, aj, acc[1]);
+                acc[2] = fmaf(w.z, aj, acc[2]); acc[3] = fmaf(w.w, aj, acc[3]);
+            }
+            const float4 te = *reinterpret_cast<const float4 *>(a.temb + (size_t)k * a.d + c);
+            const float4 gn = *reinterpret_cast<const float4 *>(a.gain + c);
+            acc[0] += te.x; acc[1] += te.y; acc[2] += te.z; acc[3] += te.w;
+            *reinterpret_cast<float4 *>(a.x + (size_t)row * a.d + c) = make_float4(acc[0], acc[1], acc[2], acc[3]);
+            store4<T>(xg + (size_t)row * a.d + c, acc[0] * gn.x, acc[1] * gn.y, acc[2] * gn.z, acc[3] * gn.w);
+            float ss = acc[0] * acc[0];
+            ss = fmaf(acc[1], acc[1], ss); ss = fmaf(acc[2], acc[2], ss); ss = fmaf(acc[3], acc[3], ss);
+            ss = warp_sum(ss);
+            if (lane == 0) a.ssq[(size_t)row * nseg + seg] = ss;
         }
-        ss = warp_sum(ss);
-        if (lane == 0) a.ssq[(size_t)row * nseg + seg] = ss;
     }
 }
 
@@ -370,12 +394,21 @@ __global__ void __launch_bounds__(512) attn_simt_kernel(AttnArgs a)
 // ---------------------------------------------------------------------------------------
 cudaError_t launch_embed(const EmbedArgs &a, int bf16, int grid, cudaStream_t st)
 {
-    const int units = a.n_envs * a.H * (a.d / SSQ_W);
-    if (units == 0) return cudaSuccess;
-    const int need = (units + 31) / 32;
+    const int rows = a.n_envs * a.H;
+    if (rows == 0) return cudaSuccess;
+    const int need = (rows + 31) / 32;
     const int g = need < grid ? need : grid;
-    if (bf16) embed_kernel<__nv_bfloat16><<<g, 1024, 0, st>>>(a);
-    else embed_kernel<float><<<g, 1024, 0, st>>>(a);
+    const size_t smem = (size_t)a.d * a.A * sizeof(float);
+    cudaError_t e;
+    if (bf16) {
+        e = cudaFuncSetAttribute(embed_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        embed_kernel<__nv_bfloat16><<<g, 1024, smem, st>>>(a);
+    } else {
+        e = cudaFuncSetAttribute(embed_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        embed_kernel<float><<<g, 1024, smem, st>>>(a);
+    }
     return cudaGetLastError();
 }
 
