@@ -172,8 +172,10 @@ ebrl_status_t ebrl_actgen_submit(ebrl_actgen_t h, int32_t n_envs, const int64_t 
 
 /* The same with HOST buffers: prefix_kv[i], noise and out point to host memory (pinned memory
  * makes the copies asynchronous).  The planes and the noise are copied to device staging
- * owned by the handle when the call is made, the group runs with its batch, and `out` is
- * copied back after the batch, all on `stream`; `out` is valid after ebrl_actgen_sync.  Needs prefix_len in ext, or every P_e = max_prefix_len. */
+ * owned by the handle when the call is made -- on a copy stream of the handle, so that the
+ * upload of one batch overlaps the kernels of the previous one -- the group runs with its batch
+ * on `stream` once its uploads are done, and `out` is copied back after the batch on `stream`;
+ * `out` is valid after ebrl_actgen_sync.  The host buffers must stay valid until then.  Needs prefix_len in ext, or every P_e = max_prefix_len. */
 ebrl_status_t ebrl_actgen_submit_host(ebrl_actgen_t h, int32_t n_envs, const int64_t *env_ids,
                                       const void *const *prefix_kv_host, const float *noise_host,
                                       float *out_host, int32_t sm_quota, void *stream,

@@ -60,6 +60,8 @@ struct Slot {
     cudaStream_t stream = nullptr;
     int grid = 0, groups_pending = 0;
     size_t stage_used = 0, chunks_used = 0;
+    cudaEvent_t h2d_done = nullptr;
+    bool has_uploads = false;
 };
 
 thread_local std::string g_create_error;
@@ -86,6 +88,7 @@ struct ebrl_actgen {
     ebrl_status_t sticky = EBRL_OK;
     ebrl_actgen_stats_t stats;
     std::vector<void *> owned;   // every device allocation, for destroy
+    cudaStream_t copy_stream = nullptr;   // host-buffer entry point: uploads run here, beside the previous batch's kernels
 };
 
 namespace {
@@ -371,6 +374,11 @@ ebrl_status_t flush_slot(ebrl_actgen *h, Slot &s)
         for (int t = 0; t < m.nsteps; ++t) { n_active[t] += 1; sum_P[t] += m.P; }
     }
     s.pending.clear();
+    if (s.has_uploads) {   // the batch's kernels wait for the uploads issued on the copy stream
+        CK(cudaEventRecord(s.h2d_done, h->copy_stream));
+        CK(cudaStreamWaitEvent(cs, s.h2d_done, 0));
+        s.has_uploads = false;
+    }
     CK(cudaMemcpyAsync(s.meta_d, s.meta_h, sizeof(EnvMeta) * (size_t)n, cudaMemcpyHostToDevice, cs));
     if (h->use_attn_mma && !(c.flags & EBRL_FLAG_TEST_PULL)) {
         // one TMA descriptor per environment: its planes as a [kv_layers * 2 * P][d] matrix
@@ -416,7 +424,7 @@ ebrl_status_t submit_impl(ebrl_actgen *h, int32_t n, const int64_t *env_ids, con
     if (s.pending.empty()) {
         // bounded queue: a slot is reused only after its previous batch has completed
         if ((st = retire(h, s)) != EBRL_OK) return st;
-        s.stream = cs; s.grid = grid; s.groups_pending = 0; s.stage_used = 0; s.chunks_used = 0;
+        s.stream = cs; s.grid = grid; s.groups_pending = 0; s.stage_used = 0; s.chunks_used = 0; s.has_uploads = false;
     }
     const bool pull = (c.flags & EBRL_FLAG_TEST_PULL) != 0;
     const size_t chunk = (size_t)c.H * c.A;
@@ -463,13 +471,14 @@ ebrl_status_t submit_impl(ebrl_actgen *h, int32_t n, const int64_t *env_ids, con
         if (!pull)
             for (int i = 0; i < n; ++i) {
                 const int P = (ext && ext->prefix_len) ? ext->prefix_len[i] : c.max_prefix_len;
-                CK(cudaMemcpyAsync(s.kv_stage + off[i], prefix_kv[i], (size_t)c.kv_layers * 2 * P * c.d * h->esz, cudaMemcpyHostToDevice, cs));
+                CK(cudaMemcpyAsync(s.kv_stage + off[i], prefix_kv[i], (size_t)c.kv_layers * 2 * P * c.d * h->esz, cudaMemcpyHostToDevice, h->copy_stream));
                 kv_dev[i] = s.kv_stage + off[i];
             }
         s.stage_used = need;
         noise_d = s.noise_stage + s.chunks_used * chunk;
         out_d = s.out_stage + s.chunks_used * chunk;
-        CK(cudaMemcpyAsync((void *)noise_d, noise, (size_t)n * chunk * 4, cudaMemcpyHostToDevice, cs));
+        CK(cudaMemcpyAsync((void *)noise_d, noise, (size_t)n * chunk * 4, cudaMemcpyHostToDevice, h->copy_stream));
+        s.has_uploads = true;
         s.copies_out.push_back(HostCopy{out, out_d, (size_t)n * chunk * 4});
         s.chunks_used += (size_t)n;
     } else if (!pull) {
@@ -506,11 +515,14 @@ void free_all(ebrl_actgen *h)
 {
     for (Slot &s : h->slots) {
         if (s.done) cudaEventDestroy(s.done);
+        if (s.h2d_done) cudaEventDestroy(s.h2d_done);
         if (s.meta_h) cudaFreeHost(s.meta_h);
         if (s.maps_h) cudaFreeHost(s.maps_h);
         if (s.kv_stage) cudaFree(s.kv_stage);
         for (TimedLaunch &t : s.timed) { if (t.t0) cudaEventDestroy(t.t0); if (t.t1) cudaEventDestroy(t.t1); }
     }
+    if (h->copy_stream) cudaStreamDestroy(h->copy_stream);
+    h->copy_stream = nullptr;
     for (void *p : h->owned) cudaFree(p);
     h->owned.clear();
 }
@@ -650,6 +662,10 @@ ebrl_status_t ebrl_actgen_create(const ebrl_actgen_cfg_t *cfg, const ebrl_actgen
         }
         if (bad) { fail(h, EBRL_ERR_CUDA, "cuTensorMapEncodeTiled failed for a weight matrix"); return bail(EBRL_ERR_CUDA); }
     }
+    if (cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking) != cudaSuccess) {
+        fail(h, EBRL_ERR_CUDA, "cudaStreamCreate failed");
+        return bail(EBRL_ERR_CUDA);
+    }
     h->slots.resize(2);
     for (Slot &s : h->slots) {
         void *p = nullptr;
@@ -697,6 +713,10 @@ ebrl_status_t ebrl_actgen_create(const ebrl_actgen_cfg_t *cfg, const ebrl_actgen
             int bad = make_tmap_bf16(&s.t_xg, s.xg, d, rows, ba) | make_tmap_bf16(&s.t_att, s.att, d, rows, ba) |
                       make_tmap_bf16(&s.t_u, s.u, md, rows, ba);
             if (bad) { fail(h, EBRL_ERR_CUDA, "cuTensorMapEncodeTiled failed for a workspace"); return bail(EBRL_ERR_CUDA); }
+        }
+        if (cudaEventCreateWithFlags(&s.h2d_done, cudaEventDisableTiming) != cudaSuccess) {
+            fail(h, EBRL_ERR_CUDA, "cudaEventCreate failed");
+            return bail(EBRL_ERR_CUDA);
         }
         if (cudaEventCreateWithFlags(&s.done, cudaEventDisableTiming) != cudaSuccess) {
             fail(h, EBRL_ERR_CUDA, "cudaEventCreate failed");

@@ -16,6 +16,7 @@
 #include "ptx_helpers.cuh"
 
 #include <cuda.h>
+#include <cstdlib>
 
 namespace ebrl {
 namespace am {
@@ -65,7 +66,7 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const void *tmap, uint
 }
 
 template <int HD>
-__global__ void __launch_bounds__(THREADS, 1) attn_mma_kernel(AttnArgs a, int hpc, unsigned long long limit_ns, int *status)
+__global__ void __launch_bounds__(THREADS, 1) attn_mma_kernel(AttnArgs a, int hpc, int la_blocks, unsigned long long limit_ns, int *status)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -94,13 +95,13 @@ __global__ void __launch_bounds__(THREADS, 1) attn_mma_kernel(AttnArgs a, int hp
 
     if (warp == MAXW) {
         // ---- producer: per key block one box of K and one of V (rows past the planes' end are
-        // zero-filled by the copy; rows of the V plane read through the K box are masked later)
+        // zero-filled by the copy; rows of the V plane read through the K box are masked later).
+        // A second cursor runs `la_blocks` key blocks ahead and asks L2 to fetch those boxes, so
+        // that the bytes in flight from HBM are not bounded by the three stages of the ring.
         int stage = 0;
         uint32_t phase = 0;
-        for (int item = blockIdx.x; item < items && ok; item += gridDim.x) {
+        auto locate = [&](int item, const void *&tm, int &P, int &krow, int &vrow, int &kgrp, int &vgrp) {
             const int env = item / nslab, slab = item - env * nslab;
-            const void *tm;
-            int P, krow, vrow, kgrp, vgrp;
             if (a.self) {
                 tm = a.self_map; P = H;
                 krow = vrow = env * H;
@@ -109,11 +110,41 @@ __global__ void __launch_bounds__(THREADS, 1) attn_mma_kernel(AttnArgs a, int hp
                 tm = a.kv_maps + env; P = a.meta[env].P;
                 krow = a.kv_plane * 2 * P; vrow = krow + P;
                 kgrp = vgrp = slab * G;
+            }
+        };
+        // look-ahead cursor
+        int la_item = blockIdx.x, la_j0 = 0, la_P = 0, la_krow = 0, la_vrow = 0, la_kgrp = 0, la_vgrp = 0;
+        const void *la_tm = nullptr;
+        const bool use_la = la_blocks > 0 && !a.self;
+        auto la_step = [&]() {
+            if (la_item >= items) return;
+            if (lane == 0) {
+                asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global [%0, {%1, %2, %3}];"
+                             ::"l"(reinterpret_cast<uint64_t>(la_tm)), "r"(0), "r"(la_krow + la_j0), "r"(la_kgrp) : "memory");
+                asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global [%0, {%1, %2, %3}];"
+                             ::"l"(reinterpret_cast<uint64_t>(la_tm)), "r"(0), "r"(la_vrow + la_j0), "r"(la_vgrp) : "memory");
+            }
+            la_j0 += KB;
+            if (la_j0 >= la_P) {
+                la_item += gridDim.x; la_j0 = 0;
+                if (la_item < items) locate(la_item, la_tm, la_P, la_krow, la_vrow, la_kgrp, la_vgrp);
+            }
+        };
+        if (use_la && la_item < items) {
+            locate(la_item, la_tm, la_P, la_krow, la_vrow, la_kgrp, la_vgrp);
+            for (int i = 0; i < la_blocks; ++i) la_step();
+        }
+        for (int item = blockIdx.x; item < items && ok; item += gridDim.x) {
+            const void *tm;
+            int P, krow, vrow, kgrp, vgrp;
+            locate(item, tm, P, krow, vrow, kgrp, vgrp);
+            if (!a.self) {
                 // descriptors are rewritten by the host between batches: drop any stale cached copy
                 if (lane == 0) asm volatile("fence.proxy.tensormap::generic.acquire.gpu [%0], 128;" ::"l"(reinterpret_cast<uint64_t>(tm)) : "memory");
                 __syncwarp();
             }
             for (int j0 = 0; j0 < P; j0 += KB) {
+                if (use_la) la_step();
                 if (!__all_sync(0xffffffffu, mbar_wait(empty(stage), phase ^ 1u, limit_ns, abort_flag))) { ok = false; break; }
                 if (lane == 0) {
                     mbar_expect_tx(full(stage), (uint32_t)(2 * stage_bytes));
@@ -310,15 +341,23 @@ cudaError_t launch_attn_mma(const AttnArgs &a, int grid, unsigned long long limi
     const int g = items < grid ? items : grid;
     const int W = hpc * a.hd;
     const size_t smem = (size_t)2 * am::NSTAGE * am::stage_keys(W) * (W / 64) * 128 + 64 + 1024;
+    // L2 look-ahead of the producer in key blocks (EBRL_ATTN_LOOKAHEAD overrides; 0 disables)
+    static int la = -1;
+    if (la < 0) {
+        const char *env = getenv("EBRL_ATTN_LOOKAHEAD");
+        la = env ? atoi(env) : 2;
+        if (la < 0) la = 0;
+        if (la > 64) la = 64;
+    }
     cudaError_t e;
     if (a.hd == 128) {
         e = cudaFuncSetAttribute(am::attn_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        am::attn_mma_kernel<128><<<g, am::THREADS, smem, st>>>(a, hpc, limit_ns, status);
+        am::attn_mma_kernel<128><<<g, am::THREADS, smem, st>>>(a, hpc, la, limit_ns, status);
     } else {
         e = cudaFuncSetAttribute(am::attn_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        am::attn_mma_kernel<64><<<g, am::THREADS, smem, st>>>(a, hpc, limit_ns, status);
+        am::attn_mma_kernel<64><<<g, am::THREADS, smem, st>>>(a, hpc, la, limit_ns, status);
     }
     return cudaGetLastError();
 }
