@@ -160,6 +160,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_mma_kernel(AttnArgs a, int hp
         const int g = lane >> 2, t = lane & 3;
         const float sc = 1.4426950408889634f / sqrtf((float)HD);   // log2(e) / sqrt(hd): scores in base-2 units
         int qbase = 0;                                              // stages consumed by earlier items
+        const int bps_sh = KB == 16 ? 0 : (KB == 32 ? 1 : 2), bps_mask = (1 << bps_sh) - 1;   // 16-key blocks per stage: 1, 2 or 4
         for (int item = blockIdx.x; item < items && ok; item += gridDim.x) {
             const int env = item / nslab, slab = item - env * nslab;
             const int P = a.self ? H : a.meta[env].P;
@@ -182,12 +183,12 @@ __global__ void __launch_bounds__(THREADS, 1) attn_mma_kernel(AttnArgs a, int hp
             for (int n = 0; n < HD / 8; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
             float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;   // rows g and g + 8
             const int g0 = warp * (HD / 64);   // first 64-column group of this warp's head
-            const int BPS = KB / 16, nblk = (P + 15) / 16;               // 16-key blocks per stage / in this item
-            // stage of block b: ring slot (qbase + b / BPS) % NSTAGE, parity ((qbase + b / BPS) / NSTAGE) & 1
+            const int nblk = (P + 15) >> 4;                // 16-key blocks in this item; BPS = 1 << bps_sh of them per stage
+            // stage of block b: ring slot (qbase + (b >> bps_sh)) % NSTAGE, parity ((qbase + (b >> bps_sh)) / NSTAGE) & 1
             auto qk = [&](int b, float (&s0)[4], float (&s1)[4]) {
-                const int qs = qbase + b / BPS;
+                const int qs = qbase + (b >> bps_sh);
                 const uint32_t kst = sK + (uint32_t)(qs % NSTAGE) * stage_bytes;
-                const int r = (b % BPS) * 16 + (lane >> 4) * 8 + (lane & 7);   // key row within the stage; r & 7 == lane & 7
+                const int r = (b & bps_mask) * 16 + (lane >> 4) * 8 + (lane & 7);   // key row within the stage; r & 7 == lane & 7
                 const int ch = (lane >> 3) & 1;                                  // 16-byte chunk within the k-step
                 auto kaddr = [&](int ks) {   // tile [group][KB rows][128 B], chunk index XOR (row & 7)
                     return kst + (uint32_t)(((g0 + (ks >> 2)) * KB + r) * 128 + (((((ks & 3) << 1) | ch) ^ (lane & 7)) << 4));
@@ -208,8 +209,8 @@ __global__ void __launch_bounds__(THREADS, 1) attn_mma_kernel(AttnArgs a, int hp
                 for (int i = 0; i < 4; ++i) { s0[i] = e0[i] + d0[i]; s1[i] = e1[i] + d1[i]; }
             };
             auto wait_block = [&](int b) -> bool {   // first block of a stage: wait until the copies have landed
-                if (b % BPS) return true;
-                const int qs = qbase + b / BPS;
+                if (b & bps_mask) return true;
+                const int qs = qbase + (b >> bps_sh);
                 return __all_sync(0xffffffffu, mbar_wait(full(qs % NSTAGE), (uint32_t)(qs / NSTAGE) & 1u, limit_ns, abort_flag));
             };
             float s0[4], s1[4];
@@ -247,9 +248,9 @@ __global__ void __launch_bounds__(THREADS, 1) attn_mma_kernel(AttnArgs a, int hp
                 uint32_t pf[4];
                 pf[0] = pack2(p[0], p[1]); pf[1] = pack2(p[2], p[3]); pf[2] = pack2(p[4], p[5]); pf[3] = pack2(p[6], p[7]);
                 // O = O * alpha + P V   (alpha is exactly 1 in every lane when no row maximum moved)
-                const int qs = qbase + b / BPS;
+                const int qs = qbase + (b >> bps_sh);
                 const uint32_t vst = sV + (uint32_t)(qs % NSTAGE) * stage_bytes;
-                const int vr = (b % BPS) * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
+                const int vr = (b & bps_mask) * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
                 if (rescale) {
 #pragma unroll
                     for (int n = 0; n < HD / 8; ++n) { o[n][0] *= al0; o[n][1] *= al0; o[n][2] *= al1; o[n][3] *= al1; }
@@ -262,14 +263,14 @@ __global__ void __launch_bounds__(THREADS, 1) attn_mma_kernel(AttnArgs a, int hp
                     mma_bf16(o[n], pf, b0, b1);
                     mma_bf16(o[n + 1], pf, b2, b3);
                 }
-                if ((b % BPS) == BPS - 1 || b == nblk - 1) {   // last block of its stage: hand the stage back
+                if ((b & bps_mask) == bps_mask || b == nblk - 1) {   // last block of its stage: hand the stage back
                     __syncwarp();
                     if (lane == 0) mbar_arrive(empty(qs % NSTAGE));
                 }
 #pragma unroll
                 for (int i = 0; i < 4; ++i) { s0[i] = n0[i]; s1[i] = n1[i]; }
             }
-            qbase += (P + KB - 1) / KB;
+            qbase += (nblk + bps_mask) >> bps_sh;
             if (!ok) break;
             // row sums across the quad, normalise, store
             l0 += __shfl_xor_sync(0xffffffffu, l0, 1); l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
