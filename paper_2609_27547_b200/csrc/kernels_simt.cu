@@ -287,7 +287,8 @@ __global__ void __launch_bounds__(512) attn_simt_kernel(AttnArgs a)
     float *p = vb + AKB * hd;
     float *alpha = p + H * AKB;
     float *lsum = alpha + H;
-    const int ncg = 128 / hd, c = t % hd, rg = t / hd;
+    const int hd_sh = hd == 32 ? 5 : (hd == 64 ? 6 : 7);   // head_dim is 32, 64 or 128: shifts, not divisions
+    const int ncg = 128 >> hd_sh, c = t & (hd - 1), rg = t >> hd_sh;
     const float scale = 1.0f / sqrtf((float)hd);
     const int items = a.n_envs * a.n_heads;
     for (int item = blockIdx.x * 4 + grp; item < items; item += gridDim.x * 4) {
@@ -306,7 +307,7 @@ __global__ void __launch_bounds__(512) attn_simt_kernel(AttnArgs a)
         }
         const T *qg = (const T *)a.q + (size_t)env * H * a.q_stride + h * hd;
         for (int e = t; e < H * hd; e += 128) {
-            const int i = e / hd, cc = e - i * hd;
+            const int i = e >> hd_sh, cc = e & (hd - 1);
             q[e] = ldf(qg + (size_t)i * a.q_stride + cc) * scale;
         }
         float acc[RMAX];
@@ -319,7 +320,7 @@ __global__ void __launch_bounds__(512) attn_simt_kernel(AttnArgs a)
             group_sync(grp);   // q ready; previous block's readers done
             const int nkeys = min(AKB, P - j0);
             for (int e = t; e < AKB * hd; e += 128) {
-                const int j = e / hd, cc = e - j * hd;
+                const int j = e >> hd_sh, cc = e & (hd - 1);
                 float kv = 0.f, vv = 0.f;
                 if (j < nkeys) {
                     kv = ldf(kbase + (size_t)(j0 + j) * kvs + cc);
@@ -332,6 +333,7 @@ __global__ void __launch_bounds__(512) attn_simt_kernel(AttnArgs a)
             // scores and running softmax statistics: lane = key, each warp owns rows warp + 4 r
 #pragma unroll
             for (int r0 = 0; r0 < 8; r0 += 4) {
+                if (warp + 4 * r0 >= H) continue;   // no query row in this pass (warp-uniform)
                 float s[4] = {0.f, 0.f, 0.f, 0.f};
                 const float *krow = kb + lane * (hd + 1);
                 for (int cc = 0; cc < hd; ++cc) {
