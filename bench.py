@@ -66,6 +66,7 @@ def parse_args():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--corunner", action="store_true", help="run the streaming co-runner on the other SMs")
     ap.add_argument("--simt", action="store_true", help="force the plain-ALU kernels")
+    ap.add_argument("--green-ctx", action="store_true", help="run inside an SM partition (green context) of the quota")
     ap.add_argument("--min-warmup", type=int, default=3, help="lower bound on warm-up steps (profiling captures use 1)")
     ap.add_argument("--inflight", type=int, default=8, help="groups queued before a batch is launched")
     return ap.parse_args()
@@ -229,7 +230,7 @@ def run_ours(args):
     out = torch.empty_like(noise)
     kv_bytes = sum(envs[e].kv.numel() * envs[e].kv.element_size() for e in ids)
     inflight = args.inflight
-    flags = B.FLAG_FORCE_SIMT if args.simt else 0
+    flags = (B.FLAG_FORCE_SIMT if args.simt else 0) | (B.FLAG_GREEN_CTX if args.green_ctx else 0)
     cfg = B.cfg_for(w, max_group_envs=max(len(g) for g in groups), max_inflight_groups=inflight, flags=flags, device=local)
     gen = B.ActGen(cfg, wt)
     stream = torch.cuda.Stream(dev)
@@ -267,7 +268,8 @@ def run_ours(args):
     barrier()
     clocks = sampler.stop()
     ms = e0.elapsed_time(e1)
-    launches = gen.stats()["kernel_launches"]
+    st0 = gen.stats()
+    launches = st0["kernel_launches"]
     if world > 1:
         t = torch.tensor([ms], device=dev)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -364,6 +366,7 @@ def run_ours(args):
                        "L": w.L, "heads": w.n_heads, "P": list(w.P), "K": w.K, "groups": len(groups),
                        "group_sizes": [min(map(len, groups)), max(map(len, groups))], "sm_quota": q_eff,
                        "inflight_groups": inflight, "corunner": bool(co_stream is not None),
+                       "green_ctx": {"requested": bool(args.green_ctx), "active": bool(st0["green_ctx_active"]), "partition_sms": st0["green_ctx_sms"]},
                        "l2": ("inputs (%.2f GB of prefix planes plus weights) larger than the 126 MB L2" % (kv_bytes / 1e9))
                        if kv_bytes > 126e6 else "inputs fit in L2 and L2 is not flushed: small parity-size case, not a bench line",
                        "seed": seed},

@@ -63,7 +63,9 @@ typedef enum { EBRL_F32 = 0, EBRL_BF16 = 1 } ebrl_dtype_t;
 
 /* cfg.flags */
 #define EBRL_FLAG_TEST_PULL   1u  /* replace the network by v = b_out - a (integrator check)    */
-#define EBRL_FLAG_GREEN_CTX   2u  /* run under a green context of sm_quota SMs when available   */
+#define EBRL_FLAG_GREEN_CTX   2u  /* run each batch inside an SM partition (green context) of at
+                                     least sm_quota SMs when the driver offers one; the grid cap
+                                     of sm_quota CTAs applies either way                         */
 #define EBRL_FLAG_TIMING      4u  /* record per-kernel-class device time (see get_stats)        */
 #define EBRL_FLAG_FORCE_SIMT  8u  /* bf16 models: use the plain-ALU kernels, not tensor cores    */
 
@@ -126,7 +128,10 @@ typedef struct {
     int32_t granted_sms;                  /* SMs of the last submit's quota actually used:
                                              CTAs of the persistent grids, or the green
                                              context's SM count when one is active             */
-    int32_t green_ctx_active;             /* 1 if the last submit ran inside a green context   */
+    int32_t green_ctx_active;             /* 1 if the last batch ran inside a green context    */
+    int32_t green_ctx_sms;                /* SMs in that context's partition (the driver rounds
+                                             the quota up to its granularity), else 0          */
+    int32_t reserved_;
     double class_ms[EBRL_KC_COUNT];       /* device time per kernel class (EBRL_FLAG_TIMING),
                                              accumulated over synced groups                    */
     uint64_t class_launches[EBRL_KC_COUNT];
@@ -245,6 +250,16 @@ ebrl_status_t ebrl_actgen_check_submit(const ebrl_actgen_cfg_t *cfg, int32_t n_s
                                        const ebrl_submit_ext_t *ext);
 int32_t ebrl_actgen_plan_group(const ebrl_actgen_cfg_t *cfg, int32_t n_envs, const ebrl_submit_ext_t *ext,
                                int32_t *order, int32_t *nsteps, int32_t *n_active);
+
+/* ---- failure detection without a fault -------------------------------------------------
+ * Every device-side wait of the library is bounded (cfg.wait_limit_ns): a producer that never
+ * arrives makes the waiting kernel record EBRL_ERR_TIMEOUT and return normally.  This call runs
+ * that wait once on `device` in a one-warp kernel: with signal_it = 0 nothing arrives and
+ * *out_status becomes EBRL_ERR_TIMEOUT after about limit_ns (1 ns .. 2 s); with signal_it = 1
+ * the barrier is signalled and *out_status is EBRL_OK.  *out_waited_ns (may be NULL) is the time
+ * the wait took on the device.  The context stays usable either way. */
+ebrl_status_t ebrl_actgen_wait_probe(int32_t device, uint64_t limit_ns, int32_t signal_it, int32_t *out_status,
+                                     uint64_t *out_waited_ns);
 
 /* ---- bench utility: the synthetic "simulation" co-runner --------------------------------
  * A memory-bound stand-in for a GPU simulator sharing the device with generation (sections

@@ -50,7 +50,8 @@ class SubmitExt(C.Structure):
 class Stats(C.Structure):
     _fields_ = [("groups", C.c_uint64), ("envs", C.c_uint64), ("env_steps", C.c_uint64),
                 ("kernel_launches", C.c_uint64), ("granted_sms", C.c_int32),
-                ("green_ctx_active", C.c_int32), ("class_ms", C.c_double * 5),
+                ("green_ctx_active", C.c_int32), ("green_ctx_sms", C.c_int32), ("reserved_", C.c_int32),
+                ("class_ms", C.c_double * 5),
                 ("class_launches", C.c_uint64 * 5), ("class_flops", C.c_double * 5),
                 ("class_bytes", C.c_double * 5)]
 
@@ -96,6 +97,7 @@ def lib():
                                              C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         L.ebrl_actgen_plan_group.restype = C.c_int32
         L.ebrl_actgen_l0_step_noalloc.argtypes = [C.c_void_p] * 7 + [C.c_int32] * 4 + [C.c_float, C.c_int32, C.c_void_p]
+        L.ebrl_actgen_wait_probe.argtypes = [C.c_int32, C.c_uint64, C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_uint64)]
         L.ebrl_sim_corunner_launch.argtypes = [C.c_void_p, C.c_uint64, C.c_int32, C.c_int32, C.c_void_p]
         _lib = L
     return _lib
@@ -216,7 +218,7 @@ class ActGen:
     def stats(self) -> dict:
         s = Stats()
         self._check(self._L.ebrl_actgen_get_stats(self._h, C.byref(s)))
-        out = {k: getattr(s, k) for k in ("groups", "envs", "env_steps", "kernel_launches", "granted_sms", "green_ctx_active")}
+        out = {k: getattr(s, k) for k in ("groups", "envs", "env_steps", "kernel_launches", "granted_sms", "green_ctx_active", "green_ctx_sms")}
         out["classes"] = {n: {"ms": s.class_ms[i], "launches": s.class_launches[i], "flops": s.class_flops[i],
                               "bytes": s.class_bytes[i]} for i, n in enumerate(KC_NAMES)}
         return out
@@ -257,6 +259,13 @@ def l0_step_noalloc(a_in: torch.Tensor, a_out: torch.Tensor, w_in: torch.Tensor,
     with torch.cuda.device(a_in.device):
         return int(lib().ebrl_actgen_l0_step_noalloc(*[t.data_ptr() for t in ts], n_rows, A, d, K_steps, rms_eps,
                                                      sm_quota, s.cuda_stream))
+
+
+def wait_probe(limit_ns: int, signal_it: bool, device: int = 0):
+    """``ebrl_actgen_wait_probe``: (status of the call, status the kernel recorded, ns waited on the device)."""
+    st, waited = C.c_int32(-1), C.c_uint64(0)
+    rc = lib().ebrl_actgen_wait_probe(device, int(limit_ns), 1 if signal_it else 0, C.byref(st), C.byref(waited))
+    return rc, st.value, waited.value
 
 
 def sim_corunner_launch(buf: torch.Tensor, n_steps: int, n_ctas: int, stream: torch.cuda.Stream):

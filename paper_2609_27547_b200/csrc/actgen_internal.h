@@ -113,6 +113,15 @@ bool attn_mma_supported(int H, int n_heads, int hd);
 int attn_mma_make_map(TensorMap128 *out, const void *base, uint64_t rows, uint64_t width, int n_heads, int hd);
 cudaError_t launch_attn_mma(const AttnArgs &a, int grid, unsigned long long limit_ns, int *status, cudaStream_t st);
 
+// An SM partition (green context) with a stream inside it.
+struct GreenPartition {
+    void *ctx = nullptr;
+    cudaStream_t stream = nullptr;
+    int sm_count = 0;
+};
+int green_partition_create(int device, int sm_quota, GreenPartition *out);
+void green_partition_destroy(GreenPartition *p);
+
 // Launchers (plain-ALU kernels).  bf16 != 0 selects bf16 activations/weights/planes.
 // grid = number of persistent CTAs (the SM quota).
 cudaError_t launch_embed(const EmbedArgs &a, int bf16, int grid, cudaStream_t st);

@@ -11,6 +11,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <map>
 #include <mutex>
 #include <new>
 #include <string>
@@ -60,7 +61,7 @@ struct Slot {
     cudaStream_t stream = nullptr;
     int grid = 0, groups_pending = 0;
     size_t stage_used = 0, chunks_used = 0;
-    cudaEvent_t h2d_done = nullptr;
+    cudaEvent_t h2d_done = nullptr, part_in = nullptr, part_out = nullptr;
     bool has_uploads = false;
 };
 
@@ -88,6 +89,7 @@ struct ebrl_actgen {
     ebrl_status_t sticky = EBRL_OK;
     ebrl_actgen_stats_t stats;
     std::vector<void *> owned;   // every device allocation, for destroy
+    std::map<int, GreenPartition> partitions;   // SM partitions by quota (EBRL_FLAG_GREEN_CTX); ctx == nullptr: creation failed
     cudaStream_t copy_stream = nullptr;   // host-buffer entry point: uploads run here, beside the previous batch's kernels
 };
 
@@ -374,6 +376,25 @@ ebrl_status_t flush_slot(ebrl_actgen *h, Slot &s)
         for (int t = 0; t < m.nsteps; ++t) { n_active[t] += 1; sum_P[t] += m.P; }
     }
     s.pending.clear();
+    // SM partition: the batch runs on the partition's stream, fenced against the caller's stream by events
+    cudaStream_t user = cs;
+    GreenPartition *gp = nullptr;
+    if ((c.flags & EBRL_FLAG_GREEN_CTX) && s.grid < h->n_sms) {
+        auto it = h->partitions.find(s.grid);
+        if (it == h->partitions.end()) {
+            GreenPartition np;
+            if (green_partition_create(c.device, s.grid, &np) != 0) np = GreenPartition();
+            it = h->partitions.emplace(s.grid, np).first;
+        }
+        if (it->second.ctx) gp = &it->second;
+    }
+    if (gp) {
+        CK(cudaEventRecord(s.part_in, user));
+        CK(cudaStreamWaitEvent(gp->stream, s.part_in, 0));
+        cs = gp->stream;
+    }
+    h->stats.green_ctx_active = gp ? 1 : 0;
+    h->stats.green_ctx_sms = gp ? gp->sm_count : 0;
     if (s.has_uploads) {   // the batch's kernels wait for the uploads issued on the copy stream
         CK(cudaEventRecord(s.h2d_done, h->copy_stream));
         CK(cudaStreamWaitEvent(cs, s.h2d_done, 0));
@@ -391,6 +412,11 @@ ebrl_status_t flush_slot(ebrl_actgen *h, Slot &s)
     if (e != cudaSuccess) {
         h->sticky = EBRL_ERR_CUDA;
         return fail(h, EBRL_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
+    }
+    if (gp) {
+        CK(cudaEventRecord(s.part_out, cs));
+        CK(cudaStreamWaitEvent(user, s.part_out, 0));
+        cs = user;
     }
     for (const HostCopy &hc : s.copies_out) CK(cudaMemcpyAsync(hc.dst, hc.src, hc.bytes, cudaMemcpyDeviceToHost, cs));
     s.copies_out.clear();
@@ -506,7 +532,6 @@ ebrl_status_t submit_impl(ebrl_actgen *h, int32_t n, const int64_t *env_ids, con
     h->stats.envs += (uint64_t)n;
     h->stats.env_steps += env_steps;
     h->stats.granted_sms = grid;
-    h->stats.green_ctx_active = 0;
     if (s.groups_pending >= c.max_inflight_groups) return flush_slot(h, s);
     return EBRL_OK;
 }
@@ -516,11 +541,15 @@ void free_all(ebrl_actgen *h)
     for (Slot &s : h->slots) {
         if (s.done) cudaEventDestroy(s.done);
         if (s.h2d_done) cudaEventDestroy(s.h2d_done);
+        if (s.part_in) cudaEventDestroy(s.part_in);
+        if (s.part_out) cudaEventDestroy(s.part_out);
         if (s.meta_h) cudaFreeHost(s.meta_h);
         if (s.maps_h) cudaFreeHost(s.maps_h);
         if (s.kv_stage) cudaFree(s.kv_stage);
         for (TimedLaunch &t : s.timed) { if (t.t0) cudaEventDestroy(t.t0); if (t.t1) cudaEventDestroy(t.t1); }
     }
+    for (auto &kv : h->partitions) green_partition_destroy(&kv.second);
+    h->partitions.clear();
     if (h->copy_stream) cudaStreamDestroy(h->copy_stream);
     h->copy_stream = nullptr;
     for (void *p : h->owned) cudaFree(p);
@@ -714,7 +743,9 @@ ebrl_status_t ebrl_actgen_create(const ebrl_actgen_cfg_t *cfg, const ebrl_actgen
                       make_tmap_bf16(&s.t_u, s.u, md, rows, ba);
             if (bad) { fail(h, EBRL_ERR_CUDA, "cuTensorMapEncodeTiled failed for a workspace"); return bail(EBRL_ERR_CUDA); }
         }
-        if (cudaEventCreateWithFlags(&s.h2d_done, cudaEventDisableTiming) != cudaSuccess) {
+        if (cudaEventCreateWithFlags(&s.part_in, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&s.part_out, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&s.h2d_done, cudaEventDisableTiming) != cudaSuccess) {
             fail(h, EBRL_ERR_CUDA, "cudaEventCreate failed");
             return bail(EBRL_ERR_CUDA);
         }
@@ -803,9 +834,9 @@ ebrl_status_t ebrl_actgen_reset_stats(ebrl_actgen_t h)
 {
     if (!h) return EBRL_ERR_INVALID_ARG;
     std::lock_guard<std::mutex> lk(h->mu);
-    const int32_t g = h->stats.granted_sms, gc = h->stats.green_ctx_active;
+    const int32_t g = h->stats.granted_sms, gc = h->stats.green_ctx_active, gs = h->stats.green_ctx_sms;
     memset(&h->stats, 0, sizeof h->stats);
-    h->stats.granted_sms = g; h->stats.green_ctx_active = gc;
+    h->stats.granted_sms = g; h->stats.green_ctx_active = gc; h->stats.green_ctx_sms = gs;
     return EBRL_OK;
 }
 

@@ -227,3 +227,46 @@ def test_errors_and_busy_ids():
     st = r.gen.stats()
     assert st["groups"] == 2 and st["envs"] == 6 and st["kernel_launches"] > 0
     r.close()
+
+
+def test_bounded_wait_times_out_cleanly_and_context_survives():
+    """A wait that nothing satisfies gives up after its limit with EBRL_ERR_TIMEOUT in the status
+    word -- no trap, no hang -- and the device keeps working afterwards."""
+    rc, st, waited = B.wait_probe(50_000_000, signal_it=True)
+    assert rc == B.OK and st == B.OK and waited < 10_000_000
+    rc, st, waited = B.wait_probe(50_000_000, signal_it=False)          # 50 ms limit, nobody arrives
+    assert rc == B.OK and st == B.ERR_TIMEOUT
+    assert 40_000_000 <= waited <= 500_000_000
+    # the context is still usable: run a normal group
+    w = synth.scaled(synth.WORKLOADS[0], B=3)
+    wt, envs = _setup(w)
+    r = Runner(w, wt, envs)
+    got = stack(r.run([[0, 1, 2]]), range(3))
+    r.close()
+    assert chunk_rel_err(got, oracle_run(w, wt, envs)) <= TOL["f32"]
+    rc, _, _ = B.wait_probe(0, False)
+    assert rc == B.ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_sm_partition_gives_the_same_bits(dtype):
+    """With EBRL_FLAG_GREEN_CTX every batch runs inside a driver-enforced SM partition of at least
+    sm_quota SMs (where the driver offers green contexts; otherwise the grid cap alone applies).
+    Either way the results are the bits of the unpartitioned run."""
+    w = synth.scaled(synth.WORKLOADS[2], B=24, dtype=dtype, P=(64, 130), group=(1, 9))
+    wt, envs = _setup(w)
+    ids = list(range(w.B))
+    r = Runner(w, wt, envs)
+    base = stack(r.run([ids]), ids)
+    r.close()
+    r = Runner(w, wt, envs, flags=B.FLAG_GREEN_CTX, max_inflight_groups=2)
+    for q in (16, 37, 74):
+        got = stack(r.run(synth.arrival_groups(w, SEED), quota=q), ids)
+        assert np.array_equal(got, base), "quota %d" % q
+        st = r.gen.stats()
+        assert st["granted_sms"] == q
+        if st["green_ctx_active"]:
+            assert q <= st["green_ctx_sms"] <= 148
+    got = stack(r.run([ids], quota=0), ids)          # full chip: no partition needed
+    assert np.array_equal(got, base) and r.gen.stats()["green_ctx_active"] == 0
+    r.close()
