@@ -75,7 +75,9 @@ __global__ void __launch_bounds__(THREADS, 1) attn_mma_kernel(AttnArgs a, int hp
     const int KB = stage_keys(W);                 // keys per stage (a multiple of 16)
     const int stage_bytes = G * KB * 128;         // one box: [G][KB][128 B]
     const uint32_t sK = smem_u32(smem), sV = sK + NSTAGE * stage_bytes;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + 2 * NSTAGE * stage_bytes);
+    const uint32_t sQ = sV + NSTAGE * stage_bytes;   // per consumer warp: its head's queries, [16 rows][HD] bf16, 16-byte chunks swizzled
+    constexpr int Q_BYTES = 16 * HD * 2;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + 2 * NSTAGE * stage_bytes + MAXW * Q_BYTES);
     const uint32_t bar0 = smem_u32(bars);
     auto full = [&](int s) { return bar0 + 8u * s; };
     auto empty = [&](int s) { return bar0 + 8u * (NSTAGE + s); };
@@ -160,24 +162,40 @@ __global__ void __launch_bounds__(THREADS, 1) attn_mma_kernel(AttnArgs a, int hp
         const int g = lane >> 2, t = lane & 3;
         const float sc = 1.4426950408889634f / sqrtf((float)HD);   // log2(e) / sqrt(hd): scores in base-2 units
         int qbase = 0;                                              // stages consumed by earlier items
+        const uint32_t myq = sQ + (uint32_t)warp * Q_BYTES;
+        for (int i = lane; i < Q_BYTES / 16; i += 32)               // rows >= H are never copied: keep them zero
+            asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(myq + (uint32_t)i * 16), "r"(0u) : "memory");
+        __syncwarp();
+        // asynchronous copy of one item's queries of this warp's head: chunk c of row r goes to c ^ (r & 7)
+        auto fetch_q = [&](int it) {
+            const int e2 = it / nslab, hd2 = (it - e2 * nslab) * hpc + warp;
+            const __nv_bfloat16 *qb = (const __nv_bfloat16 *)a.q + (size_t)e2 * H * a.q_stride + hd2 * HD;
+            constexpr int CPR = HD / 8;   // 16-byte chunks per row
+            for (int idx = lane; idx < H * CPR; idx += 32) {
+                const int r = idx / CPR, cch = idx % CPR;
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(myq + (uint32_t)(r * (HD * 2) + ((cch ^ (r & 7)) << 4))),
+                             "l"(qb + (size_t)r * a.q_stride + cch * 8) : "memory");
+            }
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        };
+        if ((int)blockIdx.x < items) fetch_q(blockIdx.x);
         const int bps_sh = KB == 16 ? 0 : (KB == 32 ? 1 : 2), bps_mask = (1 << bps_sh) - 1;   // 16-key blocks per stage: 1, 2 or 4
         for (int item = blockIdx.x; item < items && ok; item += gridDim.x) {
             const int env = item / nslab, slab = item - env * nslab;
             const int P = a.self ? H : a.meta[env].P;
             const int head = slab * hpc + warp;
-            // Q fragments (A operand, 16 x HD), rows >= H are zero
+            // Q fragments (A operand, 16 x HD; rows >= H stay zero): this item's queries were copied
+            // into the warp's buffer asynchronously while the previous item was processed
             uint32_t qf[HD / 16][4];
-            {
-                const __nv_bfloat16 *qb = (const __nv_bfloat16 *)a.q + (size_t)env * H * a.q_stride + head * HD;
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+            __syncwarp();
 #pragma unroll
-                for (int ks = 0; ks < HD / 16; ++ks) {
-                    const int c = ks * 16 + 2 * t;
-                    qf[ks][0] = g < H ? *reinterpret_cast<const uint32_t *>(qb + (size_t)g * a.q_stride + c) : 0u;
-                    qf[ks][1] = g + 8 < H ? *reinterpret_cast<const uint32_t *>(qb + (size_t)(g + 8) * a.q_stride + c) : 0u;
-                    qf[ks][2] = g < H ? *reinterpret_cast<const uint32_t *>(qb + (size_t)g * a.q_stride + c + 8) : 0u;
-                    qf[ks][3] = g + 8 < H ? *reinterpret_cast<const uint32_t *>(qb + (size_t)(g + 8) * a.q_stride + c + 8) : 0u;
-                }
+            for (int ks = 0; ks < HD / 16; ++ks) {
+                const int qr = (lane & 7) + ((lane >> 3) & 1) * 8, qc = 2 * ks + (lane >> 4);
+                ldsm_x4(myq + (uint32_t)(qr * (HD * 2) + ((qc ^ (qr & 7)) << 4)), qf[ks][0], qf[ks][1], qf[ks][2], qf[ks][3]);
             }
+            __syncwarp();
+            if (item + (int)gridDim.x < items) fetch_q(item + gridDim.x);   // lands during this item
             float o[HD / 8][4];
 #pragma unroll
             for (int n = 0; n < HD / 8; ++n) { o[n][0] = o[n][1] = o[n][2] = o[n][3] = 0.f; }
@@ -341,7 +359,7 @@ cudaError_t launch_attn_mma(const AttnArgs &a, int grid, unsigned long long limi
     if (items == 0) return cudaSuccess;
     const int g = items < grid ? items : grid;
     const int W = hpc * a.hd;
-    const size_t smem = (size_t)2 * am::NSTAGE * am::stage_keys(W) * (W / 64) * 128 + 64 + 1024;
+    const size_t smem = (size_t)2 * am::NSTAGE * am::stage_keys(W) * (W / 64) * 128 + (size_t)am::MAXW * 16 * a.hd * 2 + 64 + 1024;
     // L2 look-ahead of the producer in key blocks (EBRL_ATTN_LOOKAHEAD overrides; 0 disables)
     static int la = -1;
     if (la < 0) {
