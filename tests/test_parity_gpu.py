@@ -270,3 +270,35 @@ def test_sm_partition_gives_the_same_bits(dtype):
     got = stack(r.run([ids], quota=0), ids)          # full chip: no partition needed
     assert np.array_equal(got, base) and r.gen.stats()["green_ctx_active"] == 0
     r.close()
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_per_layer_prefix_planes(dtype):
+    """kv_layers = n_layers: every layer cross-attends to its own K/V plane pair
+    ([L][2][P][d] per environment) instead of one shared pair."""
+    import oracle
+    from helpers import oracle_cfg, oracle_weights
+    w = synth.scaled(synth.WORKLOADS[0], B=7, dtype=dtype, L=3, P=(9, 70), mixed_steps=True)
+    wt = synth.make_weights(w, SEED, random_gains=True)
+    envs = [synth.make_env(w, e, SEED) for e in range(w.B)]
+    kvs = [synth.normal(SEED, "kv_per_layer", e.env_id, (w.L, 2, e.P, w.d), dtype=w.torch_dtype) for e in envs]
+    oc = oracle_cfg(w)
+    oc.kv_layers = w.L
+    ref = oracle.actgen(oc, oracle_weights(wt), [np32(k) for k in kvs], np.stack([np32(e.noise) for e in envs]),
+                        step_index=[e.step for e in envs])
+    cfg = B.cfg_for(w, max_group_envs=w.B, max_inflight_groups=2)
+    cfg.kv_layers = w.L
+    cfg.max_prefix_len = 70
+    gen = B.ActGen(cfg, wt)
+    noise = torch.stack([e.noise for e in envs]).cuda()
+    out = torch.empty_like(noise)
+    dkv = [k.cuda() for k in kvs]
+    gen.submit(list(range(4)), dkv[:4], noise[:4], out[:4], sm_quota=37, step_index=[e.step for e in envs[:4]])
+    gen.submit(list(range(4, 7)), dkv[4:], noise[4:], out[4:], sm_quota=37, step_index=[e.step for e in envs[4:]])
+    gen.sync()
+    gen.destroy()
+    assert chunk_rel_err(out.cpu().numpy(), ref) <= TOL[dtype]
+    # the planes really differ per layer: feeding layer 0's pair to every layer changes the result
+    ref_shared = oracle.actgen(oracle_cfg(w), oracle_weights(wt), [np32(k[:1]) for k in kvs], np.stack([np32(e.noise) for e in envs]),
+                               step_index=[e.step for e in envs])
+    assert np.abs(ref_shared - ref).max() > 1e-3
