@@ -137,6 +137,7 @@ typedef struct {
     uint64_t class_launches[EBRL_KC_COUNT];
     double class_flops[EBRL_KC_COUNT];    /* algorithmic 2*m*n*k FLOPs of those launches       */
     double class_bytes[EBRL_KC_COUNT];    /* algorithmic bytes of those launches               */
+    uint64_t weights_version;             /* policy version the last launched batch ran with   */
 } ebrl_actgen_stats_t;
 
 /* Validates cfg, copies the weights to the device (re-laid-out as the kernels want), builds
@@ -185,6 +186,22 @@ ebrl_status_t ebrl_actgen_submit_host(ebrl_actgen_t h, int32_t n_envs, const int
                                       const void *const *prefix_kv_host, const float *noise_host,
                                       float *out_host, int32_t sm_quota, void *stream,
                                       const ebrl_submit_ext_t *ext);
+
+/* Non-blocking weight publication (paper section 4.2.1: training publishes updated weights to
+ * the generation workers while rollout continues; the policy version a group ran with is the
+ * staleness bookkeeping of section 6).  The handle keeps two weight sets.  The call first
+ * launches the groups queued so far (they were submitted under the current version), then
+ * copies `weights` (host or device pointers, layout as at create) into the spare set
+ * asynchronously on `stream` and makes it the set every later batch uses; batches already
+ * launched keep running on the old set.  If the spare set is still being read by an earlier
+ * batch, the copy waits for it on the device, not on the host.  The caller's weight buffers
+ * must stay valid until `stream` has passed the copy (or until ebrl_actgen_sync).  Versions
+ * count from 1 (the weights given at create); *out_version (may be NULL) receives the new one.
+ * Pending uploads are device work: ebrl_actgen_sync does not wait for an update that no batch
+ * uses yet. */
+ebrl_status_t ebrl_actgen_update_weights(ebrl_actgen_t h, const ebrl_actgen_weights_t *weights, void *stream,
+                                         uint64_t *out_version);
+uint64_t ebrl_actgen_weights_version(ebrl_actgen_t h);
 
 /* Launches the queued groups now, without blocking. */
 ebrl_status_t ebrl_actgen_flush(ebrl_actgen_t h);

@@ -53,7 +53,7 @@ class Stats(C.Structure):
                 ("green_ctx_active", C.c_int32), ("green_ctx_sms", C.c_int32), ("reserved_", C.c_int32),
                 ("class_ms", C.c_double * 5),
                 ("class_launches", C.c_uint64 * 5), ("class_flops", C.c_double * 5),
-                ("class_bytes", C.c_double * 5)]
+                ("class_bytes", C.c_double * 5), ("weights_version", C.c_uint64)]
 
 
 class EbrlError(RuntimeError):
@@ -85,6 +85,9 @@ def lib():
         L.ebrl_actgen_submit_host.argtypes = sub
         L.ebrl_actgen_sync.argtypes = [C.c_void_p]
         L.ebrl_actgen_flush.argtypes = [C.c_void_p]
+        L.ebrl_actgen_update_weights.argtypes = [C.c_void_p, C.POINTER(Weights), C.c_void_p, C.POINTER(C.c_uint64)]
+        L.ebrl_actgen_weights_version.argtypes = [C.c_void_p]
+        L.ebrl_actgen_weights_version.restype = C.c_uint64
         L.ebrl_actgen_destroy.argtypes = [C.c_void_p]
         L.ebrl_actgen_get_stats.argtypes = [C.c_void_p, C.POINTER(Stats)]
         L.ebrl_actgen_reset_stats.argtypes = [C.c_void_p]
@@ -140,6 +143,15 @@ class ActGen:
         matrices in the configured dtype, gains and b_out fp32)."""
         self._L = lib()
         self.cfg = cfg
+        w, keep = self._marshal(weights)
+        self._h = C.c_void_p()
+        st = self._L.ebrl_actgen_create(C.byref(cfg), C.byref(w), C.byref(self._h))
+        if st != OK:
+            raise EbrlError(st, (self._L.ebrl_actgen_last_error(None) or b"").decode())
+        del keep
+
+    def _marshal(self, weights: dict):
+        cfg = self.cfg
         want = torch.bfloat16 if cfg.param_dtype == BF16 else torch.float32
         keep = []
 
@@ -154,13 +166,23 @@ class ActGen:
             lw[i] = LayerWeights(ptr(l["g1"], torch.float32), ptr(l["g2"], torch.float32), ptr(l["g3"], torch.float32),
                                  ptr(l["w_qkv"], want), ptr(l["w_o"], want), ptr(l["w_qc"], want),
                                  ptr(l["w_oc"], want), ptr(l["w_1"], want), ptr(l["w_2"], want))
+        keep.append(lw)
         w = Weights(ptr(weights["w_in"], want), ptr(weights["w_out"], want), ptr(weights["b_out"], torch.float32),
                     ptr(weights["g_final"], torch.float32), C.cast(lw, C.POINTER(LayerWeights)))
-        self._h = C.c_void_p()
-        st = self._L.ebrl_actgen_create(C.byref(cfg), C.byref(w), C.byref(self._h))
-        if st != OK:
-            raise EbrlError(st, (self._L.ebrl_actgen_last_error(None) or b"").decode())
-        del keep
+        return w, keep
+
+    def update_weights(self, weights: dict, stream: Optional[torch.cuda.Stream] = None) -> int:
+        """``ebrl_actgen_update_weights``: publish a new policy version without blocking; returns its
+        version number.  The tensors are kept alive by this object until the next update."""
+        w, keep = self._marshal(weights)
+        s = stream if stream is not None else torch.cuda.current_stream(self.cfg.device)
+        ver = C.c_uint64(0)
+        self._check(self._L.ebrl_actgen_update_weights(self._h, C.byref(w), s.cuda_stream, C.byref(ver)))
+        self._published = keep
+        return int(ver.value)
+
+    def weights_version(self) -> int:
+        return int(self._L.ebrl_actgen_weights_version(self._h))
 
     def _check(self, st):
         if st != OK:
@@ -218,7 +240,7 @@ class ActGen:
     def stats(self) -> dict:
         s = Stats()
         self._check(self._L.ebrl_actgen_get_stats(self._h, C.byref(s)))
-        out = {k: getattr(s, k) for k in ("groups", "envs", "env_steps", "kernel_launches", "granted_sms", "green_ctx_active", "green_ctx_sms")}
+        out = {k: getattr(s, k) for k in ("groups", "envs", "env_steps", "kernel_launches", "granted_sms", "green_ctx_active", "green_ctx_sms", "weights_version")}
         out["classes"] = {n: {"ms": s.class_ms[i], "launches": s.class_launches[i], "flops": s.class_flops[i],
                               "bytes": s.class_bytes[i]} for i, n in enumerate(KC_NAMES)}
         return out

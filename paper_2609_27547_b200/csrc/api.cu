@@ -28,6 +28,18 @@ struct LayerDev {
     TensorMap128 t_qkv, t_o, t_qc, t_oc, t_1, t_2;   // TMA descriptors of the matrices (tensor-core path)
 };
 
+// One complete copy of the policy's weights on the device.  The handle keeps two, so that a new
+// policy version can be uploaded while batches launched under the previous one still run.
+struct WeightSet {
+    void *w_in = nullptr, *w_out = nullptr;
+    float *b_out = nullptr, *g_final = nullptr;
+    std::vector<LayerDev> layers;
+    bool allocated = false, ever_used = false;
+    uint64_t version = 0;
+    cudaEvent_t ready = nullptr;      // upload complete
+    cudaEvent_t last_use = nullptr;   // last batch that reads this set
+};
+
 struct TimedLaunch {
     cudaEvent_t t0, t1;
     int cls;
@@ -78,9 +90,10 @@ struct ebrl_actgen {
     int *status_d = nullptr;      // device status word written by kernels whose waits ran out
     unsigned long long wait_ns = 0;
     size_t esz = 4;   // bytes per element of matrices / activations / planes
-    void *w_in = nullptr, *w_out = nullptr;
-    float *b_out = nullptr, *g_final = nullptr, *temb = nullptr;
-    std::vector<LayerDev> layers;
+    WeightSet wset[2];
+    int active = 0;               // the set new batches use
+    uint64_t version = 1;         // policy version of wset[active]
+    float *temb = nullptr;
     std::vector<Slot> slots;
     size_t fill = 0;              // slot collecting groups for the next batch
     std::unordered_set<int64_t> busy_ids;
@@ -223,6 +236,79 @@ ebrl_status_t dev_copy_in(ebrl_actgen *h, void **dst, const void *src, size_t by
     return EBRL_OK;
 }
 
+// Device buffers (and, on the tensor-core path, TMA descriptors) of one weight set.
+ebrl_status_t alloc_weight_set(ebrl_actgen *h, WeightSet &ws)
+{
+    const ebrl_actgen_cfg_t &c = h->cfg;
+    const size_t d = c.d, A = c.A, md = h->md, esz = h->esz;
+    ebrl_status_t st;
+    void *p = nullptr;
+    if ((st = dev_alloc(h, &ws.w_in, d * A * esz)) != EBRL_OK) return st;
+    if ((st = dev_alloc(h, &ws.w_out, A * d * esz)) != EBRL_OK) return st;
+    if ((st = dev_alloc(h, &p, A * 4)) != EBRL_OK) return st; ws.b_out = (float *)p;
+    if ((st = dev_alloc(h, &p, d * 4)) != EBRL_OK) return st; ws.g_final = (float *)p;
+    ws.layers.resize(c.n_layers);
+    for (LayerDev &o : ws.layers) {
+        if ((st = dev_alloc(h, &p, d * 4)) != EBRL_OK) return st; o.g1 = (float *)p;
+        if ((st = dev_alloc(h, &p, d * 4)) != EBRL_OK) return st; o.g2 = (float *)p;
+        if ((st = dev_alloc(h, &p, d * 4)) != EBRL_OK) return st; o.g3 = (float *)p;
+        if ((st = dev_alloc(h, &o.w_qkv, 3 * d * d * esz)) != EBRL_OK) return st;
+        if ((st = dev_alloc(h, &o.w_o, d * d * esz)) != EBRL_OK) return st;
+        if ((st = dev_alloc(h, &o.w_qc, d * d * esz)) != EBRL_OK) return st;
+        if ((st = dev_alloc(h, &o.w_oc, d * d * esz)) != EBRL_OK) return st;
+        if ((st = dev_alloc(h, &o.w_1, md * d * esz)) != EBRL_OK) return st;
+        if ((st = dev_alloc(h, &o.w_2, d * md * esz)) != EBRL_OK) return st;
+        if (h->use_tc) {
+            const uint32_t bw = (uint32_t)gemm_tc_box_rows_w();
+            int bad = make_tmap_bf16(&o.t_qkv, o.w_qkv, d, 3 * d, bw) | make_tmap_bf16(&o.t_o, o.w_o, d, d, bw) |
+                      make_tmap_bf16(&o.t_qc, o.w_qc, d, d, bw) | make_tmap_bf16(&o.t_oc, o.w_oc, d, d, bw) |
+                      make_tmap_bf16(&o.t_1, o.w_1, d, md, bw) | make_tmap_bf16(&o.t_2, o.w_2, md, d, bw);
+            if (bad) return fail(h, EBRL_ERR_CUDA, "cuTensorMapEncodeTiled failed for a weight matrix");
+        }
+    }
+    if (cudaEventCreateWithFlags(&ws.ready, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ws.last_use, cudaEventDisableTiming) != cudaSuccess)
+        return fail(h, EBRL_ERR_CUDA, "cudaEventCreate failed");
+    ws.allocated = true;
+    return EBRL_OK;
+}
+
+// Copies the caller's weights (host or device pointers) into a set, on `st` when async.
+ebrl_status_t upload_weight_set(ebrl_actgen *h, WeightSet &ws, const ebrl_actgen_weights_t *wts, cudaStream_t st, bool async)
+{
+    const ebrl_actgen_cfg_t &c = h->cfg;
+    const size_t d = c.d, A = c.A, md = h->md, esz = h->esz;
+    if (!wts || !wts->w_in || !wts->w_out || !wts->b_out || !wts->g_final || (c.n_layers > 0 && !wts->layers))
+        return fail(h, EBRL_ERR_INVALID_ARG, "a weight pointer is NULL");
+    for (int l = 0; l < c.n_layers; ++l) {
+        const ebrl_layer_weights_t &w = wts->layers[l];
+        if (!w.g1 || !w.g2 || !w.g3 || !w.w_qkv || !w.w_o || !w.w_qc || !w.w_oc || !w.w_1 || !w.w_2)
+            return fail(h, EBRL_ERR_INVALID_ARG, "a weight pointer of layer %d is NULL", l);
+    }
+    auto cp = [&](void *dst, const void *src, size_t bytes) {
+        return async ? cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDefault, st) : cudaMemcpy(dst, src, bytes, cudaMemcpyDefault);
+    };
+    cudaError_t e = cp(ws.w_in, wts->w_in, d * A * esz);
+    if (e == cudaSuccess) e = cp(ws.w_out, wts->w_out, A * d * esz);
+    if (e == cudaSuccess) e = cp(ws.b_out, wts->b_out, A * 4);
+    if (e == cudaSuccess) e = cp(ws.g_final, wts->g_final, d * 4);
+    for (int l = 0; l < c.n_layers && e == cudaSuccess; ++l) {
+        const ebrl_layer_weights_t &w = wts->layers[l];
+        LayerDev &o = ws.layers[l];
+        e = cp(o.g1, w.g1, d * 4);
+        if (e == cudaSuccess) e = cp(o.g2, w.g2, d * 4);
+        if (e == cudaSuccess) e = cp(o.g3, w.g3, d * 4);
+        if (e == cudaSuccess) e = cp(o.w_qkv, w.w_qkv, 3 * d * d * esz);
+        if (e == cudaSuccess) e = cp(o.w_o, w.w_o, d * d * esz);
+        if (e == cudaSuccess) e = cp(o.w_qc, w.w_qc, d * d * esz);
+        if (e == cudaSuccess) e = cp(o.w_oc, w.w_oc, d * d * esz);
+        if (e == cudaSuccess) e = cp(o.w_1, w.w_1, md * d * esz);
+        if (e == cudaSuccess) e = cp(o.w_2, w.w_2, d * md * esz);
+    }
+    if (e != cudaSuccess) return fail(h, EBRL_ERR_CUDA, "copying the weights failed: %s", cudaGetErrorString(e));
+    return EBRL_OK;
+}
+
 // Waits for a slot's group and folds its timing into the statistics.
 ebrl_status_t retire(ebrl_actgen *h, Slot &s)
 {
@@ -293,15 +379,16 @@ cudaError_t enqueue_batch(ebrl_actgen *h, Slot &s, int S, const int32_t *n_activ
     const bool pull = (c.flags & EBRL_FLAG_TEST_PULL) != 0;
     const double esz = (double)h->esz;
     Launcher ln{h, &s, st, grid, (c.flags & EBRL_FLAG_TIMING) != 0};
+    const WeightSet &W = h->wset[h->active];
     for (int step = 0; step < S; ++step) {
         const int ne = n_active[step], M = ne * H;
         if (ne == 0) break;
         if (!pull) {
-            EmbedArgs ea{s.meta_d, ne, H, c.A, d, step, s.a_state, h->w_in, h->temb,
-                         L > 0 ? h->layers[0].g1 : h->g_final, s.x, s.xg, s.ssq};
+            EmbedArgs ea{s.meta_d, ne, H, c.A, d, step, s.a_state, W.w_in, h->temb,
+                         L > 0 ? W.layers[0].g1 : W.g_final, s.x, s.xg, s.ssq};
             ln.run(EBRL_KC_EMBED, 2.0 * M * d * c.A, (double)M * d * (4 + esz), [&] { return launch_embed(ea, bf, grid, st); });
             for (int l = 0; l < L; ++l) {
-                const LayerDev &w = h->layers[l];
+                const LayerDev &w = W.layers[l];
                 auto gemm = [&](const void *A, const TensorMap128 &tA, const void *W, const TensorMap128 &tW, int N, int K, int epi,
                                 void *C, const float *gain) {
                     GemmArgs g{};
@@ -344,10 +431,10 @@ cudaError_t enqueue_batch(ebrl_actgen *h, Slot &s, int S, const int32_t *n_activ
                 gemm(s.att, s.t_att, w.w_oc, w.t_oc, d, d, EPI_RESID, nullptr, w.g3);
                 // MLP block
                 gemm(s.xg, s.t_xg, w.w_1, w.t_1, md, d, EPI_SCALE_GELU, s.u, nullptr);
-                gemm(s.u, s.t_u, w.w_2, w.t_2, d, md, EPI_RESID, nullptr, (l + 1 < L) ? h->layers[l + 1].g1 : h->g_final);
+                gemm(s.u, s.t_u, w.w_2, w.t_2, d, md, EPI_RESID, nullptr, (l + 1 < L) ? W.layers[l + 1].g1 : W.g_final);
             }
         }
-        HeadArgs ha{s.meta_d, ne, H, c.A, d, step, c.K_steps, s.a_state, s.x, h->g_final, h->w_out, h->b_out, c.rms_eps, pull ? 1 : 0};
+        HeadArgs ha{s.meta_d, ne, H, c.A, d, step, c.K_steps, s.a_state, s.x, W.g_final, W.w_out, W.b_out, c.rms_eps, pull ? 1 : 0};
         ln.run(EBRL_KC_HEAD, 2.0 * M * d * c.A, (double)M * d * 4, [&] { return launch_head(ha, bf, grid, st); });
     }
     return ln.err;
@@ -395,6 +482,9 @@ ebrl_status_t flush_slot(ebrl_actgen *h, Slot &s)
     }
     h->stats.green_ctx_active = gp ? 1 : 0;
     h->stats.green_ctx_sms = gp ? gp->sm_count : 0;
+    WeightSet &wsel = h->wset[h->active];
+    if (wsel.version > 1) CK(cudaStreamWaitEvent(cs, wsel.ready, 0));   // a published version: its upload must have landed
+    h->stats.weights_version = wsel.version;
     if (s.has_uploads) {   // the batch's kernels wait for the uploads issued on the copy stream
         CK(cudaEventRecord(s.h2d_done, h->copy_stream));
         CK(cudaStreamWaitEvent(cs, s.h2d_done, 0));
@@ -413,6 +503,8 @@ ebrl_status_t flush_slot(ebrl_actgen *h, Slot &s)
         h->sticky = EBRL_ERR_CUDA;
         return fail(h, EBRL_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
     }
+    CK(cudaEventRecord(wsel.last_use, cs));
+    wsel.ever_used = true;
     if (gp) {
         CK(cudaEventRecord(s.part_out, cs));
         CK(cudaStreamWaitEvent(user, s.part_out, 0));
@@ -548,6 +640,11 @@ void free_all(ebrl_actgen *h)
         if (s.kv_stage) cudaFree(s.kv_stage);
         for (TimedLaunch &t : s.timed) { if (t.t0) cudaEventDestroy(t.t0); if (t.t1) cudaEventDestroy(t.t1); }
     }
+    for (WeightSet &ws : h->wset) {
+        if (ws.ready) cudaEventDestroy(ws.ready);
+        if (ws.last_use) cudaEventDestroy(ws.last_use);
+        ws.ready = ws.last_use = nullptr;
+    }
     for (auto &kv : h->partitions) green_partition_destroy(&kv.second);
     h->partitions.clear();
     if (h->copy_stream) cudaStreamDestroy(h->copy_stream);
@@ -629,26 +726,15 @@ ebrl_status_t ebrl_actgen_create(const ebrl_actgen_cfg_t *cfg, const ebrl_actgen
         cudaGetLastError();
         return bail(EBRL_ERR_CUDA);
     }
-    const int d = cfg->d, A = cfg->A, md = h->md, L = cfg->n_layers;
+    const int d = cfg->d, A = cfg->A, md = h->md;
     const size_t esz = h->esz;
-    if ((st = dev_copy_in(h, &h->w_in, wts->w_in, (size_t)d * A * esz)) != EBRL_OK) return bail(st);
-    if ((st = dev_copy_in(h, &h->w_out, wts->w_out, (size_t)A * d * esz)) != EBRL_OK) return bail(st);
-    if ((st = dev_copy_in(h, (void **)&h->b_out, wts->b_out, (size_t)A * 4)) != EBRL_OK) return bail(st);
-    if ((st = dev_copy_in(h, (void **)&h->g_final, wts->g_final, (size_t)d * 4)) != EBRL_OK) return bail(st);
-    h->layers.resize(L);
-    for (int l = 0; l < L; ++l) {
-        const ebrl_layer_weights_t &w = wts->layers[l];
-        LayerDev &o = h->layers[l];
-        if ((st = dev_copy_in(h, (void **)&o.g1, w.g1, (size_t)d * 4)) != EBRL_OK) return bail(st);
-        if ((st = dev_copy_in(h, (void **)&o.g2, w.g2, (size_t)d * 4)) != EBRL_OK) return bail(st);
-        if ((st = dev_copy_in(h, (void **)&o.g3, w.g3, (size_t)d * 4)) != EBRL_OK) return bail(st);
-        if ((st = dev_copy_in(h, &o.w_qkv, w.w_qkv, (size_t)3 * d * d * esz)) != EBRL_OK) return bail(st);
-        if ((st = dev_copy_in(h, &o.w_o, w.w_o, (size_t)d * d * esz)) != EBRL_OK) return bail(st);
-        if ((st = dev_copy_in(h, &o.w_qc, w.w_qc, (size_t)d * d * esz)) != EBRL_OK) return bail(st);
-        if ((st = dev_copy_in(h, &o.w_oc, w.w_oc, (size_t)d * d * esz)) != EBRL_OK) return bail(st);
-        if ((st = dev_copy_in(h, &o.w_1, w.w_1, (size_t)md * d * esz)) != EBRL_OK) return bail(st);
-        if ((st = dev_copy_in(h, &o.w_2, w.w_2, (size_t)d * md * esz)) != EBRL_OK) return bail(st);
-    }
+    h->use_tc = h->bf16 && !(cfg->flags & EBRL_FLAG_FORCE_SIMT) && gemm_tc_supported(d, d) && gemm_tc_supported(md, d) &&
+                gemm_tc_supported(d, md) && gemm_tc_supported(3 * d, d);
+    if (const char *e2 = getenv("EBRL_GEMM_PAIR")) h->use_pairs = atoi(e2) != 0;
+    h->use_attn_mma = h->bf16 && !(cfg->flags & EBRL_FLAG_FORCE_SIMT) && attn_mma_supported(cfg->H, cfg->n_heads, h->hd);
+    if ((st = alloc_weight_set(h, h->wset[0])) != EBRL_OK) return bail(st);
+    if ((st = upload_weight_set(h, h->wset[0], wts, nullptr, false)) != EBRL_OK) return bail(st);
+    h->wset[0].version = 1;
     {   // timestep-embedding table [K][d], evaluated in double on the host and rounded once
         std::vector<float> t((size_t)cfg->K_steps * d);
         const int half = d / 2;
@@ -672,24 +758,6 @@ ebrl_status_t ebrl_actgen_create(const ebrl_actgen_cfg_t *cfg, const ebrl_actgen
         if ((st = dev_alloc(h, &p, 16)) != EBRL_OK) return bail(st);
         h->status_d = (int *)p;
         if (cudaMemset(h->status_d, 0, 16) != cudaSuccess) { fail(h, EBRL_ERR_CUDA, "cudaMemset failed"); return bail(EBRL_ERR_CUDA); }
-    }
-    h->use_tc = h->bf16 && !(cfg->flags & EBRL_FLAG_FORCE_SIMT) && gemm_tc_supported(d, d) && gemm_tc_supported(md, d) &&
-                gemm_tc_supported(d, md) && gemm_tc_supported(3 * d, d);
-    if (const char *e = getenv("EBRL_GEMM_PAIR")) h->use_pairs = atoi(e) != 0;
-    h->use_attn_mma = h->bf16 && !(cfg->flags & EBRL_FLAG_FORCE_SIMT) && attn_mma_supported(cfg->H, cfg->n_heads, h->hd);
-    if (h->use_tc) {
-        const uint32_t bw = (uint32_t)gemm_tc_box_rows_w();
-        int bad = 0;
-        for (int l = 0; l < L; ++l) {
-            LayerDev &o = h->layers[l];
-            bad |= make_tmap_bf16(&o.t_qkv, o.w_qkv, d, 3 * (uint64_t)d, bw);
-            bad |= make_tmap_bf16(&o.t_o, o.w_o, d, d, bw);
-            bad |= make_tmap_bf16(&o.t_qc, o.w_qc, d, d, bw);
-            bad |= make_tmap_bf16(&o.t_oc, o.w_oc, d, d, bw);
-            bad |= make_tmap_bf16(&o.t_1, o.w_1, d, md, bw);
-            bad |= make_tmap_bf16(&o.t_2, o.w_2, md, d, bw);
-        }
-        if (bad) { fail(h, EBRL_ERR_CUDA, "cuTensorMapEncodeTiled failed for a weight matrix"); return bail(EBRL_ERR_CUDA); }
     }
     if (cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking) != cudaSuccess) {
         fail(h, EBRL_ERR_CUDA, "cudaStreamCreate failed");
@@ -835,9 +903,39 @@ ebrl_status_t ebrl_actgen_reset_stats(ebrl_actgen_t h)
     if (!h) return EBRL_ERR_INVALID_ARG;
     std::lock_guard<std::mutex> lk(h->mu);
     const int32_t g = h->stats.granted_sms, gc = h->stats.green_ctx_active, gs = h->stats.green_ctx_sms;
+    const uint64_t wv = h->stats.weights_version;
     memset(&h->stats, 0, sizeof h->stats);
+    h->stats.weights_version = wv;
     h->stats.granted_sms = g; h->stats.green_ctx_active = gc; h->stats.green_ctx_sms = gs;
     return EBRL_OK;
+}
+
+ebrl_status_t ebrl_actgen_update_weights(ebrl_actgen_t h, const ebrl_actgen_weights_t *weights, void *stream, uint64_t *out_version)
+{
+    if (!h) return EBRL_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lk(h->mu);
+    if (h->sticky != EBRL_OK) return fail(h, h->sticky, "handle is in a failed state: %s", h->err.c_str());
+    CK(cudaSetDevice(h->cfg.device));
+    // groups queued so far were submitted under the current version: launch them with it
+    ebrl_status_t st = flush_slot(h, h->slots[h->fill]);
+    if (st != EBRL_OK) return st;
+    WeightSet &t = h->wset[1 - h->active];
+    if (!t.allocated && (st = alloc_weight_set(h, t)) != EBRL_OK) return st;
+    cudaStream_t cs = (cudaStream_t)stream;
+    if (t.ever_used) CK(cudaStreamWaitEvent(cs, t.last_use, 0));   // batches still reading the set being replaced
+    if ((st = upload_weight_set(h, t, weights, cs, true)) != EBRL_OK) return st;
+    CK(cudaEventRecord(t.ready, cs));
+    h->active = 1 - h->active;
+    t.version = ++h->version;
+    if (out_version) *out_version = t.version;
+    return EBRL_OK;
+}
+
+uint64_t ebrl_actgen_weights_version(ebrl_actgen_t h)
+{
+    if (!h) return 0;
+    std::lock_guard<std::mutex> lk(h->mu);
+    return h->version;
 }
 
 ebrl_status_t ebrl_actgen_set_timing(ebrl_actgen_t h, int32_t on)

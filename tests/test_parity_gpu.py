@@ -302,3 +302,38 @@ def test_per_layer_prefix_planes(dtype):
     ref_shared = oracle.actgen(oracle_cfg(w), oracle_weights(wt), [np32(k[:1]) for k in kvs], np.stack([np32(e.noise) for e in envs]),
                                step_index=[e.step for e in envs])
     assert np.abs(ref_shared - ref).max() > 1e-3
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_weight_publication_switches_versions_between_batches(dtype):
+    """A new policy version is uploaded while earlier groups are still queued or running: groups
+    submitted before the update run with the old weights, groups submitted after it with the new
+    ones, and a third update reuses the first set.  Results equal those of fresh handles, bit for bit."""
+    w = synth.scaled(synth.WORKLOADS[0], B=10, dtype=dtype, P=(20, 60))
+    wA = synth.make_weights(w, 101, random_gains=True)
+    wB = synth.make_weights(w, 202, random_gains=True)
+    envs = [synth.make_env(w, e, SEED) for e in range(w.B)]
+    ids = list(range(w.B))
+    refs = {}
+    for name, wt in (("A", wA), ("B", wB)):
+        r = Runner(w, wt, envs)
+        refs[name] = stack(r.run([ids]), ids)
+        r.close()
+    assert not np.array_equal(refs["A"], refs["B"])
+    r = Runner(w, wA, envs, max_inflight_groups=4)
+    assert r.gen.weights_version() == 1
+    noise = torch.stack([r.noise[e] for e in ids])
+    out1, out2 = torch.empty_like(noise), torch.empty_like(noise)
+    kv = [r.kv[e] for e in ids]
+    r.gen.submit(ids[:6], kv[:6], noise[:6], out1[:6])                 # queued under version 1
+    side = torch.cuda.Stream()
+    assert r.gen.update_weights(wB, stream=side) == 2                     # launches the queued group, then uploads on a side stream
+    r.gen.submit([100 + e for e in ids], kv, noise, out2)                # runs with version 2
+    r.gen.sync()
+    assert np.array_equal(out1[:6].cpu().numpy(), refs["A"][:6])
+    assert np.array_equal(out2.cpu().numpy(), refs["B"])
+    assert r.gen.stats()["weights_version"] == 2 and r.gen.weights_version() == 2
+    assert r.gen.update_weights(wA) == 3                                  # the first set is overwritten only after its readers
+    got = stack(r.run([ids]), ids)
+    assert np.array_equal(got, refs["A"]) and r.gen.stats()["weights_version"] == 3
+    r.close()
