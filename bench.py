@@ -67,6 +67,8 @@ def parse_args():
     ap.add_argument("--corunner", action="store_true", help="run the streaming co-runner on the other SMs")
     ap.add_argument("--simt", action="store_true", help="force the plain-ALU kernels")
     ap.add_argument("--green-ctx", action="store_true", help="run inside an SM partition (green context) of the quota")
+    ap.add_argument("--pgen-sweep", action="store_true",
+                    help="emit the generation profile P_gen(s_g, B_g): chunks/s on a grid of SM quotas and group sizes")
     ap.add_argument("--min-warmup", type=int, default=3, help="lower bound on warm-up steps (profiling captures use 1)")
     ap.add_argument("--inflight", type=int, default=8, help="groups queued before a batch is launched")
     return ap.parse_args()
@@ -378,8 +380,51 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_pgen_sweep(args):
+    """The paper's generation profiling (section 4.3.2: observation batches replayed under different SM
+    quotas and batch sizes, stored in a lookup table): chunks/s of one group of B_g environments at
+    quota s_g, on the programming model's example grid (20/40/60/80 % x 8/16/32/64).  The table is the
+    P_gen input of ebrl_alloc_elastic."""
+    import torch
+    from paper_2609_27547_b200 import binding as B
+    from paper_2609_27547_b200 import synth
+    torch.cuda.set_device(0)
+    w = synth.WORKLOADS[args.config]
+    seed = args.seed or synth.DEFAULT_SEED
+    quotas, batches = [20, 40, 60, 80], [8, 16, 32, 64]
+    wt = synth.make_weights(w, seed, device="cuda")
+    envs = [synth.make_env(w, e, seed, device="cuda") for e in range(max(batches))]
+    gen = B.ActGen(B.cfg_for(w, max_group_envs=max(batches), max_inflight_groups=1), wt)
+    stream = torch.cuda.Stream()
+    noise = torch.stack([e.noise for e in envs]).contiguous()
+    out = torch.empty_like(noise)
+    rate = []
+    for q in quotas:
+        sms = max(1, round(N_SMS * q / 100))
+        row = []
+        for b in batches:
+            def step():
+                gen.submit(list(range(b)), [e.kv for e in envs[:b]], noise[:b], out[:b], sm_quota=sms, stream=stream)
+                gen.sync()
+            for _ in range(3):
+                step()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(args.steps):
+                step()
+            e1.record(stream)
+            torch.cuda.synchronize()
+            row.append(b * args.steps / (e0.elapsed_time(e1) * 1e-3))
+        rate.append(row)
+    gen.destroy()
+    print(json.dumps({"pgen": {"workload": "configs[%d] %s" % (args.config, w.name), "unit": UNIT, "quota_pct": quotas,
+                               "quota_sms": [max(1, round(N_SMS * q / 100)) for q in quotas], "batch": batches, "rate": rate}}))
+
+
 def main():
     args = parse_args()
+    if args.pgen_sweep:
+        return run_pgen_sweep(args)
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -15,15 +15,20 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 def _declared_symbols():
-    text = open(os.path.join(ROOT, "include", "ebrl_actgen.h")).read()
-    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(ebrl_[a-z0-9_]+)\s*\(", text)))
+    names = set()
+    inc = os.path.join(ROOT, "include")
+    for fn in sorted(os.listdir(inc)):
+        if fn.endswith(".h"):
+            text = open(os.path.join(inc, fn)).read()
+            text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+            names.update(re.findall(r"\b(ebrl_[a-z0-9_]+)\s*\(", text))
+    return sorted(names)
 
 
 def test_library_exports_every_declared_symbol():
     names = _declared_symbols()
     assert "ebrl_actgen_create" in names and "ebrl_actgen_submit" in names and "ebrl_actgen_sync" in names
-    assert len(names) >= 14
+    assert len(names) >= 24 and "ebrl_alloc_elastic" in names and "ebrl_actgen_update_weights" in names
     lib = B.lib()
     for n in names:
         assert hasattr(lib, n), n
