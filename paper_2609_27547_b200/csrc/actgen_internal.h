@@ -101,7 +101,7 @@ int make_tmap_bf16(TensorMap128 *out, const void *base, uint64_t inner, uint64_t
 bool gemm_tc_supported(int N, int K);
 int gemm_tc_box_rows_a();
 int gemm_tc_box_rows_w();
-cudaError_t launch_gemm_tc(const TensorMap128 &ta, const TensorMap128 &tw, const GemmArgs &a, int grid,
+cudaError_t launch_gemm_tc(const TensorMap128 &ta, const TensorMap128 &tw, const GemmArgs &a, int grid, int bn,
                            unsigned long long limit_ns, int *status, cudaStream_t st);
 
 // The same GEMM on CTA pairs (tcgen05 cta_group::2, 256 x 256 tiles); needs grid >= 2.

@@ -85,7 +85,8 @@ struct ebrl_actgen {
     ebrl_actgen_cfg_t cfg;
     int bf16 = 0, n_sms = 0, hd = 0, md = 0;
     bool use_tc = false;          // tensor-core GEMMs (bf16, d a multiple of 256)
-    bool use_pairs = true;        // CTA-pair GEMM (EBRL_GEMM_PAIR=0 selects one CTA per tile)
+    bool use_pairs = true;        // CTA-pair GEMM allowed (EBRL_GEMM_PAIR=0 forbids it)
+    int force_shape = 0;          // EBRL_GEMM_SHAPE = 2 (pairs), 256 or 128 forces one tile shape (tests, tuning)
     bool use_attn_mma = false;    // tensor-core attention (bf16, H <= 16, head_dim 64/128)
     int *status_d = nullptr;      // device status word written by kernels whose waits ran out
     unsigned long long wait_ns = 0;
@@ -396,10 +397,21 @@ cudaError_t enqueue_batch(ebrl_actgen *h, Slot &s, int S, const int32_t *n_activ
                     g.ssq_in = s.ssq; g.n_ssq = nseg; g.inv_d = 1.0f / (float)d; g.eps = c.rms_eps;
                     g.C = C; g.x = s.x; g.gain = gain; g.xg = s.xg; g.ssq_out = s.ssq;
                     const double bytes = ((double)M * K + (double)N * K + (double)M * N) * esz + (epi == EPI_RESID ? 8.0 * M * N : 0.0);
-                    if (h->use_tc && h->use_pairs && grid >= 2)
-                        ln.run(EBRL_KC_GEMM, 2.0 * M * N * K, bytes, [&] { return launch_gemm_tc2(tA, tW, g, grid, h->wait_ns, h->status_d, st); });
-                    else if (h->use_tc)
-                        ln.run(EBRL_KC_GEMM, 2.0 * M * N * K, bytes, [&] { return launch_gemm_tc(tA, tW, g, grid, h->wait_ns, h->status_d, st); });
+                    if (h->use_tc) {
+                        // tile shape by estimated time = waves x tile area / relative efficiency (the
+                        // accumulation order per output element is the same for every shape, so the
+                        // choice does not change a single bit of the result)
+                        const long mt = (M + 127) / 128, mp = (M + 255) / 256;
+                        const long pairs = grid / 2;
+                        const double t_pair = (h->use_pairs && pairs >= 1) ? (double)((mp * (N / 256) + pairs - 1) / pairs) * 32768.0 / 1.0 : 1e30;
+                        const double t_256 = (double)((mt * (N / 256) + grid - 1) / grid) * 32768.0 / 0.88;
+                        const double t_128 = (double)((mt * (N / 128) + grid - 1) / grid) * 16384.0 / 0.72;
+                        const int shape = h->force_shape ? h->force_shape : (t_pair <= t_256 && t_pair <= t_128 ? 2 : (t_256 <= t_128 ? 256 : 128));
+                        if (shape == 2)
+                            ln.run(EBRL_KC_GEMM, 2.0 * M * N * K, bytes, [&] { return launch_gemm_tc2(tA, tW, g, grid, h->wait_ns, h->status_d, st); });
+                        else
+                            ln.run(EBRL_KC_GEMM, 2.0 * M * N * K, bytes, [&] { return launch_gemm_tc(tA, tW, g, grid, shape, h->wait_ns, h->status_d, st); });
+                    }
                     else
                         ln.run(EBRL_KC_GEMM, 2.0 * M * N * K, bytes, [&] { return launch_gemm_simt(g, bf, grid, st); });
                 };
@@ -731,6 +743,7 @@ ebrl_status_t ebrl_actgen_create(const ebrl_actgen_cfg_t *cfg, const ebrl_actgen
     h->use_tc = h->bf16 && !(cfg->flags & EBRL_FLAG_FORCE_SIMT) && gemm_tc_supported(d, d) && gemm_tc_supported(md, d) &&
                 gemm_tc_supported(d, md) && gemm_tc_supported(3 * d, d);
     if (const char *e2 = getenv("EBRL_GEMM_PAIR")) h->use_pairs = atoi(e2) != 0;
+    if (const char *e3 = getenv("EBRL_GEMM_SHAPE")) { const int v = atoi(e3); if (v == 2 || v == 256 || v == 128) h->force_shape = v; }
     h->use_attn_mma = h->bf16 && !(cfg->flags & EBRL_FLAG_FORCE_SIMT) && attn_mma_supported(cfg->H, cfg->n_heads, h->hd);
     if ((st = alloc_weight_set(h, h->wset[0])) != EBRL_OK) return bail(st);
     if ((st = upload_weight_set(h, h->wset[0], wts, nullptr, false)) != EBRL_OK) return bail(st);

@@ -22,11 +22,19 @@ namespace tc {
 
 using namespace ptx;
 
-constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4, UMMA_K = 16;
-constexpr int THREADS = 320;          // TMA warp, MMA warp, 8 epilogue warps
-constexpr int EPI_WARPS = 8;
-constexpr int A_BYTES = BM * BK * 2, B_BYTES = BN * BK * 2;
-constexpr int SMEM_BYTES = STAGES * (A_BYTES + B_BYTES) + 256 + 1024 + EPI_WARPS * EPI_STAGE_FLOATS * 4;   // + barriers + alignment slack
+constexpr int BM = 128, BK = 64, UMMA_K = 16;
+constexpr int A_BYTES = BM * BK * 2;
+
+// Tile shapes: 128 x 256 (4 stages of 48 KB, 8 epilogue warps: lane quarter x column half) and
+// 128 x 128 (6 stages of 32 KB, 4 epilogue warps) for GEMMs with too few tiles to fill the grid.
+template <int BN> struct Shape {
+    static constexpr int STAGES = BN == 256 ? 4 : 6;
+    static constexpr int EPI_WARPS = BN / 128 * 4;
+    static constexpr int THREADS = 64 + 32 * EPI_WARPS;   // TMA warp, MMA warp, epilogue warps
+    static constexpr int B_BYTES = BN * BK * 2;
+    static constexpr int SMEM_BYTES = STAGES * (A_BYTES + B_BYTES) + 256 + 1024 + EPI_WARPS * EPI_STAGE_FLOATS * 4;   // + barriers + alignment slack
+    static constexpr uint32_t TMEM_COLS = 2 * BN;
+};
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tm, uint32_t bar, int c0, int c1)
 {
@@ -60,11 +68,12 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N)
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
-template <int EPI>
-__global__ void __launch_bounds__(THREADS, 1)
+template <int EPI, int BN>
+__global__ void __launch_bounds__(Shape<BN>::THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmArgs g,
                unsigned long long limit_ns, int *status)
 {
+    constexpr int STAGES = Shape<BN>::STAGES, EPI_WARPS = Shape<BN>::EPI_WARPS, B_BYTES = Shape<BN>::B_BYTES;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t sA = smem_u32(smem), sB = sA + STAGES * A_BYTES;
@@ -89,7 +98,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmB)) : "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void *)tmem_slot)), "r"(512u) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void *)tmem_slot)), "r"(Shape<BN>::TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
@@ -109,8 +118,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 if (lane == 0) {
                     mbar_expect_tx(full(stage), A_BYTES + B_BYTES);
                     tma_load_2d(sA + stage * A_BYTES, &tmA, full(stage), kb * BK, m0);
-                    tma_load_2d(sB + stage * B_BYTES, &tmB, full(stage), kb * BK, n0);                      // weight rows n0 .. n0+127
-                    tma_load_2d(sB + stage * B_BYTES + B_BYTES / 2, &tmB, full(stage), kb * BK, n0 + BN / 2);   // and n0+128 .. n0+255
+                    tma_load_2d(sB + stage * B_BYTES, &tmB, full(stage), kb * BK, n0);   // weight rows n0 .. n0+127 (128-row boxes)
+                    if (BN == 256) tma_load_2d(sB + stage * B_BYTES + B_BYTES / 2, &tmB, full(stage), kb * BK, n0 + 128);
                 }
                 __syncwarp();
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -147,14 +156,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
     } else {
         // ---- epilogue: warp w reads TMEM lanes 32 (w % 4) .. +31 and half of the tile's columns; one thread per row
-        const int q = warp & 3, half = (warp - 2) >> 2;
+        const int q = warp & 3, half = (warp - 2) >> 2;   // half is 0 for the 128-column shape
         float *stg = reinterpret_cast<float *>(smem + STAGES * (A_BYTES + B_BYTES) + 256) + (warp - 2) * EPI_STAGE_FLOATS;
         int it = 0;
         for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++it) {
             const int buf = it & 1;
             const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
-            const int m0 = (tile / ntn) * BM, n0 = (tile % ntn) * BN + half * (BN / 2);
-            if (!epilogue_rows<EPI, BN / 2>(g, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + half * (BN / 2)), m0 + q * 32, n0, stg,
+            const int m0 = (tile / ntn) * BM, n0 = (tile % ntn) * BN + half * 128;
+            if (!epilogue_rows<EPI, 128>(g, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + half * 128), m0 + q * 32, n0, stg,
                                             [&] { return __all_sync(0xffffffffu, mbar_wait(tfull(buf), acc_phase, limit_ns, abort_flag)) != 0; })) {
                 ok = false;
                 break;
@@ -180,7 +189,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(Shape<BN>::TMEM_COLS) : "memory");
     }
 }
 
@@ -220,35 +229,43 @@ int make_tmap_bf16(TensorMap128 *out, const void *base, uint64_t inner, uint64_t
     return r == CUDA_SUCCESS ? 0 : 2;
 }
 
-bool gemm_tc_supported(int N, int K) { return N % tc::BN == 0 && K % tc::BK == 0; }
+bool gemm_tc_supported(int N, int K) { return N % 256 == 0 && K % tc::BK == 0; }
 int gemm_tc_box_rows_a() { return tc::BM; }
-int gemm_tc_box_rows_w() { return tc::BN / 2; }   // weight maps serve both kernels: 128-row boxes
+int gemm_tc_box_rows_w() { return 128; }   // weight maps serve every kernel: 128-row boxes
 
-template <int EPI>
+template <int EPI, int BN>
 static cudaError_t tc_launch(const TensorMap128 &ta, const TensorMap128 &tw, const GemmArgs &a, int g, unsigned long long limit_ns,
                              int *status, cudaStream_t st)
 {
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(tc::gemm_tc_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_BYTES);
+        cudaError_t e = cudaFuncSetAttribute(tc::gemm_tc_kernel<EPI, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::Shape<BN>::SMEM_BYTES);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    tc::gemm_tc_kernel<EPI><<<g, tc::THREADS, tc::SMEM_BYTES, st>>>(*reinterpret_cast<const CUtensorMap *>(&ta),
-                                                                    *reinterpret_cast<const CUtensorMap *>(&tw), a, limit_ns, status);
+    tc::gemm_tc_kernel<EPI, BN><<<g, tc::Shape<BN>::THREADS, tc::Shape<BN>::SMEM_BYTES, st>>>(
+        *reinterpret_cast<const CUtensorMap *>(&ta), *reinterpret_cast<const CUtensorMap *>(&tw), a, limit_ns, status);
     return cudaGetLastError();
 }
 
-cudaError_t launch_gemm_tc(const TensorMap128 &ta, const TensorMap128 &tw, const GemmArgs &a, int grid, unsigned long long limit_ns,
+// One CTA per tile; bn = 256 or 128 columns per tile.
+cudaError_t launch_gemm_tc(const TensorMap128 &ta, const TensorMap128 &tw, const GemmArgs &a, int grid, int bn, unsigned long long limit_ns,
                            int *status, cudaStream_t st)
 {
     if (a.M == 0) return cudaSuccess;
-    const int tiles = ((a.M + tc::BM - 1) / tc::BM) * (a.N / tc::BN);
+    const int tiles = ((a.M + tc::BM - 1) / tc::BM) * (a.N / bn);
     const int g = tiles < grid ? tiles : grid;
+    if (bn == 256) {
+        switch (a.epi) {
+        case EPI_SCALE_STORE: return tc_launch<EPI_SCALE_STORE, 256>(ta, tw, a, g, limit_ns, status, st);
+        case EPI_SCALE_GELU: return tc_launch<EPI_SCALE_GELU, 256>(ta, tw, a, g, limit_ns, status, st);
+        default: return tc_launch<EPI_RESID, 256>(ta, tw, a, g, limit_ns, status, st);
+        }
+    }
     switch (a.epi) {
-    case EPI_SCALE_STORE: return tc_launch<EPI_SCALE_STORE>(ta, tw, a, g, limit_ns, status, st);
-    case EPI_SCALE_GELU: return tc_launch<EPI_SCALE_GELU>(ta, tw, a, g, limit_ns, status, st);
-    default: return tc_launch<EPI_RESID>(ta, tw, a, g, limit_ns, status, st);
+    case EPI_SCALE_STORE: return tc_launch<EPI_SCALE_STORE, 128>(ta, tw, a, g, limit_ns, status, st);
+    case EPI_SCALE_GELU: return tc_launch<EPI_SCALE_GELU, 128>(ta, tw, a, g, limit_ns, status, st);
+    default: return tc_launch<EPI_RESID, 128>(ta, tw, a, g, limit_ns, status, st);
     }
 }
 
