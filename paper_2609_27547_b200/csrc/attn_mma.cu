@@ -242,25 +242,30 @@ __global__ void __launch_bounds__(THREADS, 1) attn_mma_kernel(AttnArgs a, int hp
                     if (!wait_block(b + 1)) { ok = false; break; }
                     qk(b + 1, n0, n1);
                 }
-                // mask keys past the prefix, running max / sum per row
-                const int kleft = P - b * 16;
+                // running max / sum per row on the raw scores (the scale log2(e)/sqrt(hd) is positive and is
+                // folded into the exponent); keys past the prefix are masked, which only the last block needs
                 float v[8] = {s0[0], s0[1], s0[2], s0[3], s1[0], s1[1], s1[2], s1[3]};
+                if (b == nblk - 1) {
+                    const int kleft = P - b * 16;
 #pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    const int key = (e >> 2) * 8 + 2 * t + (e & 1);
-                    v[e] = key < kleft ? v[e] * sc : -INFINITY;
+                    for (int e = 0; e < 8; ++e) {
+                        const int key = (e >> 2) * 8 + 2 * t + (e & 1);
+                        if (key >= kleft) v[e] = -INFINITY;
+                    }
                 }
                 float mx0 = fmaxf(fmaxf(v[0], v[1]), fmaxf(v[4], v[5]));
                 float mx1 = fmaxf(fmaxf(v[2], v[3]), fmaxf(v[6], v[7]));
                 mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1)); mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
                 mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1)); mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
                 const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
-                const float al0 = ex2(m0 - mn0), al1 = ex2(m1 - mn1);
                 const bool rescale = __any_sync(0xffffffffu, (mn0 != m0) || (mn1 != m1));   // warp-uniform
+                float al0 = 1.f, al1 = 1.f;
+                if (rescale) { al0 = ex2((m0 - mn0) * sc); al1 = ex2((m1 - mn1) * sc); }
                 m0 = mn0; m1 = mn1;
+                const float ms0 = -mn0 * sc, ms1 = -mn1 * sc;
                 float p[8];
-                p[0] = ex2(v[0] - mn0); p[1] = ex2(v[1] - mn0); p[4] = ex2(v[4] - mn0); p[5] = ex2(v[5] - mn0);
-                p[2] = ex2(v[2] - mn1); p[3] = ex2(v[3] - mn1); p[6] = ex2(v[6] - mn1); p[7] = ex2(v[7] - mn1);
+                p[0] = ex2(fmaf(v[0], sc, ms0)); p[1] = ex2(fmaf(v[1], sc, ms0)); p[4] = ex2(fmaf(v[4], sc, ms0)); p[5] = ex2(fmaf(v[5], sc, ms0));
+                p[2] = ex2(fmaf(v[2], sc, ms1)); p[3] = ex2(fmaf(v[3], sc, ms1)); p[6] = ex2(fmaf(v[6], sc, ms1)); p[7] = ex2(fmaf(v[7], sc, ms1));
                 l0 = l0 * al0 + ((p[0] + p[1]) + (p[4] + p[5]));
                 l1 = l1 * al1 + ((p[2] + p[3]) + (p[6] + p[7]));
                 uint32_t pf[4];
