@@ -69,6 +69,7 @@ struct Slot {
     size_t timed_used = 0;
     // groups queued in this slot and not yet launched
     std::vector<EnvMeta> pending;
+    std::vector<TensorMap128> pending_maps;   // TMA descriptor of each pending environment's planes (encoded at submit)
     std::vector<HostCopy> copies_out;
     cudaStream_t stream = nullptr;
     int grid = 0, groups_pending = 0;
@@ -468,13 +469,18 @@ ebrl_status_t flush_slot(ebrl_actgen *h, Slot &s)
     std::vector<int32_t> n_active(c.K_steps, 0);
     std::vector<double> sum_P(c.K_steps, 0.0);
     int S = 0;
+    std::vector<TensorMap128> maps_packed;
+    const bool with_maps = h->use_attn_mma && !(c.flags & EBRL_FLAG_TEST_PULL);
+    if (with_maps) maps_packed.resize(n);
     for (int j = 0; j < n; ++j) {
         const EnvMeta &m = s.pending[order[j]];
         s.meta_h[j] = m;
+        if (with_maps) maps_packed[j] = s.pending_maps[order[j]];
         S = std::max(S, (int)m.nsteps);
         for (int t = 0; t < m.nsteps; ++t) { n_active[t] += 1; sum_P[t] += m.P; }
     }
     s.pending.clear();
+    s.pending_maps.clear();
     // SM partition: the batch runs on the partition's stream, fenced against the caller's stream by events
     cudaStream_t user = cs;
     GreenPartition *gp = nullptr;
@@ -505,9 +511,8 @@ ebrl_status_t flush_slot(ebrl_actgen *h, Slot &s)
     CK(cudaMemcpyAsync(s.meta_d, s.meta_h, sizeof(EnvMeta) * (size_t)n, cudaMemcpyHostToDevice, cs));
     if (h->use_attn_mma && !(c.flags & EBRL_FLAG_TEST_PULL)) {
         // one TMA descriptor per environment: its planes as a [kv_layers * 2 * P][d] matrix
-        for (int j = 0; j < n; ++j)
-            if (attn_mma_make_map(&s.maps_h[j], s.meta_h[j].kv, (uint64_t)c.kv_layers * 2 * s.meta_h[j].P, c.d, c.n_heads, h->hd))
-                return fail(h, EBRL_ERR_CUDA, "cuTensorMapEncodeTiled failed for the prefix planes of a batch entry");
+        // (encoded when the group was submitted, so that the host work overlaps the previous batch)
+        for (int j = 0; j < n; ++j) s.maps_h[j] = maps_packed[j];
         CK(cudaMemcpyAsync(s.maps_d + 1, s.maps_h, sizeof(TensorMap128) * (size_t)n, cudaMemcpyHostToDevice, cs));
     }
     cudaError_t e = enqueue_batch(h, s, S, n_active.data(), sum_P.data(), s.grid, cs);
@@ -615,6 +620,16 @@ ebrl_status_t submit_impl(ebrl_actgen *h, int32_t n, const int64_t *env_ids, con
         for (int i = 0; i < n; ++i) kv_dev[i] = prefix_kv[i];
     }
 
+    // descriptors of the group's planes first: a failure must leave nothing of the group queued
+    std::vector<TensorMap128> group_maps;
+    if (h->use_attn_mma && !pull) {
+        group_maps.resize(n);
+        for (int i = 0; i < n; ++i) {
+            const int P = (ext && ext->prefix_len) ? ext->prefix_len[i] : c.max_prefix_len;
+            if (attn_mma_make_map(&group_maps[i], kv_dev[i], (uint64_t)c.kv_layers * 2 * P, c.d, c.n_heads, h->hd))
+                return fail(h, EBRL_ERR_CUDA, "cuTensorMapEncodeTiled failed for the prefix planes of environment %lld", (long long)env_ids[i]);
+        }
+    }
     uint64_t env_steps = 0;
     for (int i = 0; i < n; ++i) {
         EnvMeta m{};
@@ -627,6 +642,7 @@ ebrl_status_t submit_impl(ebrl_actgen *h, int32_t n, const int64_t *env_ids, con
         m.noise = noise_d + (size_t)i * chunk;
         m.out = out_d + (size_t)i * chunk;
         s.pending.push_back(m);
+        if (!group_maps.empty()) s.pending_maps.push_back(group_maps[i]);
         env_steps += (uint64_t)ns;
         s.ids.push_back(env_ids[i]);
         h->busy_ids.insert(env_ids[i]);
