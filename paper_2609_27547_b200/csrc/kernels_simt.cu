@@ -47,7 +47,7 @@ template <> __device__ __forceinline__ void store4<__nv_bfloat16>(__nv_bfloat16 
     *reinterpret_cast<uint2 *>(p) = make_uint2(*reinterpret_cast<uint32_t *>(&lo), *reinterpret_cast<uint32_t *>(&hi));
 }
 
-template <typename T>
+template <typename T, int AMAX>
 __global__ void __launch_bounds__(1024) embed_kernel(EmbedArgs a)
 {
     extern __shared__ float wT[];   // [A][d]
@@ -55,104 +55,129 @@ __global__ void __launch_bounds__(1024) embed_kernel(EmbedArgs a)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const T *w_in = (const T *)a.w_in;
     T *xg = (T *)a.xg;
-    for (int e = threadIdx.x; e < a.d * a.A; e += blockDim.x) {
-        const int c = e / a.A, j = e - c * a.A;
-        wT[j * a.d + c] = ldf(w_in + e);
-    }
+    for (int c = threadIdx.x; c < a.d; c += blockDim.x)
+        for (int j = 0; j < a.A; ++j) wT[j * a.d + c] = ldf(w_in + (size_t)c * a.A + j);
     __syncthreads();
-    for (int row = blockIdx.x * 32 + warp; row < rows; row += gridDim.x * 32) {
-        const int env = row / a.H, h = row - env * a.H;
-        const EnvMeta m = a.meta[env];
-        const int k = m.k0 + a.s;
-        const float *av = (a.s == 0) ? m.noise + (size_t)h * a.A : a.a_state + (size_t)row * a.A;
-        const float mine = lane < a.A ? av[lane] : 0.f;
+    // two rows per warp pass: each staged weight is used for both
+    for (int row0 = (blockIdx.x * 32 + warp) * 2; row0 < rows; row0 += gridDim.x * 64) {
+        float aj[2][AMAX];
+        int kk[2];
+        const int nr = min(2, rows - row0);
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            const int row = row0 + (r < nr ? r : 0);
+            const int env = row / a.H, h = row - env * a.H;
+            const EnvMeta m = a.meta[env];
+            kk[r] = m.k0 + a.s;
+            const float *av = (a.s == 0) ? m.noise + (size_t)h * a.A : a.a_state + (size_t)row * a.A;
+            const float mine = lane < a.A ? av[lane] : 0.f;
+#pragma unroll
+            for (int j = 0; j < AMAX; ++j) aj[r][j] = __shfl_sync(0xffffffffu, mine, j);
+        }
         for (int seg = 0; seg < nseg; ++seg) {
             const int c = seg * SSQ_W + 4 * lane;
-            float acc[4] = {0.f, 0.f, 0.f, 0.f};
-            for (int j = 0; j < a.A; ++j) {
-                const float aj = __shfl_sync(0xffffffffu, mine, j);
-                const float4 w = *reinterpret_cast<const float4 *>(wT + j * a.d + c);
-                acc[0] = fmaf(w.x, aj, acc[0]); acc[1] = fmaf(w.y, aj, acc[1]);
-                acc[2] = fmaf(w.z, aj, acc[2]); acc[3] = fmaf(w.w, aj, acc[3]);
+            float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+#pragma unroll
+            for (int j = 0; j < AMAX; ++j) {
+                if (j < a.A) {
+                    const float4 w = *reinterpret_cast<const float4 *>(wT + j * a.d + c);
+#pragma unroll
+                    for (int r = 0; r < 2; ++r) {
+                        acc[r][0] = fmaf(w.x, aj[r][j], acc[r][0]); acc[r][1] = fmaf(w.y, aj[r][j], acc[r][1]);
+                        acc[r][2] = fmaf(w.z, aj[r][j], acc[r][2]); acc[r][3] = fmaf(w.w, aj[r][j], acc[r][3]);
+                    }
+                }
             }
-            const float4 te = *reinterpret_cast<const float4 *>(a.temb + (size_t)k * a.d + c);
             const float4 gn = *reinterpret_cast<const float4 *>(a.gain + c);
-            acc[0] += te.x; acc[1] += te.y; acc[2] += te.z; acc[3] += te.w;
-            *reinterpret_cast<float4 *>(a.x + (size_t)row * a.d + c) = make_float4(acc[0], acc[1], acc[2], acc[3]);
-            store4<T>(xg + (size_t)row * a.d + c, acc[0] * gn.x, acc[1] * gn.y, acc[2] * gn.z, acc[3] * gn.w);
-            float ss = acc[0] * acc[0];
-            ss = fmaf(acc[1], acc[1], ss); ss = fmaf(acc[2], acc[2], ss); ss = fmaf(acc[3], acc[3], ss);
-            ss = warp_sum(ss);
-            if (lane == 0) a.ssq[(size_t)row * nseg + seg] = ss;
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                if (r < nr) {
+                    const int row = row0 + r;
+                    const float4 te = *reinterpret_cast<const float4 *>(a.temb + (size_t)kk[r] * a.d + c);
+                    const float v0 = acc[r][0] + te.x, v1 = acc[r][1] + te.y, v2 = acc[r][2] + te.z, v3 = acc[r][3] + te.w;
+                    *reinterpret_cast<float4 *>(a.x + (size_t)row * a.d + c) = make_float4(v0, v1, v2, v3);
+                    store4<T>(xg + (size_t)row * a.d + c, v0 * gn.x, v1 * gn.y, v2 * gn.z, v3 * gn.w);
+                    float ss = v0 * v0;
+                    ss = fmaf(v1, v1, ss); ss = fmaf(v2, v2, ss); ss = fmaf(v3, v3, ss);
+                    ss = warp_sum(ss);
+                    if (lane == 0) a.ssq[(size_t)row * nseg + seg] = ss;
+                }
+            }
         }
     }
 }
 
 // ---------------------------------------------------------------------------------------
-// v = W_out RMSNorm(x; g_final) + b_out;  a += v / K.  One warp per row.
+// v = W_out RMSNorm(x; g_final) + b_out;  a += v / K.  W_out is staged once per CTA in shared
+// memory as fp32 [A][d]; one warp handles two rows per pass (each staged weight serves both),
+// each lane four consecutive columns of a 128-column segment at a time.
 // ---------------------------------------------------------------------------------------
-template <typename T> __device__ __forceinline__ void load8(const T *p, float (&v)[8]);
-template <> __device__ __forceinline__ void load8<float>(const float *p, float (&v)[8])
-{
-    const float4 a = *reinterpret_cast<const float4 *>(p), b = *reinterpret_cast<const float4 *>(p + 4);
-    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
-}
-template <> __device__ __forceinline__ void load8<__nv_bfloat16>(const __nv_bfloat16 *p, float (&v)[8])
-{
-    const uint4 u = *reinterpret_cast<const uint4 *>(p);
-    const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&u);
-#pragma unroll
-    for (int i = 0; i < 4; ++i) { v[2 * i] = __bfloat162float(h[i].x); v[2 * i + 1] = __bfloat162float(h[i].y); }
-}
-
 constexpr int HEAD_WARPS = 16;
 
 template <typename T, int AMAX>
 __global__ void __launch_bounds__(HEAD_WARPS * 32) head_kernel(HeadArgs a)
 {
+    extern __shared__ float wO[];   // [A][d]
     const int rows = a.n_envs * a.H;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const T *w_out = (const T *)a.w_out;
-    for (int row = blockIdx.x * HEAD_WARPS + warp; row < rows; row += gridDim.x * HEAD_WARPS) {
-        const int env = row / a.H, h = row - env * a.H;
-        const EnvMeta m = a.meta[env];
-        const float *xr = a.x + (size_t)row * a.d;
-        float acc[AMAX];
+    if (!a.pull) {
+        for (int e = threadIdx.x; e < a.A * a.d; e += blockDim.x) wO[e] = ldf(w_out + e);
+    }
+    __syncthreads();
+    for (int row0 = (blockIdx.x * HEAD_WARPS + warp) * 2; row0 < rows; row0 += gridDim.x * HEAD_WARPS * 2) {
+        const int nr = min(2, rows - row0);
+        float acc[2][AMAX];
 #pragma unroll
-        for (int j = 0; j < AMAX; ++j) acc[j] = 0.f;
-        float ss = 0.f;
+        for (int r = 0; r < 2; ++r)
+#pragma unroll
+            for (int j = 0; j < AMAX; ++j) acc[r][j] = 0.f;
+        float ss[2] = {0.f, 0.f};
         if (!a.pull) {
-            // each lane takes 8 consecutive columns per pass (d is a multiple of 128)
-            for (int c = lane * 8; c < a.d; c += 256) {
-                float xv[8], gv[8], t[8];
-                load8<float>(xr + c, xv);
-                load8<float>(a.gain + c, gv);
+            for (int c = lane * 4; c < a.d; c += 128) {
+                const float4 gv = *reinterpret_cast<const float4 *>(a.gain + c);
+                float t[2][4];
 #pragma unroll
-                for (int i = 0; i < 8; ++i) { ss = fmaf(xv[i], xv[i], ss); t[i] = xv[i] * gv[i]; }
+                for (int r = 0; r < 2; ++r) {
+                    const float4 xv = *reinterpret_cast<const float4 *>(a.x + (size_t)(row0 + (r < nr ? r : 0)) * a.d + c);
+                    ss[r] = fmaf(xv.x, xv.x, ss[r]); ss[r] = fmaf(xv.y, xv.y, ss[r]);
+                    ss[r] = fmaf(xv.z, xv.z, ss[r]); ss[r] = fmaf(xv.w, xv.w, ss[r]);
+                    t[r][0] = xv.x * gv.x; t[r][1] = xv.y * gv.y; t[r][2] = xv.z * gv.z; t[r][3] = xv.w * gv.w;
+                }
 #pragma unroll
                 for (int j = 0; j < AMAX; ++j) {
                     if (j < a.A) {
-                        float wv[8];
-                        load8<T>(w_out + (size_t)j * a.d + c, wv);
+                        const float4 w = *reinterpret_cast<const float4 *>(wO + j * a.d + c);
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) acc[j] = fmaf(t[i], wv[i], acc[j]);
+                        for (int r = 0; r < 2; ++r) {
+                            acc[r][j] = fmaf(t[r][0], w.x, acc[r][j]); acc[r][j] = fmaf(t[r][1], w.y, acc[r][j]);
+                            acc[r][j] = fmaf(t[r][2], w.z, acc[r][j]); acc[r][j] = fmaf(t[r][3], w.w, acc[r][j]);
+                        }
                     }
                 }
             }
-            ss = warp_sum(ss);
         }
-        const float inv = 1.0f / sqrtf(ss / (float)a.d + a.eps);
-        const float *a_old = (a.s == 0) ? m.noise + (size_t)h * a.A : a.a_state + (size_t)row * a.A;
 #pragma unroll
-        for (int j = 0; j < AMAX; ++j) {
-            if (j < a.A) {
-                const float dot = warp_sum(acc[j]);
-                if (lane == 0) {
-                    const float ao = a_old[j];
-                    const float v = a.pull ? (a.b_out[j] - ao) : (dot * inv + a.b_out[j]);
-                    const float an = ao + v / (float)a.K;
-                    a.a_state[(size_t)row * a.A + j] = an;
-                    if (a.s == m.nsteps - 1) m.out[(size_t)h * a.A + j] = an;
+        for (int r = 0; r < 2; ++r) {
+            if (r < nr) {   // warp-uniform
+                const int row = row0 + r;
+                const int env = row / a.H, h = row - env * a.H;
+                const EnvMeta m = a.meta[env];
+                const float ssr = a.pull ? 0.f : warp_sum(ss[r]);
+                const float inv = 1.0f / sqrtf(ssr / (float)a.d + a.eps);
+                const float *a_old = (a.s == 0) ? m.noise + (size_t)h * a.A : a.a_state + (size_t)row * a.A;
+#pragma unroll
+                for (int j = 0; j < AMAX; ++j) {
+                    if (j < a.A) {
+                        const float dot = warp_sum(acc[r][j]);
+                        if (lane == 0) {
+                            const float ao = a_old[j];
+                            const float v = a.pull ? (a.b_out[j] - ao) : (dot * inv + a.b_out[j]);
+                            const float an = ao + v / (float)a.K;
+                            a.a_state[(size_t)row * a.A + j] = an;
+                            if (a.s == m.nsteps - 1) m.out[(size_t)h * a.A + j] = an;
+                        }
+                    }
                 }
             }
         }
@@ -394,43 +419,58 @@ __global__ void __launch_bounds__(512) attn_simt_kernel(AttnArgs a)
 // ---------------------------------------------------------------------------------------
 // launchers
 // ---------------------------------------------------------------------------------------
-cudaError_t launch_embed(const EmbedArgs &a, int bf16, int grid, cudaStream_t st)
+template <typename T, int AMAX>
+static cudaError_t embed_launch(const EmbedArgs &a, int g, size_t smem, cudaStream_t st)
 {
-    const int rows = a.n_envs * a.H;
-    if (rows == 0) return cudaSuccess;
-    const int need = (rows + 31) / 32;
-    const int g = need < grid ? need : grid;
-    const size_t smem = (size_t)a.d * a.A * sizeof(float);
-    cudaError_t e;
-    if (bf16) {
-        e = cudaFuncSetAttribute(embed_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        embed_kernel<__nv_bfloat16><<<g, 1024, smem, st>>>(a);
-    } else {
-        e = cudaFuncSetAttribute(embed_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        embed_kernel<float><<<g, 1024, smem, st>>>(a);
-    }
+    cudaError_t e = cudaFuncSetAttribute(embed_kernel<T, AMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    embed_kernel<T, AMAX><<<g, 1024, smem, st>>>(a);
     return cudaGetLastError();
 }
 
 template <typename T>
-static void head_dispatch(const HeadArgs &a, int g, cudaStream_t st)
+static cudaError_t embed_dispatch(const EmbedArgs &a, int g, size_t smem, cudaStream_t st)
 {
-    if (a.A <= 8) head_kernel<T, 8><<<g, HEAD_WARPS * 32, 0, st>>>(a);
-    else if (a.A <= 16) head_kernel<T, 16><<<g, HEAD_WARPS * 32, 0, st>>>(a);
-    else head_kernel<T, 32><<<g, HEAD_WARPS * 32, 0, st>>>(a);
+    if (a.A <= 8) return embed_launch<T, 8>(a, g, smem, st);
+    if (a.A <= 16) return embed_launch<T, 16>(a, g, smem, st);
+    return embed_launch<T, 32>(a, g, smem, st);
+}
+
+cudaError_t launch_embed(const EmbedArgs &a, int bf16, int grid, cudaStream_t st)
+{
+    const int rows = a.n_envs * a.H;
+    if (rows == 0) return cudaSuccess;
+    const int need = (rows + 63) / 64;
+    const int g = need < grid ? need : grid;
+    const size_t smem = (size_t)a.d * a.A * sizeof(float);
+    return bf16 ? embed_dispatch<__nv_bfloat16>(a, g, smem, st) : embed_dispatch<float>(a, g, smem, st);
+}
+
+template <typename T, int AMAX>
+static cudaError_t head_launch(const HeadArgs &a, int g, size_t smem, cudaStream_t st)
+{
+    cudaError_t e = cudaFuncSetAttribute(head_kernel<T, AMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    head_kernel<T, AMAX><<<g, HEAD_WARPS * 32, smem, st>>>(a);
+    return cudaGetLastError();
+}
+
+template <typename T>
+static cudaError_t head_dispatch(const HeadArgs &a, int g, size_t smem, cudaStream_t st)
+{
+    if (a.A <= 8) return head_launch<T, 8>(a, g, smem, st);
+    if (a.A <= 16) return head_launch<T, 16>(a, g, smem, st);
+    return head_launch<T, 32>(a, g, smem, st);
 }
 
 cudaError_t launch_head(const HeadArgs &a, int bf16, int grid, cudaStream_t st)
 {
     const int rows = a.n_envs * a.H;
     if (rows == 0) return cudaSuccess;
-    const int need = (rows + HEAD_WARPS - 1) / HEAD_WARPS;
+    const int need = (rows + 2 * HEAD_WARPS - 1) / (2 * HEAD_WARPS);
     const int g = need < grid ? need : grid;
-    if (bf16) head_dispatch<__nv_bfloat16>(a, g, st);
-    else head_dispatch<float>(a, g, st);
-    return cudaGetLastError();
+    const size_t smem = (size_t)a.d * a.A * sizeof(float);
+    return bf16 ? head_dispatch<__nv_bfloat16>(a, g, smem, st) : head_dispatch<float>(a, g, smem, st);
 }
 
 template <typename T>
