@@ -69,6 +69,9 @@ def parse_args():
     ap.add_argument("--green-ctx", action="store_true", help="run inside an SM partition (green context) of the quota")
     ap.add_argument("--pgen-sweep", action="store_true",
                     help="emit the generation profile P_gen(s_g, B_g): chunks/s on a grid of SM quotas and group sizes")
+    ap.add_argument("--rollout-sim", action="store_true",
+                    help="event-driven rollout with a synthetic simulator-latency model: chunk latency avg/P50/P99 under "
+                         "group-level batching and under step-level continuous batching")
     ap.add_argument("--min-warmup", type=int, default=3, help="lower bound on warm-up steps (profiling captures use 1)")
     ap.add_argument("--inflight", type=int, default=8, help="groups queued before a batch is launched")
     return ap.parse_args()
@@ -425,6 +428,21 @@ def main():
     args = parse_args()
     if args.pgen_sweep:
         return run_pgen_sweep(args)
+    if args.rollout_sim:
+        import torch
+        from paper_2609_27547_b200 import rollout_sim as R
+        from paper_2609_27547_b200 import synth
+        torch.cuda.set_device(0)
+        w = synth.WORKLOADS[args.config]
+        wt = synth.make_weights(w, args.seed or synth.DEFAULT_SEED, device="cuda")
+        n = args.envs or 128
+        quota = w.quota if args.quota < 0 else args.quota
+        out = [R.run(w, wt, n, max(1, args.steps), pol, quota=quota, max_group=64, sim_steps_per_chunk=w.H).summary()
+               for pol in ("chunk", "step")]
+        print(json.dumps({"rollout_sim": {"workload": "configs[%d] %s" % (args.config, w.name), "envs": n, "chunks_per_env": max(1, args.steps),
+                                          "sm_quota": quota or N_SMS, "simulator": "log-normal step time, mean 40 ms, P99 60 ms, H steps per chunk",
+                                          "policies": out}}))
+        return
     if args.impl == "reference":
         run_reference(args)
     else:

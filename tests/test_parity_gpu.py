@@ -337,3 +337,40 @@ def test_weight_publication_switches_versions_between_batches(dtype):
     got = stack(r.run([ids]), ids)
     assert np.array_equal(got, refs["A"]) and r.gen.stats()["weights_version"] == 3
     r.close()
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_rollout_policies_deliver_identical_chunks(dtype):
+    """Group-level batching and step-level continuous batching (every Euler step its own submit,
+    environments joining mid-chunk) serve the same seeded rollout: every (environment, visit) gets
+    the same bits under both policies, and those bits are the oracle's within tolerance."""
+    from paper_2609_27547_b200 import rollout_sim as R
+    from helpers import oracle_cfg, oracle_weights
+    import oracle
+    w = synth.scaled(synth.WORKLOADS[0], B=20, dtype=dtype, P=(16, 48), K=4)
+    wt = synth.make_weights(w, SEED, random_gains=True)
+    a = R.run(w, wt, 20, 3, "chunk", max_group=8, keep_outputs=True)
+    b = R.run(w, wt, 20, 3, "step", max_group=8, keep_outputs=True)
+    assert a.chunks == b.chunks == 60 and set(a.outputs) == set(b.outputs)
+    for k in a.outputs:
+        assert torch.equal(a.outputs[k], b.outputs[k]), k
+    assert b.submits > a.submits                      # the step policy re-batches every Euler step
+    for r in (a, b):
+        s = r.summary()
+        assert 0 < s["latency_ms"]["p50"] <= s["latency_ms"]["p99"] and 0 < s["generation_busy_frac"] <= 1.0
+    # against the oracle for a few (env, visit) pairs
+    keys = [(0, 0), (7, 1), (19, 2)]
+    envs = [synth.make_env(w, e, SEED) for e, _ in keys]
+    noise = np.stack([np32(synth.normal(SEED, "noise_visit%d" % v, e, (w.H, w.A))) for e, v in keys])
+    ref = oracle.actgen(oracle_cfg(w), oracle_weights(wt), [np32(e.kv) for e in envs], noise)
+    got = np.stack([a.outputs[k].cpu().numpy() for k in keys])
+    assert chunk_rel_err(got, ref) <= TOL[dtype]
+
+
+def test_simulator_latency_model_moments():
+    """The synthetic simulator step time: log-normal with mean 40 ms and 99th percentile 60 ms."""
+    from paper_2609_27547_b200 import rollout_sim as R
+    z = synth.normal(SEED, "sim_latency", 0, (200000,)).double()
+    t = torch.exp(R.SIM_MU + R.SIM_SIGMA * z)
+    assert abs(float(t.mean()) - 40.0) < 0.2
+    assert abs(float(torch.quantile(t, 0.99)) - 60.0) < 0.8
