@@ -374,3 +374,19 @@ def test_simulator_latency_model_moments():
     t = torch.exp(R.SIM_MU + R.SIM_SIGMA * z)
     assert abs(float(t.mean()) - 40.0) < 0.2
     assert abs(float(torch.quantile(t, 0.99)) - 60.0) < 0.8
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_chunk_of_five_actions(dtype):
+    """The paper's other chunk length ("next 5 or 8 actions"): H = 5, which is neither a power of two nor a
+    divisor of the 128-row tile, so environments straddle tile and warp boundaries."""
+    w = synth.scaled(synth.WORKLOADS[0], B=53, dtype=dtype, H=5, P=(30, 90), K=3, mixed_steps=True)
+    wt, envs = _setup(w)
+    ref = oracle_run(w, wt, envs)
+    r = Runner(w, wt, envs, max_inflight_groups=3)
+    ids = list(range(w.B))
+    got = stack(r.run([ids[:20], ids[20:21], ids[21:]], quota=37), ids)
+    alone = stack(r.run([[e] for e in ids[:5]]), ids[:5])
+    r.close()
+    assert chunk_rel_err(got, ref) <= TOL[dtype]
+    assert np.array_equal(alone, got[:5])
