@@ -28,16 +28,18 @@ __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sy
 // keeps the GELU epilogue of the MLP-up GEMM shorter than its tile's mainloop.
 __device__ __forceinline__ float gelu_erf(float z)
 {
-    const float u = z * 0.70710678118654752440f, ax = fabsf(u);
+    // Phi(z) = 0.5 (1 + erf(z / sqrt 2)):  q = 0.5 (a1 t + ... + a5 t^5) exp(-z^2 / 2),  Phi = z >= 0 ? 1 - q : q
+    const float az = fabsf(z);
+    const float a1 = az * 0.84932180028801904f;           // |z| sqrt(log2(e) / 2): exp(-z^2/2) = 2^(-a1^2)
     float t, e;
-    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(fmaf(0.3275911f, ax, 1.0f)));
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(ax * ax * -1.4426950408889634f));
-    float p = fmaf(1.061405429f, t, -1.453152027f);
-    p = fmaf(p, t, 1.421413741f);
-    p = fmaf(p, t, -0.284496736f);
-    p = fmaf(p, t, 0.254829592f);
-    const float erf_abs = fmaf(-p * t, e, 1.0f);
-    return 0.5f * z * (1.0f + copysignf(erf_abs, u));
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(fmaf(az, 0.23164189f, 1.0f)));   // p / sqrt 2
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(-a1 * a1));
+    float p = fmaf(0.5307027145f, t, -0.7265760135f);     // the five coefficients, halved
+    p = fmaf(p, t, 0.7107068705f);
+    p = fmaf(p, t, -0.142248368f);
+    p = fmaf(p, t, 0.127414796f);
+    const float q = p * t * e;
+    return z * (z >= 0.f ? 1.0f - q : q);
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 {
