@@ -147,7 +147,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_mma_kernel(AttnArgs a, int hp
             }
             for (int j0 = 0; j0 < P; j0 += KB) {
                 if (use_la) la_step();
-                if (!__all_sync(0xffffffffu, mbar_wait(empty(stage), phase ^ 1u, limit_ns, abort_flag))) { ok = false; break; }
+                if (!__all_sync(0xffffffffu, mbar_wait_relaxed(empty(stage), phase ^ 1u, limit_ns, abort_flag))) { ok = false; break; }
                 if (lane == 0) {
                     mbar_expect_tx(full(stage), (uint32_t)(2 * stage_bytes));
                     tma_load_3d(sK + stage * stage_bytes, tm, full(stage), 0, krow + j0, kgrp);

@@ -114,7 +114,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
             const int m0 = (tile / ntn) * BM, n0 = (tile % ntn) * BN;
             for (int kb = 0; kb < nkb; ++kb) {
-                if (!__all_sync(0xffffffffu, mbar_wait(empty(stage), phase ^ 1u, limit_ns, abort_flag))) { ok = false; break; }
+                if (!__all_sync(0xffffffffu, mbar_wait_relaxed(empty(stage), phase ^ 1u, limit_ns, abort_flag))) { ok = false; break; }
                 if (lane == 0) {
                     mbar_expect_tx(full(stage), A_BYTES + B_BYTES);
                     tma_load_2d(sA + stage * A_BYTES, &tmA, full(stage), kb * BK, m0);
@@ -164,7 +164,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
             const int m0 = (tile / ntn) * BM, n0 = (tile % ntn) * BN + half * 128;
             if (!epilogue_rows<EPI, 128>(g, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + half * 128), m0 + q * 32, n0, stg,
-                                            [&] { return __all_sync(0xffffffffu, mbar_wait(tfull(buf), acc_phase, limit_ns, abort_flag)) != 0; })) {
+                                            [&] { return __all_sync(0xffffffffu, mbar_wait_relaxed(tfull(buf), acc_phase, limit_ns, abort_flag)) != 0; })) {
                 ok = false;
                 break;
             }

@@ -132,7 +132,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         for (int tile = pair; tile < ntiles && ok; tile += npairs) {
             const int m0 = (tile / ntn) * (2 * BM) + (int)rank * BM, n0 = (tile % ntn) * BN + (int)rank * BNH;
             for (int kb = 0; kb < nkb; ++kb) {
-                if (!__all_sync(0xffffffffu, mbar_wait(empty(stage), phase ^ 1u, limit_ns, abort_flag))) { ok = false; break; }
+                if (!__all_sync(0xffffffffu, mbar_wait_relaxed(empty(stage), phase ^ 1u, limit_ns, abort_flag))) { ok = false; break; }
                 if (lane == 0) {
                     if (rank == 0) mbar_expect_tx(full(stage), 2 * (A_BYTES + B_BYTES));
                     const uint32_t lead_full = mapa(full(stage), 0);
@@ -184,7 +184,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
             const int m0 = (tile / ntn) * (2 * BM) + (int)rank * BM, n0 = (tile % ntn) * BN + half * (BN / 2);
             if (!epilogue_rows<EPI, BN / 2>(g, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + half * (BN / 2)), m0 + q * 32, n0, stg,
-                                            [&] { return __all_sync(0xffffffffu, mbar_wait(tfull(buf), acc_phase, limit_ns, abort_flag)) != 0; })) {
+                                            [&] { return __all_sync(0xffffffffu, mbar_wait_relaxed(tfull(buf), acc_phase, limit_ns, abort_flag)) != 0; })) {
                 ok = false;
                 break;
             }

@@ -44,6 +44,23 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigne
         if (gtimer() - t0 > limit_ns) return false;
     }
 }
+// The same for waits that are expected to last (a consumer waiting for the next tile, a producer
+// waiting for a free stage): polls are spaced by a short sleep so that idle warps do not burn issue
+// slots and power beside the warps that do the work.
+__device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, unsigned long long limit_ns, volatile int *abort_flag)
+{
+    for (int i = 0; i < 4; ++i)
+        if (mbar_try(bar, parity)) return true;
+    const unsigned long long t0 = gtimer();
+    for (;;) {
+        for (int i = 0; i < 64; ++i) {
+            if (mbar_try(bar, parity)) return true;
+            __nanosleep(64);
+        }
+        if (*abort_flag) return false;
+        if (gtimer() - t0 > limit_ns) return false;
+    }
+}
 // 1-D bulk copy global -> shared (both 16-byte aligned, size a multiple of 16), completing on an mbarrier.
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
 {
