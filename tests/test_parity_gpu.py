@@ -390,3 +390,50 @@ def test_chunk_of_five_actions(dtype):
     r.close()
     assert chunk_rel_err(got, ref) <= TOL[dtype]
     assert np.array_equal(alone, got[:5])
+
+
+def test_queue_semantics_flush_streams_and_timing():
+    """Queue depth 1 launches at submit (the result is ready after a stream synchronisation, no library
+    sync needed); a deeper queue holds groups until flush / a stream or quota change / sync; the
+    per-class timing adds up launches and device time."""
+    w = synth.scaled(synth.WORKLOADS[0], B=9, P=(20, 40))
+    wt, envs = _setup(w)
+    ids = list(range(w.B))
+    r1 = Runner(w, wt, envs, max_inflight_groups=1)
+    base = stack(r1.run([ids]), ids)
+    noise = torch.stack([r1.noise[e] for e in ids])
+    kv = [r1.kv[e] for e in ids]
+    st = torch.cuda.Stream()
+    out = torch.zeros_like(noise)
+    r1.gen.submit([100 + e for e in ids], kv, noise, out, stream=st)
+    st.synchronize()                                   # depth 1: already launched on the caller's stream
+    assert np.array_equal(out.cpu().numpy(), base)
+    r1.gen.sync()
+    r1.close()
+
+    r = Runner(w, wt, envs, max_inflight_groups=4, flags=B.FLAG_TIMING)
+    out_a, out_b, out_c = torch.zeros_like(noise), torch.zeros_like(noise), torch.zeros_like(noise)
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    r.gen.submit(ids[:4], kv[:4], noise[:4], out_a[:4], stream=s1)          # queued
+    s1.synchronize()
+    assert float(out_a.abs().sum()) == 0.0 and r.gen.stats()["kernel_launches"] == 0
+    r.gen.submit(ids[4:], kv[4:], noise[4:], out_a[4:], stream=s1)          # queued with the first
+    r.gen.flush()                                                            # launches both as one batch
+    s1.synchronize()
+    assert np.array_equal(out_a.cpu().numpy(), base)
+    n1 = r.gen.stats()["kernel_launches"]
+    assert n1 == w.K * (w.L * 8 + 2)                                        # one batch, not two
+    r.gen.sync()                                                             # retire: the ids may be used again
+    r.gen.submit(ids[:5], kv[:5], noise[:5], out_b[:5], stream=s1, sm_quota=37)
+    r.gen.submit(ids[5:], kv[5:], noise[5:], out_c[5:], stream=s2, sm_quota=37)   # other stream: closes the first batch
+    s1.synchronize()
+    assert np.array_equal(out_b[:5].cpu().numpy(), base[:5])
+    r.gen.sync()
+    assert np.array_equal(out_c[5:].cpu().numpy(), base[5:])
+    stt = r.gen.stats()
+    assert stt["kernel_launches"] == 3 * n1 and stt["groups"] == 4
+    cls = stt["classes"]
+    assert sum(c["launches"] for c in cls.values()) == stt["kernel_launches"]
+    assert cls["gemm"]["launches"] == 3 * w.K * w.L * 6 and cls["gemm"]["ms"] > 0 and cls["gemm"]["flops"] > 0
+    assert cls["cross_attn"]["bytes"] > 0 and cls["head"]["launches"] == 3 * w.K
+    r.close()
