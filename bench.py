@@ -73,7 +73,7 @@ def parse_args():
                     help="event-driven rollout with a synthetic simulator-latency model: chunk latency avg/P50/P99 under "
                          "group-level batching and under step-level continuous batching")
     ap.add_argument("--min-warmup", type=int, default=3, help="lower bound on warm-up steps (profiling captures use 1)")
-    ap.add_argument("--inflight", type=int, default=8, help="groups queued before a batch is launched")
+    ap.add_argument("--inflight", type=int, default=16, help="groups queued before a batch is launched")
     return ap.parse_args()
 
 

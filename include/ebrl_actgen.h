@@ -181,7 +181,11 @@ ebrl_status_t ebrl_actgen_submit(ebrl_actgen_t h, int32_t n_envs, const int64_t 
  * owned by the handle when the call is made -- on a copy stream of the handle, so that the
  * upload of one batch overlaps the kernels of the previous one -- the group runs with its batch
  * on `stream` once its uploads are done, and `out` is copied back after the batch on `stream`;
- * `out` is valid after ebrl_actgen_sync.  The host buffers must stay valid until then.  Needs prefix_len in ext, or every P_e = max_prefix_len. */
+ * `out` is valid after ebrl_actgen_sync.  The host buffers must stay valid until then.  Needs
+ * prefix_len in ext, or every P_e = max_prefix_len.
+ * Batches of host-staged groups ramp up: after create and after every sync the first batch
+ * closes at 1 group, the next at 2, then 4, ... up to max_inflight_groups, so that only the first
+ * group's upload is exposed and every later batch uploads behind the previous one's kernels. */
 ebrl_status_t ebrl_actgen_submit_host(ebrl_actgen_t h, int32_t n_envs, const int64_t *env_ids,
                                       const void *const *prefix_kv_host, const float *noise_host,
                                       float *out_host, int32_t sm_quota, void *stream,

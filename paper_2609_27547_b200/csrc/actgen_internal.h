@@ -122,6 +122,47 @@ struct GreenPartition {
 int green_partition_create(int device, int sm_quota, GreenPartition *out);
 void green_partition_destroy(GreenPartition *p);
 
+// Programmatic dependent launch: every kernel of a batch is launched with the attribute that lets
+// its CTAs start (and run their on-chip set-up) while the previous kernel's last CTAs are still
+// finishing; each kernel then calls pdl_wait() before it touches global memory of the batch, which
+// blocks until the previous kernel has completed and its writes are visible.  Dependencies are
+// unchanged; only the launch latency and the set-up move off the critical path.  The attribute is
+// used only for batches whose grid fills every SM their stream can reach: under a smaller SM quota
+// the early CTAs would park on SMs outside the quota (and measured slower).  pdl_set() states the
+// choice for the calling thread's next launches; EBRL_PDL=0 turns the attribute off altogether.
+void pdl_set(bool on);
+bool pdl_enabled();
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kern)(KArgs...), int grid, int block, size_t smem, cudaStream_t st, int cluster, Args &&...args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid, 1, 1);
+    cfg.blockDim = dim3((unsigned)block, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    int n = 0;
+    if (pdl_enabled()) {
+        attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n].val.programmaticStreamSerializationAllowed = 1;
+        ++n;
+    }
+    if (cluster > 1) {
+        attr[n].id = cudaLaunchAttributeClusterDimension;
+        attr[n].val.clusterDim.x = (unsigned)cluster;
+        attr[n].val.clusterDim.y = 1;
+        attr[n].val.clusterDim.z = 1;
+        ++n;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = (unsigned)n;
+    return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+#endif
+
 // Launchers (plain-ALU kernels).  bf16 != 0 selects bf16 activations/weights/planes.
 // grid = number of persistent CTAs (the SM quota).
 cudaError_t launch_embed(const EmbedArgs &a, int bf16, int grid, cudaStream_t st);

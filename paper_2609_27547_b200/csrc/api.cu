@@ -20,6 +20,17 @@
 
 using namespace ebrl;
 
+namespace ebrl {
+static thread_local bool t_pdl = false;
+void pdl_set(bool on) { t_pdl = on; }
+bool pdl_enabled()
+{
+    static int allowed = -1;
+    if (allowed < 0) { const char *e = getenv("EBRL_PDL"); allowed = (e && atoi(e) == 0) ? 0 : 1; }
+    return allowed != 0 && t_pdl;
+}
+}  // namespace ebrl
+
 namespace {
 
 struct LayerDev {
@@ -98,6 +109,8 @@ struct ebrl_actgen {
     float *temb = nullptr;
     std::vector<Slot> slots;
     size_t fill = 0;              // slot collecting groups for the next batch
+    size_t stage_hint = 0;        // plane staging a full batch has needed so far (bytes per slot)
+    int host_depth = 1;           // groups per batch of host-staged submits: doubles per batch, back to 1 at sync
     std::unordered_set<int64_t> busy_ids;
     std::mutex mu;
     std::string err;
@@ -507,6 +520,7 @@ ebrl_status_t flush_slot(ebrl_actgen *h, Slot &s)
         CK(cudaEventRecord(s.h2d_done, h->copy_stream));
         CK(cudaStreamWaitEvent(cs, s.h2d_done, 0));
         s.has_uploads = false;
+        h->host_depth = std::min(2 * h->host_depth, c.max_inflight_groups);
     }
     CK(cudaMemcpyAsync(s.meta_d, s.meta_h, sizeof(EnvMeta) * (size_t)n, cudaMemcpyHostToDevice, cs));
     if (h->use_attn_mma && !(c.flags & EBRL_FLAG_TEST_PULL)) {
@@ -515,7 +529,9 @@ ebrl_status_t flush_slot(ebrl_actgen *h, Slot &s)
         for (int j = 0; j < n; ++j) s.maps_h[j] = maps_packed[j];
         CK(cudaMemcpyAsync(s.maps_d + 1, s.maps_h, sizeof(TensorMap128) * (size_t)n, cudaMemcpyHostToDevice, cs));
     }
+    pdl_set(s.grid >= (gp ? gp->sm_count : h->n_sms));
     cudaError_t e = enqueue_batch(h, s, S, n_active.data(), sum_P.data(), s.grid, cs);
+    pdl_set(false);
     if (e != cudaSuccess) {
         h->sticky = EBRL_ERR_CUDA;
         return fail(h, EBRL_ERR_CUDA, "kernel launch failed: %s", cudaGetErrorString(e));
@@ -577,17 +593,22 @@ ebrl_status_t submit_impl(ebrl_actgen *h, int32_t n, const int64_t *env_ids, con
             off[i] = need;
             need += ((size_t)c.kv_layers * 2 * P * c.d * h->esz + 255) & ~(size_t)255;
         }
-        if (!pull && s.kv_stage_bytes < need) {
-            if (s.stage_used != 0) {   // staging already referenced by queued groups: close the batch first
-                if ((st = flush_slot(h, s)) != EBRL_OK) return st;
-                return submit_impl(h, n, env_ids, prefix_kv, noise, out, sm_quota, stream, ext, host_buffers);
-            }
+        if (!pull && s.stage_used != 0 && s.kv_stage_bytes < need) {
+            // staging already referenced by queued groups: close the batch first, and remember how much
+            // a whole batch of such groups would have taken so that the slots grow to it when next empty
+            const size_t whole = need / (size_t)(s.groups_pending + 1) * (size_t)c.max_inflight_groups;
+            h->stage_hint = std::max(h->stage_hint, std::max(need, whole));
+            if ((st = flush_slot(h, s)) != EBRL_OK) return st;
+            return submit_impl(h, n, env_ids, prefix_kv, noise, out, sm_quota, stream, ext, host_buffers);
+        }
+        if (!pull && (s.kv_stage_bytes < need || (s.stage_used == 0 && s.kv_stage_bytes < h->stage_hint))) {   // nothing staged in the slot: grow it
             if (s.kv_stage) cudaFree(s.kv_stage);
             s.kv_stage = nullptr; s.kv_stage_bytes = 0;
-            const size_t want = (size_t)c.max_inflight_groups * need;   // room for a whole batch of such groups
+            const size_t want = std::max((size_t)c.max_inflight_groups * need, h->stage_hint);   // room for a whole batch of such groups
             cudaError_t e = cudaMalloc((void **)&s.kv_stage, want);
             if (e != cudaSuccess) {
                 cudaGetLastError();
+                h->stage_hint = 0;
                 e = cudaMalloc((void **)&s.kv_stage, need);
                 if (e != cudaSuccess) { cudaGetLastError(); return fail(h, EBRL_ERR_NOMEM, "staging of %zu bytes: %s", need, cudaGetErrorString(e)); }
                 s.kv_stage_bytes = need;
@@ -652,7 +673,11 @@ ebrl_status_t submit_impl(ebrl_actgen *h, int32_t n, const int64_t *env_ids, con
     h->stats.envs += (uint64_t)n;
     h->stats.env_steps += env_steps;
     h->stats.granted_sms = grid;
-    if (s.groups_pending >= c.max_inflight_groups) return flush_slot(h, s);
+    // Batches of host-staged groups ramp up after a sync (1, 2, 4, ... groups, up to the configured
+    // depth): the first uploads are the only ones nothing can hide, so the first batch is kept small
+    // and every later batch uploads while the one before it computes.
+    const int depth = host_buffers ? std::min(h->host_depth, c.max_inflight_groups) : c.max_inflight_groups;
+    if (s.groups_pending >= depth) return flush_slot(h, s);
     return EBRL_OK;
 }
 
@@ -891,6 +916,7 @@ ebrl_status_t ebrl_actgen_sync(ebrl_actgen_t h)
         ebrl_status_t st = retire(h, s);
         if (st != EBRL_OK && first == EBRL_OK) first = st;
     }
+    h->host_depth = 1;
     if (first == EBRL_OK && h->status_d) {
         int word = 0;
         if (cudaMemcpy(&word, h->status_d, sizeof word, cudaMemcpyDeviceToHost) == cudaSuccess && word != 0) {

@@ -92,6 +92,8 @@ __global__ void __launch_bounds__(THREADS, 1) attn_mma_kernel(AttnArgs a, int hp
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    pdl_launch_dependents();
+    pdl_wait();
 
     bool ok = true;
 
@@ -377,11 +379,11 @@ cudaError_t launch_attn_mma(const AttnArgs &a, int grid, unsigned long long limi
     if (a.hd == 128) {
         e = cudaFuncSetAttribute(am::attn_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        am::attn_mma_kernel<128><<<g, am::THREADS, smem, st>>>(a, hpc, la, limit_ns, status);
+        return launch_kernel(am::attn_mma_kernel<128>, g, am::THREADS, smem, st, 1, a, hpc, la, limit_ns, status);
     } else {
         e = cudaFuncSetAttribute(am::attn_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        am::attn_mma_kernel<64><<<g, am::THREADS, smem, st>>>(a, hpc, la, limit_ns, status);
+        return launch_kernel(am::attn_mma_kernel<64>, g, am::THREADS, smem, st, 1, a, hpc, la, limit_ns, status);
     }
     return cudaGetLastError();
 }

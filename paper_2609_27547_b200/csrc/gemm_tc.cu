@@ -106,6 +106,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     bool ok = true;
+    pdl_launch_dependents();
+    pdl_wait();   // set-up done; from here on the previous kernel's results are needed
 
     if (warp == 0) {
         // ---- TMA producer
@@ -243,9 +245,8 @@ static cudaError_t tc_launch(const TensorMap128 &ta, const TensorMap128 &tw, con
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    tc::gemm_tc_kernel<EPI, BN><<<g, tc::Shape<BN>::THREADS, tc::Shape<BN>::SMEM_BYTES, st>>>(
-        *reinterpret_cast<const CUtensorMap *>(&ta), *reinterpret_cast<const CUtensorMap *>(&tw), a, limit_ns, status);
-    return cudaGetLastError();
+    return launch_kernel(tc::gemm_tc_kernel<EPI, BN>, g, tc::Shape<BN>::THREADS, tc::Shape<BN>::SMEM_BYTES, st, 1,
+                         *reinterpret_cast<const CUtensorMap *>(&ta), *reinterpret_cast<const CUtensorMap *>(&tw), a, limit_ns, status);
 }
 
 // One CTA per tile; bn = 256 or 128 columns per tile.

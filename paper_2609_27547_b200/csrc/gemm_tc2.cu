@@ -124,6 +124,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     bool ok = true;
+    pdl_launch_dependents();
+    pdl_wait();   // set-up done; from here on the previous kernel's results are needed
 
     if (warp == 0) {
         // ---- TMA producer (both CTAs): own A rows, own half of the weight tile; bytes land on the leader's barrier
@@ -225,20 +227,8 @@ static cudaError_t tc2_launch(const TensorMap128 &ta, const TensorMap128 &tw, co
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)g, 1, 1);
-    cfg.blockDim = dim3(tc2::THREADS, 1, 1);
-    cfg.dynamicSmemBytes = tc2::SMEM_BYTES;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, tc2::gemm_tc2_kernel<EPI>, *reinterpret_cast<const CUtensorMap *>(&ta),
-                              *reinterpret_cast<const CUtensorMap *>(&tw), a, limit_ns, status);
+    return launch_kernel(tc2::gemm_tc2_kernel<EPI>, g, tc2::THREADS, tc2::SMEM_BYTES, st, 2, *reinterpret_cast<const CUtensorMap *>(&ta),
+                         *reinterpret_cast<const CUtensorMap *>(&tw), a, limit_ns, status);
 }
 
 // grid = SM quota; the kernel uses floor(grid / 2) CTA pairs.  Needs grid >= 2.

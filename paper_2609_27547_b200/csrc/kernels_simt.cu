@@ -55,9 +55,11 @@ __global__ void __launch_bounds__(1024) embed_kernel(EmbedArgs a)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const T *w_in = (const T *)a.w_in;
     T *xg = (T *)a.xg;
-    for (int c = threadIdx.x; c < a.d; c += blockDim.x)
+    pdl_launch_dependents();
+    for (int c = threadIdx.x; c < a.d; c += blockDim.x)   // weights do not depend on the previous kernel
         for (int j = 0; j < a.A; ++j) wT[j * a.d + c] = ldf(w_in + (size_t)c * a.A + j);
     __syncthreads();
+    pdl_wait();
     // two rows per warp pass: each staged weight is used for both
     for (int row0 = (blockIdx.x * 32 + warp) * 2; row0 < rows; row0 += gridDim.x * 64) {
         float aj[2][AMAX];
@@ -121,10 +123,12 @@ __global__ void __launch_bounds__(HEAD_WARPS * 32) head_kernel(HeadArgs a)
     const int rows = a.n_envs * a.H;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const T *w_out = (const T *)a.w_out;
+    pdl_launch_dependents();
     if (!a.pull) {
-        for (int e = threadIdx.x; e < a.A * a.d; e += blockDim.x) wO[e] = ldf(w_out + e);
+        for (int e = threadIdx.x; e < a.A * a.d; e += blockDim.x) wO[e] = ldf(w_out + e);   // weights: no dependency
     }
     __syncthreads();
+    pdl_wait();
     for (int row0 = (blockIdx.x * HEAD_WARPS + warp) * 2; row0 < rows; row0 += gridDim.x * HEAD_WARPS * 2) {
         const int nr = min(2, rows - row0);
         float acc[2][AMAX];
@@ -212,6 +216,8 @@ __global__ void __launch_bounds__(1024) gemm_simt_kernel(GemmArgs g)
     const T *A = (const T *)g.A;
     const T *W = (const T *)g.W;
     const int ntm = (g.M + GT - 1) / GT, ntn = g.N / GT, ntiles = ntm * ntn, nk = g.K / GK;
+    pdl_launch_dependents();
+    pdl_wait();
     for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
         const int m0 = (tile / ntn) * GT, n0 = (tile % ntn) * GT;
         float acc[4][4];
@@ -316,6 +322,8 @@ __global__ void __launch_bounds__(512) attn_simt_kernel(AttnArgs a)
     const int ncg = 128 >> hd_sh, c = t & (hd - 1), rg = t >> hd_sh;
     const float scale = 1.0f / sqrtf((float)hd);
     const int items = a.n_envs * a.n_heads;
+    pdl_launch_dependents();
+    pdl_wait();
     for (int item = blockIdx.x * 4 + grp; item < items; item += gridDim.x * 4) {
         const int env = item / a.n_heads, h = item - env * a.n_heads;
         const T *kbase, *vbase;
@@ -424,8 +432,7 @@ static cudaError_t embed_launch(const EmbedArgs &a, int g, size_t smem, cudaStre
 {
     cudaError_t e = cudaFuncSetAttribute(embed_kernel<T, AMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    embed_kernel<T, AMAX><<<g, 1024, smem, st>>>(a);
-    return cudaGetLastError();
+    return launch_kernel(embed_kernel<T, AMAX>, g, 1024, smem, st, 1, a);
 }
 
 template <typename T>
@@ -451,8 +458,7 @@ static cudaError_t head_launch(const HeadArgs &a, int g, size_t smem, cudaStream
 {
     cudaError_t e = cudaFuncSetAttribute(head_kernel<T, AMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    head_kernel<T, AMAX><<<g, HEAD_WARPS * 32, smem, st>>>(a);
-    return cudaGetLastError();
+    return launch_kernel(head_kernel<T, AMAX>, g, HEAD_WARPS * 32, smem, st, 1, a);
 }
 
 template <typename T>
@@ -477,11 +483,10 @@ template <typename T>
 static cudaError_t gemm_simt_dispatch(const GemmArgs &a, int g, cudaStream_t st)
 {
     switch (a.epi) {
-    case EPI_SCALE_STORE: gemm_simt_kernel<T, EPI_SCALE_STORE><<<g, 1024, 0, st>>>(a); break;
-    case EPI_SCALE_GELU: gemm_simt_kernel<T, EPI_SCALE_GELU><<<g, 1024, 0, st>>>(a); break;
-    default: gemm_simt_kernel<T, EPI_RESID><<<g, 1024, 0, st>>>(a); break;
+    case EPI_SCALE_STORE: return launch_kernel(gemm_simt_kernel<T, EPI_SCALE_STORE>, g, 1024, 0, st, 1, a);
+    case EPI_SCALE_GELU: return launch_kernel(gemm_simt_kernel<T, EPI_SCALE_GELU>, g, 1024, 0, st, 1, a);
+    default: return launch_kernel(gemm_simt_kernel<T, EPI_RESID>, g, 1024, 0, st, 1, a);
     }
-    return cudaGetLastError();
 }
 
 cudaError_t launch_gemm_simt(const GemmArgs &a, int bf16, int grid, cudaStream_t st)
@@ -497,8 +502,7 @@ static cudaError_t attn_launch(const AttnArgs &a, int g, size_t smem, cudaStream
 {
     cudaError_t e = cudaFuncSetAttribute(attn_simt_kernel<T, RMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    attn_simt_kernel<T, RMAX><<<g, 512, smem, st>>>(a);
-    return cudaGetLastError();
+    return launch_kernel(attn_simt_kernel<T, RMAX>, g, 512, smem, st, 1, a);
 }
 
 template <typename T>
