@@ -39,7 +39,7 @@ class _Cfg(C.Structure):
     _fields_ = [("H", C.c_int32), ("A", C.c_int32), ("d", C.c_int32), ("n_layers", C.c_int32),
                 ("n_heads", C.c_int32), ("mlp_mult", C.c_int32), ("K_steps", C.c_int32),
                 ("kv_layers", C.c_int32), ("rms_eps", C.c_double), ("temb_scale", C.c_double),
-                ("temb_max_period", C.c_double)]
+                ("temb_max_period", C.c_double), ("d_ctx", C.c_int32)]
 
 
 _FP = C.POINTER(C.c_float)
@@ -49,7 +49,7 @@ _FPP = C.POINTER(_FP)
 class _Weights(C.Structure):
     _fields_ = [("w_in", _FP), ("w_out", _FP), ("b_out", _FP), ("g_final", _FP),
                 ("g1", _FPP), ("g2", _FPP), ("g3", _FPP), ("w_qkv", _FPP), ("w_o", _FPP),
-                ("w_qc", _FPP), ("w_oc", _FPP), ("w_1", _FPP), ("w_2", _FPP)]
+                ("w_qc", _FPP), ("w_oc", _FPP), ("w_1", _FPP), ("w_2", _FPP), ("w_kc", _FPP), ("w_vc", _FPP)]
 
 
 _lib = None
@@ -80,11 +80,12 @@ class OracleConfig:
     rms_eps: float = 1e-6
     temb_scale: float = 1000.0
     temb_max_period: float = 10000.0
+    d_ctx: int = 0     # > 0: prefixes are hidden states [P][d_ctx]; layers carry w_kc, w_vc [d][d_ctx]
 
     def _c(self) -> _Cfg:
         return _Cfg(self.H, self.A, self.d, self.n_layers, self.n_heads, self.mlp_mult,
                     self.K_steps, self.kv_layers, self.rms_eps, self.temb_scale,
-                    self.temb_max_period)
+                    self.temb_max_period, self.d_ctx)
 
 
 def _f32(a) -> np.ndarray:
@@ -99,7 +100,8 @@ def _fp(a: np.ndarray):
 class OracleWeights:
     """Weights as float32 numpy arrays (bf16 models pass values already rounded to bf16).
 
-    ``layers`` is a list of dicts with keys g1, g2, g3, w_qkv, w_o, w_qc, w_oc, w_1, w_2.
+    ``layers`` is a list of dicts with keys g1, g2, g3, w_qkv, w_o, w_qc, w_oc, w_1, w_2 (and
+    w_kc, w_vc [d][d_ctx] when the prefix is given as hidden states).
     All matrices are [out][in] row-major: y = W x.
     """
     w_in: np.ndarray
@@ -115,7 +117,9 @@ class OracleWeights:
             arr = _f32(getattr(self, name))
             keep.append(arr)
             setattr(w, name, _fp(arr))
-        for name in ("g1", "g2", "g3", "w_qkv", "w_o", "w_qc", "w_oc", "w_1", "w_2"):
+        for name in ("g1", "g2", "g3", "w_qkv", "w_o", "w_qc", "w_oc", "w_1", "w_2", "w_kc", "w_vc"):
+            if name in ("w_kc", "w_vc") and not all(name in l for l in self.layers):
+                continue   # only models with hidden-state prefixes carry them
             arrs = [_f32(l[name]) for l in self.layers]
             keep.extend(arrs)
             ptrs = (_FP * max(1, len(arrs)))(*[_fp(a) for a in arrs])
@@ -163,7 +167,8 @@ def attention_head(q, k, v) -> np.ndarray:
 
 
 def velocity(cfg: OracleConfig, w: OracleWeights, kv, a, k: int) -> np.ndarray:
-    """Network velocity of one environment at Euler step k.  kv: [kv_layers][2][P][d]."""
+    """Network velocity of one environment at Euler step k.  kv: [kv_layers][2][P][d], or the
+    hidden states [P][d_ctx] when ``cfg.d_ctx > 0``."""
     kv = _f32(kv)
     P = kv.shape[-2]
     a = np.ascontiguousarray(np.asarray(a, dtype=np.float64)).reshape(cfg.H, cfg.A)
@@ -184,7 +189,8 @@ def actgen(cfg: OracleConfig, w: OracleWeights, prefix_kv: Sequence, noise,
            n_threads: Optional[int] = None, pull: bool = False) -> np.ndarray:
     """Advance every environment of a group; returns float64 [n][H][A].
 
-    prefix_kv[i]: array [kv_layers][2][P_i][d] (values already rounded to the stored dtype).
+    prefix_kv[i]: array [kv_layers][2][P_i][d] (values already rounded to the stored dtype), or the
+    hidden states [P_i][d_ctx] when ``cfg.d_ctx > 0``.
     noise: [n][H][A] float32, environment i's action state at step ``step_index[i]``.
     ``pull`` replaces the network by the linear field v = b_out - a (integrator pin).
     """
@@ -195,7 +201,10 @@ def actgen(cfg: OracleConfig, w: OracleWeights, prefix_kv: Sequence, noise,
     plen = np.array([p.shape[-2] for p in kvs] if kvs else [0] * n, dtype=np.int32)
     if kvs:
         for p in kvs:
-            assert p.shape[-1] == cfg.d and p.shape[-3] == 2
+            if cfg.d_ctx > 0:
+                assert p.ndim == 2 and p.shape[-1] == cfg.d_ctx     # hidden states [P][d_ctx]
+            else:
+                assert p.shape[-1] == cfg.d and p.shape[-3] == 2
         ptrs = (_FP * max(1, n))(*[_fp(p) for p in kvs])
         ptrs_arg = C.cast(ptrs, _FPP)
     else:

@@ -41,6 +41,10 @@ typedef struct {
     double rms_eps;
     double temb_scale;
     double temb_max_period;
+    int32_t d_ctx;      /* 0: the prefix is the cached K/V planes.  > 0: the prefix is the backbone's
+                           hidden states [P][d_ctx] and every layer projects its own keys and values
+                           from them (the cross-attention form of heads that attend to backbone
+                           features rather than to a ready-made cache, section 2.1)               */
 } ebrl_oracle_cfg;
 
 typedef struct {
@@ -58,6 +62,8 @@ typedef struct {
     const float *const *w_oc;  /* [d][d]   */
     const float *const *w_1;   /* [md][d]  */
     const float *const *w_2;   /* [d][md]  */
+    const float *const *w_kc;  /* [d][d_ctx]  key projection of the hidden-state prefix (d_ctx > 0)   */
+    const float *const *w_vc;  /* [d][d_ctx]  value projection, likewise                              */
 } ebrl_oracle_weights;
 
 /* ------------------------------------------------------------------------------------------
@@ -155,7 +161,9 @@ void ebrl_oracle_attention_head(const double *q, int nq, const float *k, const f
 
 /* ------------------------------------------------------------------------------------------
  * The velocity network for one environment at Euler step k:  v = f(a, t_k; prefix K/V).
- * a, v: [H][A] doubles.  kv: [kv_layers][2][P][d] floats (plane 0 = K, plane 1 = V).
+ * a, v: [H][A] doubles.  kv: [kv_layers][2][P][d] floats (plane 0 = K, plane 1 = V); with
+ * d_ctx > 0 it is the hidden states [P][d_ctx] and layer l attends to Kc = h W_kc_l^T,
+ * Vc = h W_vc_l^T (nothing rounded in between).
  * ---------------------------------------------------------------------------------------- */
 int ebrl_oracle_velocity(const ebrl_oracle_cfg *c, const ebrl_oracle_weights *w,
                          const float *kv, int P, const double *a, int k, double *v)
@@ -198,7 +206,23 @@ int ebrl_oracle_velocity(const ebrl_oracle_cfg *c, const ebrl_oracle_weights *w,
             ebrl_oracle_rmsnorm(x + (size_t)h * d, w->g2[l], d, c->rms_eps, y);
             matvec(w->w_qc[l], y, d, d, qc + (size_t)h * d, 0);
         }
-        {
+        if (c->d_ctx > 0) {
+            /* keys and values of this layer from the prefix's hidden states, row by row */
+            const int dc = c->d_ctx;
+            double *Kd = (double *)malloc(sizeof(double) * (size_t)P * d);
+            double *Vd = (double *)malloc(sizeof(double) * (size_t)P * d);
+            double *hrow = (double *)malloc(sizeof(double) * (size_t)dc);
+            if (!Kd || !Vd || !hrow) return 1;
+            for (int p = 0; p < P; ++p) {
+                for (int j = 0; j < dc; ++j) hrow[j] = (double)kv[(size_t)p * dc + j];
+                matvec(w->w_kc[l], hrow, d, dc, Kd + (size_t)p * d, 0);
+                matvec(w->w_vc[l], hrow, d, dc, Vd + (size_t)p * d, 0);
+            }
+            for (int hh = 0; hh < nh; ++hh)
+                attention_head(qc + (size_t)hh * hd, d, H, Kd + (size_t)hh * hd, Vd + (size_t)hh * hd,
+                               NULL, NULL, d, P, hd, att + (size_t)hh * hd, d, scores);
+            free(Kd); free(Vd); free(hrow);
+        } else {
             const int pl = (c->kv_layers == 1) ? 0 : l;
             const float *Kc = kv + (size_t)pl * 2 * (size_t)P * d;
             const float *Vc = Kc + (size_t)P * d;

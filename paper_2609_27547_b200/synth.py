@@ -112,6 +112,7 @@ class Workload:
     quota: int                  # SM quota the configuration names (0 = all)
     mixed_steps: bool = False   # environments start at independent Euler steps
     mlp_mult: int = 4
+    d_ctx: int = 0              # > 0: prefixes are hidden states [P][d_ctx], projected to K/V per layer
 
     @property
     def torch_dtype(self):
@@ -169,6 +170,9 @@ def make_weights(w: Workload, seed: int = DEFAULT_SEED, device="cpu", random_gai
             "w_qc": mat("w_qc", d, d, l), "w_oc": mat("w_oc", d, d, l),
             "w_1": mat("w_1", md, d, l), "w_2": mat("w_2", d, md, l),
         })
+        if w.d_ctx > 0:
+            out["layers"][-1]["w_kc"] = mat("w_kc", d, w.d_ctx, l)
+            out["layers"][-1]["w_vc"] = mat("w_vc", d, w.d_ctx, l)
     return out
 
 
@@ -176,7 +180,8 @@ def make_weights(w: Workload, seed: int = DEFAULT_SEED, device="cpu", random_gai
 class EnvInputs:
     env_id: int
     noise: torch.Tensor        # [H][A] fp32: the action state at step ``step``
-    kv: torch.Tensor           # [1][2][P][d] in the workload's dtype (plane 0 = K, 1 = V)
+    kv: torch.Tensor           # [1][2][P][d] in the workload's dtype (plane 0 = K, 1 = V); with
+                               # d_ctx > 0 the hidden states [P][d_ctx] instead
     P: int
     step: int                  # Euler step index the environment sits at
 
@@ -185,7 +190,10 @@ def make_env(w: Workload, env_id: int, seed: int = DEFAULT_SEED, device="cpu") -
     P = uniform_int(seed, "prefix_len", env_id, w.P[0], w.P[1])
     step = uniform_int(seed, "step_index", env_id, 0, w.K - 1) if w.mixed_steps else 0
     noise = normal(seed, "noise", env_id, (w.H, w.A), device=device)
-    kv = normal(seed, "prefix_kv", env_id, (1, 2, P, w.d), dtype=w.torch_dtype, device=device)
+    if w.d_ctx > 0:
+        kv = normal(seed, "prefix_hidden", env_id, (P, w.d_ctx), dtype=w.torch_dtype, device=device)
+    else:
+        kv = normal(seed, "prefix_kv", env_id, (1, 2, P, w.d), dtype=w.torch_dtype, device=device)
     return EnvInputs(env_id, noise, kv, P, step)
 
 

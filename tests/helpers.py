@@ -10,7 +10,7 @@ from paper_2609_27547_b200 import synth
 
 def oracle_cfg(w: synth.Workload) -> oracle.OracleConfig:
     return oracle.OracleConfig(H=w.H, A=w.A, d=w.d, n_layers=w.L, n_heads=w.n_heads, K_steps=w.K,
-                               mlp_mult=w.mlp_mult)
+                               mlp_mult=w.mlp_mult, d_ctx=w.d_ctx, kv_layers=w.L if w.d_ctx > 0 else 1)
 
 
 def np32(t: torch.Tensor) -> np.ndarray:

@@ -410,7 +410,8 @@ def _torch_reference(w, wt, env, n_steps=0):
     D = torch.float64
     H, d, nh, hd = w.H, w.d, w.n_heads, w.head_dim
     a = env.noise.to(D)
-    Kc, Vc = env.kv[0, 0].to(D), env.kv[0, 1].to(D)
+    if w.d_ctx == 0:
+        Kc, Vc = env.kv[0, 0].to(D), env.kv[0, 1].to(D)
     k1 = w.K if n_steps == 0 else min(w.K, env.step + n_steps)
     for k in range(env.step, k1):
         j = torch.arange(d // 2, dtype=D)
@@ -424,6 +425,8 @@ def _torch_reference(w, wt, env, n_steps=0):
             x = x + (p @ sh(v, H)).transpose(0, 1).reshape(H, d) @ l["w_o"].to(D).T
             y = F.rms_norm(x, (d,), l["g2"].to(D), 1e-6)
             qc = y @ l["w_qc"].to(D).T
+            if w.d_ctx > 0:   # this layer's keys and values from the prefix's hidden states
+                Kc, Vc = env.kv.to(D) @ l["w_kc"].to(D).T, env.kv.to(D) @ l["w_vc"].to(D).T
             P = Kc.shape[0]
             p = torch.softmax(sh(qc, H) @ sh(Kc, P).transpose(1, 2) / math.sqrt(hd), dim=-1)
             x = x + (p @ sh(Vc, P)).transpose(0, 1).reshape(H, d) @ l["w_oc"].to(D).T
@@ -445,6 +448,60 @@ def test_against_torch_fp64_composition(dtype):
     got1 = oracle_run(w, wt, envs, n_steps=1)
     for i, e in enumerate(envs):
         assert np.abs(got1[i] - _torch_reference(w, wt, e, n_steps=1)).max() < 1e-11
+
+
+# ---------------------------------------------------------------- hidden-state prefixes
+
+def test_hidden_prefix_with_identity_projections_is_the_plane_form():
+    """d_ctx = d and W_kc = W_vc = I in every layer: keys and values are the hidden states
+    themselves, i.e. the cached-plane form with K = V = h (exact: the products add only zeros)."""
+    w = small(d_ctx=16)
+    wt = synth.make_weights(w, SEED, random_gains=True)
+    for l in wt["layers"]:
+        l["w_kc"] = torch.eye(w.d)
+        l["w_vc"] = torch.eye(w.d)
+    envs = [synth.make_env(w, e, SEED) for e in range(w.B)]
+    got = oracle_run(w, wt, envs)
+    wp = small()
+    plane_envs = [synth.EnvInputs(e.env_id, e.noise, torch.stack([e.kv, e.kv])[None], e.P, e.step) for e in envs]
+    want = oracle_run(wp, wt, plane_envs)
+    assert np.array_equal(got, want)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_hidden_prefix_against_torch_fp64_composition(dtype):
+    """Per-layer K = h W_kc^T, V = h W_vc^T composed from torch matmuls: pins the orientation of the
+    projections, which of the two feeds keys and which values, and the layer each pair belongs to."""
+    w = synth.scaled(synth.WORKLOADS[0], B=3, dtype=dtype, P=(9, 33), mixed_steps=True, d_ctx=64)
+    wt = synth.make_weights(w, SEED, random_gains=True)
+    envs = [synth.make_env(w, e, SEED) for e in range(w.B)]
+    assert envs[0].kv.shape == (envs[0].P, 64) and wt["layers"][1]["w_kc"].shape == (w.d, 64)
+    got = oracle_run(w, wt, envs)
+    for i, e in enumerate(envs):
+        assert np.abs(got[i] - _torch_reference(w, wt, e)).max() < 1e-11
+    # swapping the two projections, or the two layers' projections, must change the result
+    sw = {**wt, "layers": [{**l, "w_kc": l["w_vc"], "w_vc": l["w_kc"]} for l in wt["layers"]]}
+    assert np.abs(oracle_run(w, sw, envs) - got).max() > 1e-4
+    l0, l1 = wt["layers"]
+    sl = {**wt, "layers": [{**l0, "w_kc": l1["w_kc"], "w_vc": l1["w_vc"]}, {**l1, "w_kc": l0["w_kc"], "w_vc": l0["w_vc"]}]}
+    assert np.abs(oracle_run(w, sl, envs) - got).max() > 1e-4
+
+
+def test_hidden_prefix_single_token_closed_form():
+    """P = 1: the softmax over one key is 1, so the cross-attention block adds W_oc W_vc h_0 to
+    every token whatever the queries and W_kc are; with the other blocks silenced,
+    v = W_out RMSNorm(x0 + W_oc W_vc h_0) + b."""
+    w = small(L=1, K=1, P=(1, 1), d_ctx=64)
+    wt = _only_cross(w, synth.make_weights(w, SEED, random_gains=True))
+    e = synth.make_env(w, 0, SEED)
+    l = wt["layers"][0]
+    x = _embed(w, wt, np32(e.noise), 0)
+    add = np32(l["w_oc"]).astype(np.float64) @ (np32(l["w_vc"]).astype(np.float64) @ np32(e.kv).astype(np.float64)[0])
+    want = np32(e.noise) + _head(w, wt, x + add[None, :])
+    got = oracle_run(w, wt, [e])[0]
+    assert np.abs(got - want).max() < 1e-12
+    l["w_kc"] = torch.zeros_like(l["w_kc"])
+    assert np.abs(oracle_run(w, wt, [e])[0] - want).max() < 1e-12
 
 
 def test_golden_regression():
