@@ -19,6 +19,9 @@
  *     v     = W_out RMSNorm(x; g_final) + b_out
  *     a    += v / K                                                   (explicit Euler)
  *
+ *     (variant cfg.d_ctx > 0, the prefix given as hidden states h in R^{P_e x d_ctx}: layer l uses
+ *      Kc = h W_kc_l^T, Vc = h W_vc_l^T, computed once per batch and stored in kv_dtype)
+ *
  *     temb(t)_j = sin(temb_scale * t * w_j), temb(t)_{d/2+j} = cos(temb_scale * t * w_j),
  *     w_j = temb_max_period^(-j/(d/2));   RMSNorm(x; g)_j = g_j x_j / sqrt(mean(x^2) + rms_eps).
  *
@@ -44,7 +47,7 @@
 extern "C" {
 #endif
 
-#define EBRL_ACTGEN_ABI_VERSION 1u
+#define EBRL_ACTGEN_ABI_VERSION 2u
 
 typedef struct ebrl_actgen *ebrl_actgen_t;
 
@@ -88,6 +91,12 @@ typedef struct {
     uint32_t flags;              /* EBRL_FLAG_*                                                 */
     int32_t device;              /* CUDA device ordinal                                         */
     uint64_t wait_limit_ns;      /* bound for device-side waits; 0 = default                    */
+    int32_t d_ctx;               /* 0: prefix_kv[i] holds the cached K/V planes themselves.
+                                    > 0: prefix_kv[i] holds the backbone's hidden states
+                                    [P_e][d_ctx] (kv_dtype) and every layer projects its own
+                                    planes Kc = h W_kc^T, Vc = h W_vc^T once per batch, before
+                                    the first Euler step; needs kv_layers == n_layers         */
+    int32_t reserved_;
 } ebrl_actgen_cfg_t;
 
 typedef struct {
@@ -99,6 +108,9 @@ typedef struct {
     const void *w_oc;            /* [d][d]   cross-attention output projection                  */
     const void *w_1;             /* [mlp_mult*d][d]                                             */
     const void *w_2;             /* [d][mlp_mult*d]                                             */
+    const void *w_kc;            /* [d][d_ctx] cross-attention key projection of the prefix's
+                                    hidden states; read only when cfg.d_ctx > 0, else NULL     */
+    const void *w_vc;            /* [d][d_ctx] value projection, likewise                       */
 } ebrl_layer_weights_t;
 
 /* Pointers may be host or device memory; everything is copied to the device at create and the
@@ -120,7 +132,8 @@ typedef struct {
 
 /* Kernel classes of the per-class timing (EBRL_FLAG_TIMING). */
 enum { EBRL_KC_EMBED = 0, EBRL_KC_GEMM = 1, EBRL_KC_SELF_ATTN = 2, EBRL_KC_CROSS_ATTN = 3,
-       EBRL_KC_HEAD = 4, EBRL_KC_COUNT = 5 };
+       EBRL_KC_HEAD = 4, EBRL_KC_PREFIX = 5 /* packing and projecting hidden-state prefixes */,
+       EBRL_KC_COUNT = 6 };
 
 typedef struct {
     uint64_t groups, envs, env_steps;     /* submitted since create                            */
@@ -152,7 +165,11 @@ ebrl_status_t ebrl_actgen_create(const ebrl_actgen_cfg_t *cfg, const ebrl_actgen
  *   env_ids    host [n]: unique within the group and among groups not yet synced.  Used only
  *              for these checks and for error text; they never enter the arithmetic.
  *   prefix_kv  host [n] of DEVICE pointers; env i: [kv_layers][2][P_i][d] in kv_dtype, plane 0
- *              = K, plane 1 = V, rows contiguous, 16-byte aligned.
+ *              = K, plane 1 = V, rows contiguous, 16-byte aligned.  With cfg.d_ctx > 0 env i's
+ *              pointer is instead its hidden states [P_i][d_ctx] in kv_dtype; the projected
+ *              planes live in scratch of the handle that grows to the largest batch seen
+ *              (n_layers * 2 * sum(P_i) * d elements per batch in flight; EBRL_ERR_NOMEM when
+ *              the device cannot hold it).
  *   noise      DEVICE [n][H][A] fp32: env i's action state at its step index (the initial
  *              noise when that is 0).
  *   out        DEVICE [n][H][A] fp32; may equal noise.
@@ -228,6 +245,11 @@ ebrl_status_t ebrl_actgen_reset_stats(ebrl_actgen_t h);
 ebrl_status_t ebrl_actgen_set_timing(ebrl_actgen_t h, int32_t on);
 
 uint32_t ebrl_actgen_abi_version(void);
+
+/* sizeof of an ABI struct as this library was compiled: 0 ebrl_actgen_cfg_t, 1 ebrl_layer_weights_t,
+ * 2 ebrl_actgen_weights_t, 3 ebrl_submit_ext_t, 4 ebrl_actgen_stats_t; 0 for any other index.  For
+ * bindings that mirror the structs by hand. */
+uint64_t ebrl_actgen_struct_size(int32_t which);
 
 /* ---- an entry point that allocates nothing ---------------------------------------------
  * (The paper has no counterpart; this serves callers that cannot call cudaMalloc.)

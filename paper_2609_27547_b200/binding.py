@@ -14,11 +14,11 @@ import torch
 
 from . import build as _build
 
-ABI_VERSION = 1
+ABI_VERSION = 2
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_NOMEM, ERR_CUDA, ERR_ENV_BUSY, ERR_QUOTA, ERR_TIMEOUT = range(8)
 F32, BF16 = 0, 1
 FLAG_TEST_PULL, FLAG_GREEN_CTX, FLAG_TIMING, FLAG_FORCE_SIMT = 1, 2, 4, 8
-KC_NAMES = ("embed", "gemm", "self_attn", "cross_attn", "head")
+KC_NAMES = ("embed", "gemm", "self_attn", "cross_attn", "head", "prefix")
 
 
 class Cfg(C.Structure):
@@ -28,13 +28,13 @@ class Cfg(C.Structure):
                 ("max_inflight_groups", C.c_int32), ("param_dtype", C.c_int32), ("kv_dtype", C.c_int32),
                 ("kv_layers", C.c_int32), ("rms_eps", C.c_float), ("temb_scale", C.c_float),
                 ("temb_max_period", C.c_float), ("flags", C.c_uint32), ("device", C.c_int32),
-                ("wait_limit_ns", C.c_uint64)]
+                ("wait_limit_ns", C.c_uint64), ("d_ctx", C.c_int32), ("reserved_", C.c_int32)]
 
 
 class LayerWeights(C.Structure):
     _fields_ = [("g1", C.c_void_p), ("g2", C.c_void_p), ("g3", C.c_void_p), ("w_qkv", C.c_void_p),
                 ("w_o", C.c_void_p), ("w_qc", C.c_void_p), ("w_oc", C.c_void_p), ("w_1", C.c_void_p),
-                ("w_2", C.c_void_p)]
+                ("w_2", C.c_void_p), ("w_kc", C.c_void_p), ("w_vc", C.c_void_p)]
 
 
 class Weights(C.Structure):
@@ -51,9 +51,9 @@ class Stats(C.Structure):
     _fields_ = [("groups", C.c_uint64), ("envs", C.c_uint64), ("env_steps", C.c_uint64),
                 ("kernel_launches", C.c_uint64), ("granted_sms", C.c_int32),
                 ("green_ctx_active", C.c_int32), ("green_ctx_sms", C.c_int32), ("reserved_", C.c_int32),
-                ("class_ms", C.c_double * 5),
-                ("class_launches", C.c_uint64 * 5), ("class_flops", C.c_double * 5),
-                ("class_bytes", C.c_double * 5), ("weights_version", C.c_uint64)]
+                ("class_ms", C.c_double * len(KC_NAMES)),
+                ("class_launches", C.c_uint64 * len(KC_NAMES)), ("class_flops", C.c_double * len(KC_NAMES)),
+                ("class_bytes", C.c_double * len(KC_NAMES)), ("weights_version", C.c_uint64)]
 
 
 class EbrlError(RuntimeError):
@@ -78,6 +78,8 @@ def lib():
         L.ebrl_actgen_last_error.restype = C.c_char_p
         L.ebrl_actgen_last_error.argtypes = [C.c_void_p]
         L.ebrl_actgen_abi_version.restype = C.c_uint32
+        L.ebrl_actgen_struct_size.restype = C.c_uint64
+        L.ebrl_actgen_struct_size.argtypes = [C.c_int32]
         L.ebrl_actgen_create.argtypes = [C.POINTER(Cfg), C.POINTER(Weights), C.POINTER(C.c_void_p)]
         sub = [C.c_void_p, C.c_int32, C.POINTER(C.c_int64), C.POINTER(C.c_void_p), C.c_void_p,
                C.c_void_p, C.c_int32, C.c_void_p, C.POINTER(SubmitExt)]
@@ -108,10 +110,11 @@ def lib():
 
 def make_cfg(*, H, A, d, n_layers, n_heads, K_steps, max_prefix_len, max_group_envs,
              max_inflight_groups=1, dtype=F32, mlp_mult=4, kv_layers=1, rms_eps=1e-6,
-             temb_scale=1000.0, temb_max_period=10000.0, flags=0, device=0) -> Cfg:
+             temb_scale=1000.0, temb_max_period=10000.0, flags=0, device=0, d_ctx=0) -> Cfg:
+    """``d_ctx > 0``: prefixes are hidden states [P][d_ctx] projected per layer (then kv_layers = n_layers)."""
     return Cfg(ABI_VERSION, H, A, d, n_layers, n_heads, mlp_mult, K_steps, max_prefix_len,
-               max_group_envs, max_inflight_groups, dtype, dtype, kv_layers, rms_eps, temb_scale,
-               temb_max_period, flags, device, 0)
+               max_group_envs, max_inflight_groups, dtype, dtype, n_layers if d_ctx > 0 else kv_layers, rms_eps,
+               temb_scale, temb_max_period, flags, device, 0, d_ctx, 0)
 
 
 def _ext(prefix_len, step_index, n_steps):
@@ -165,7 +168,9 @@ class ActGen:
         for i, l in enumerate(weights["layers"]):
             lw[i] = LayerWeights(ptr(l["g1"], torch.float32), ptr(l["g2"], torch.float32), ptr(l["g3"], torch.float32),
                                  ptr(l["w_qkv"], want), ptr(l["w_o"], want), ptr(l["w_qc"], want),
-                                 ptr(l["w_oc"], want), ptr(l["w_1"], want), ptr(l["w_2"], want))
+                                 ptr(l["w_oc"], want), ptr(l["w_1"], want), ptr(l["w_2"], want),
+                                 ptr(l["w_kc"], want) if cfg.d_ctx > 0 else None,
+                                 ptr(l["w_vc"], want) if cfg.d_ctx > 0 else None)
         keep.append(lw)
         w = Weights(ptr(weights["w_in"], want), ptr(weights["w_out"], want), ptr(weights["b_out"], torch.float32),
                     ptr(weights["g_final"], torch.float32), C.cast(lw, C.POINTER(LayerWeights)))
@@ -199,7 +204,8 @@ class ActGen:
                out: torch.Tensor, sm_quota: int = 0, stream: Optional[torch.cuda.Stream] = None,
                prefix_len: Optional[Sequence[int]] = None, step_index: Optional[Sequence[int]] = None,
                n_steps: int = 0):
-        """``ebrl_actgen_submit``: device tensors; prefix_kv[i] is [kv_layers][2][P_i][d]."""
+        """``ebrl_actgen_submit``: device tensors; prefix_kv[i] is [kv_layers][2][P_i][d], or the
+        hidden states [P_i][d_ctx] when the handle was created with ``d_ctx > 0``."""
         if noise.device.type != "cuda" or out.device.type != "cuda":
             raise ValueError("noise and out must be CUDA tensors")
         if noise.dtype != torch.float32 or out.dtype != torch.float32 or not noise.is_contiguous() or not out.is_contiguous():
@@ -301,4 +307,4 @@ def cfg_for(w, *, max_group_envs: Optional[int] = None, max_inflight_groups: int
     return make_cfg(H=w.H, A=w.A, d=w.d, n_layers=w.L, n_heads=w.n_heads, K_steps=w.K, max_prefix_len=w.P[1],
                     max_group_envs=max_group_envs or (w.group[1] if w.group else w.B),
                     max_inflight_groups=max_inflight_groups, dtype=BF16 if w.dtype == "bf16" else F32,
-                    mlp_mult=w.mlp_mult, flags=flags, device=device)
+                    mlp_mult=w.mlp_mult, flags=flags, device=device, d_ctx=getattr(w, "d_ctx", 0))

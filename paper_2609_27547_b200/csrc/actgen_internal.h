@@ -20,9 +20,10 @@ struct EnvMeta {
     int32_t P;         // prefix length
     int32_t k0;        // Euler step index the environment starts from
     int32_t nsteps;    // steps to run in this submit
-    int32_t pad_;
+    int32_t row0;      // hidden-state prefixes: first row of the environment in the batch's packed prefix rows
     const float *noise;  // device: the environment's [H][A] state on entry
     float *out;          // device: where its [H][A] result goes
+    const void *hid;   // hidden-state prefixes: device [P][d_ctx] as given by the caller (kv then points into the projected planes)
 };
 
 // Opaque storage of a CUtensorMap (the driver's 128-byte TMA descriptor).
@@ -62,6 +63,8 @@ struct AttnArgs {
     const EnvMeta *meta;   // used when self == 0
     int d;                 // plane row length
     int kv_plane;          // plane pair index (layer index when kv_layers > 1, else 0)
+    int plane_rows;        // rows from one plane of an environment to its next: 0 = the environment's own P
+                           // (planes given by the caller), else the batch's packed prefix rows (projected planes)
     // self attention: keys/values are the environment's own rows
     int self;
     const void *k_self;    // [rows][kv_stride]
@@ -162,6 +165,17 @@ inline cudaError_t launch_kernel(void (*kern)(KArgs...), int grid, int block, si
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 #endif
+
+// Gathers the hidden-state prefixes of a batch into one [sum P][d_ctx] matrix (row0 of each
+// environment from its record), the A operand of the K/V projections.
+struct PackArgs {
+    const EnvMeta *meta;
+    int n_envs;
+    int slices;            // 64-row slices per environment: ceil(longest prefix / 64)
+    int row_bytes;         // d_ctx * sizeof(element), a multiple of 16
+    void *dst;
+};
+cudaError_t launch_pack_prefix(const PackArgs &a, int grid, cudaStream_t st);
 
 // Launchers (plain-ALU kernels).  bf16 != 0 selects bf16 activations/weights/planes.
 // grid = number of persistent CTAs (the SM quota).

@@ -36,7 +36,8 @@ namespace {
 struct LayerDev {
     float *g1 = nullptr, *g2 = nullptr, *g3 = nullptr;
     void *w_qkv = nullptr, *w_o = nullptr, *w_qc = nullptr, *w_oc = nullptr, *w_1 = nullptr, *w_2 = nullptr;
-    TensorMap128 t_qkv, t_o, t_qc, t_oc, t_1, t_2;   // TMA descriptors of the matrices (tensor-core path)
+    void *w_kc = nullptr, *w_vc = nullptr;           // hidden-state prefixes (cfg.d_ctx > 0): [d][d_ctx] each
+    TensorMap128 t_qkv, t_o, t_qc, t_oc, t_1, t_2, t_kc, t_vc;   // TMA descriptors of the matrices (tensor-core path)
 };
 
 // One complete copy of the policy's weights on the device.  The handle keeps two, so that a new
@@ -87,6 +88,12 @@ struct Slot {
     size_t stage_used = 0, chunks_used = 0;
     cudaEvent_t h2d_done = nullptr, part_in = nullptr, part_out = nullptr;
     bool has_uploads = false;
+    // hidden-state prefixes: the batch's packed hidden rows and the planes projected from them
+    // ([n_layers][2][prefix_rows][d]); both grow to the largest batch seen
+    void *hid_pack = nullptr, *planes = nullptr;
+    size_t proj_cap_rows = 0;
+    int prefix_rows = 0, prefix_slices = 0;   // of the batch being launched
+    TensorMap128 t_hid;
 };
 
 thread_local std::string g_create_error;
@@ -157,6 +164,11 @@ ebrl_status_t check_cfg(const ebrl_actgen_cfg_t *c, std::string *why)
     if (hd != 32 && hd != 64 && hd != 128) return bad(EBRL_ERR_UNSUPPORTED, "head_dim must be 32, 64 or 128");
     if (c->param_dtype != c->kv_dtype) return bad(EBRL_ERR_UNSUPPORTED, "param_dtype and kv_dtype must match");
     if ((int64_t)c->d * c->A * 4 > 200 * 1024) return bad(EBRL_ERR_UNSUPPORTED, "d * A is limited to 51200 (the input embedding is staged in shared memory)");
+    if (c->d_ctx < 0) return bad(EBRL_ERR_INVALID_ARG, "d_ctx < 0");
+    if (c->d_ctx > 0) {
+        if (c->kv_layers != c->n_layers) return bad(EBRL_ERR_INVALID_ARG, "d_ctx > 0 (hidden-state prefixes) needs kv_layers == n_layers");
+        if (c->d_ctx % 64) return bad(EBRL_ERR_UNSUPPORTED, "d_ctx must be a multiple of 64");
+    }
     if ((int64_t)c->max_group_envs * c->max_inflight_groups * c->H > (int64_t)1 << 22)
         return bad(EBRL_ERR_UNSUPPORTED, "max_group_envs * max_inflight_groups * H is limited to 4M rows");
     return EBRL_OK;
@@ -273,6 +285,15 @@ ebrl_status_t alloc_weight_set(ebrl_actgen *h, WeightSet &ws)
         if ((st = dev_alloc(h, &o.w_oc, d * d * esz)) != EBRL_OK) return st;
         if ((st = dev_alloc(h, &o.w_1, md * d * esz)) != EBRL_OK) return st;
         if ((st = dev_alloc(h, &o.w_2, d * md * esz)) != EBRL_OK) return st;
+        if (c.d_ctx > 0) {
+            if ((st = dev_alloc(h, &o.w_kc, d * (size_t)c.d_ctx * esz)) != EBRL_OK) return st;
+            if ((st = dev_alloc(h, &o.w_vc, d * (size_t)c.d_ctx * esz)) != EBRL_OK) return st;
+            if (h->use_tc) {
+                const uint32_t bw = (uint32_t)gemm_tc_box_rows_w();
+                if (make_tmap_bf16(&o.t_kc, o.w_kc, (uint64_t)c.d_ctx, d, bw) | make_tmap_bf16(&o.t_vc, o.w_vc, (uint64_t)c.d_ctx, d, bw))
+                    return fail(h, EBRL_ERR_CUDA, "cuTensorMapEncodeTiled failed for a weight matrix");
+            }
+        }
         if (h->use_tc) {
             const uint32_t bw = (uint32_t)gemm_tc_box_rows_w();
             int bad = make_tmap_bf16(&o.t_qkv, o.w_qkv, d, 3 * d, bw) | make_tmap_bf16(&o.t_o, o.w_o, d, d, bw) |
@@ -299,6 +320,8 @@ ebrl_status_t upload_weight_set(ebrl_actgen *h, WeightSet &ws, const ebrl_actgen
         const ebrl_layer_weights_t &w = wts->layers[l];
         if (!w.g1 || !w.g2 || !w.g3 || !w.w_qkv || !w.w_o || !w.w_qc || !w.w_oc || !w.w_1 || !w.w_2)
             return fail(h, EBRL_ERR_INVALID_ARG, "a weight pointer of layer %d is NULL", l);
+        if (c.d_ctx > 0 && (!w.w_kc || !w.w_vc))
+            return fail(h, EBRL_ERR_INVALID_ARG, "w_kc / w_vc of layer %d is NULL although d_ctx > 0", l);
     }
     auto cp = [&](void *dst, const void *src, size_t bytes) {
         return async ? cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDefault, st) : cudaMemcpy(dst, src, bytes, cudaMemcpyDefault);
@@ -319,6 +342,8 @@ ebrl_status_t upload_weight_set(ebrl_actgen *h, WeightSet &ws, const ebrl_actgen
         if (e == cudaSuccess) e = cp(o.w_oc, w.w_oc, d * d * esz);
         if (e == cudaSuccess) e = cp(o.w_1, w.w_1, md * d * esz);
         if (e == cudaSuccess) e = cp(o.w_2, w.w_2, d * md * esz);
+        if (e == cudaSuccess && c.d_ctx > 0) e = cp(o.w_kc, w.w_kc, d * (size_t)c.d_ctx * esz);
+        if (e == cudaSuccess && c.d_ctx > 0) e = cp(o.w_vc, w.w_vc, d * (size_t)c.d_ctx * esz);
     }
     if (e != cudaSuccess) return fail(h, EBRL_ERR_CUDA, "copying the weights failed: %s", cudaGetErrorString(e));
     return EBRL_OK;
@@ -384,6 +409,20 @@ cudaError_t launch_attn(ebrl_actgen *h, const AttnArgs &a, int grid, cudaStream_
     return launch_attn_simt(a, h->bf16, grid, st);
 }
 
+// Tile shape of a tensor-core GEMM by estimated time = waves x tile area / relative efficiency:
+// 2 = CTA pairs (256 x 256), 256 = one CTA 128 x 256, 128 = one CTA 128 x 128.  The accumulation
+// order per output element is the same for every shape, so the choice does not change a single
+// bit of the result.
+int pick_tile_shape(const ebrl_actgen *h, long M, int N, int grid)
+{
+    if (h->force_shape) return h->force_shape;
+    const long mt = (M + 127) / 128, mp = (M + 255) / 256, pairs = grid / 2;
+    const double t_pair = (h->use_pairs && pairs >= 1) ? (double)((mp * (N / 256) + pairs - 1) / pairs) * 32768.0 / 1.0 : 1e30;
+    const double t_256 = (double)((mt * (N / 256) + grid - 1) / grid) * 32768.0 / 0.88;
+    const double t_128 = (double)((mt * (N / 128) + grid - 1) / grid) * 16384.0 / 0.72;
+    return (t_pair <= t_256 && t_pair <= t_128) ? 2 : (t_256 <= t_128 ? 256 : 128);
+}
+
 // Enqueues every kernel of one batch (the groups coalesced in one slot) on the stream.
 cudaError_t enqueue_batch(ebrl_actgen *h, Slot &s, int S, const int32_t *n_active, const double *sum_P_active, int grid,
                           cudaStream_t st)
@@ -395,6 +434,32 @@ cudaError_t enqueue_batch(ebrl_actgen *h, Slot &s, int S, const int32_t *n_activ
     const double esz = (double)h->esz;
     Launcher ln{h, &s, st, grid, (c.flags & EBRL_FLAG_TIMING) != 0};
     const WeightSet &W = h->wset[h->active];
+    if (c.d_ctx > 0 && !pull && L > 0) {
+        // hidden-state prefixes: gather the batch's hidden rows, then every layer's K and V planes as
+        // two dense GEMMs over all of them (once per batch: the planes do not change over the Euler steps)
+        const int R = s.prefix_rows, dc = c.d_ctx;
+        PackArgs pa{s.meta_d, n_active[0], s.prefix_slices, (int)(dc * h->esz), s.hid_pack};
+        ln.run(EBRL_KC_PREFIX, 0.0, 2.0 * R * dc * esz, [&] { return launch_pack_prefix(pa, grid, st); });
+        for (int l = 0; l < L; ++l)
+            for (int j = 0; j < 2; ++j) {
+                const LayerDev &w = W.layers[l];
+                GemmArgs g{};
+                g.A = s.hid_pack; g.W = j ? w.w_vc : w.w_kc; g.M = R; g.N = d; g.K = dc; g.epi = EPI_SCALE_STORE;
+                g.ssq_in = s.ssq; g.n_ssq = 0; g.inv_d = 0.f; g.eps = 1.f;   // row scale 1 / sqrt(0 + 1) = 1: a plain store
+                g.C = (char *)s.planes + (size_t)(l * 2 + j) * R * d * h->esz;
+                const TensorMap128 &tW = j ? w.t_vc : w.t_kc;
+                const double bytes = ((double)R * dc + (double)d * dc + (double)R * d) * esz, flops = 2.0 * R * d * dc;
+                if (h->use_tc) {
+                    const int shape = pick_tile_shape(h, R, d, grid);
+                    if (shape == 2)
+                        ln.run(EBRL_KC_PREFIX, flops, bytes, [&] { return launch_gemm_tc2(s.t_hid, tW, g, grid, h->wait_ns, h->status_d, st); });
+                    else
+                        ln.run(EBRL_KC_PREFIX, flops, bytes, [&] { return launch_gemm_tc(s.t_hid, tW, g, grid, shape, h->wait_ns, h->status_d, st); });
+                } else {
+                    ln.run(EBRL_KC_PREFIX, flops, bytes, [&] { return launch_gemm_simt(g, bf, grid, st); });
+                }
+            }
+    }
     for (int step = 0; step < S; ++step) {
         const int ne = n_active[step], M = ne * H;
         if (ne == 0) break;
@@ -412,15 +477,7 @@ cudaError_t enqueue_batch(ebrl_actgen *h, Slot &s, int S, const int32_t *n_activ
                     g.C = C; g.x = s.x; g.gain = gain; g.xg = s.xg; g.ssq_out = s.ssq;
                     const double bytes = ((double)M * K + (double)N * K + (double)M * N) * esz + (epi == EPI_RESID ? 8.0 * M * N : 0.0);
                     if (h->use_tc) {
-                        // tile shape by estimated time = waves x tile area / relative efficiency (the
-                        // accumulation order per output element is the same for every shape, so the
-                        // choice does not change a single bit of the result)
-                        const long mt = (M + 127) / 128, mp = (M + 255) / 256;
-                        const long pairs = grid / 2;
-                        const double t_pair = (h->use_pairs && pairs >= 1) ? (double)((mp * (N / 256) + pairs - 1) / pairs) * 32768.0 / 1.0 : 1e30;
-                        const double t_256 = (double)((mt * (N / 256) + grid - 1) / grid) * 32768.0 / 0.88;
-                        const double t_128 = (double)((mt * (N / 128) + grid - 1) / grid) * 16384.0 / 0.72;
-                        const int shape = h->force_shape ? h->force_shape : (t_pair <= t_256 && t_pair <= t_128 ? 2 : (t_256 <= t_128 ? 256 : 128));
+                        const int shape = pick_tile_shape(h, M, N, grid);
                         if (shape == 2)
                             ln.run(EBRL_KC_GEMM, 2.0 * M * N * K, bytes, [&] { return launch_gemm_tc2(tA, tW, g, grid, h->wait_ns, h->status_d, st); });
                         else
@@ -450,6 +507,7 @@ cudaError_t enqueue_batch(ebrl_actgen *h, Slot &s, int S, const int32_t *n_activ
                     a.q = s.qc; a.q_stride = d; a.out = s.att; a.o_stride = d;
                     a.H = H; a.n_heads = c.n_heads; a.hd = h->hd; a.n_envs = ne; a.d = d;
                     a.meta = s.meta_d; a.kv_plane = (c.kv_layers == 1) ? 0 : l; a.self = 0;
+                    a.plane_rows = c.d_ctx > 0 ? s.prefix_rows : 0;
                     a.self_map = s.maps_d; a.kv_maps = s.maps_d + 1;
                     ln.run(EBRL_KC_CROSS_ATTN, 4.0 * H * sum_P_active[step] * d,
                            2.0 * sum_P_active[step] * d * esz + 2.0 * M * d * esz, [&] { return launch_attn(h, a, grid, st); });
@@ -484,16 +542,52 @@ ebrl_status_t flush_slot(ebrl_actgen *h, Slot &s)
     int S = 0;
     std::vector<TensorMap128> maps_packed;
     const bool with_maps = h->use_attn_mma && !(c.flags & EBRL_FLAG_TEST_PULL);
+    const bool hidden = c.d_ctx > 0 && !(c.flags & EBRL_FLAG_TEST_PULL) && c.n_layers > 0;
     if (with_maps) maps_packed.resize(n);
+    long prefix_rows = 0;
+    int longest = 0;
     for (int j = 0; j < n; ++j) {
         const EnvMeta &m = s.pending[order[j]];
         s.meta_h[j] = m;
-        if (with_maps) maps_packed[j] = s.pending_maps[order[j]];
+        if (with_maps && !hidden) maps_packed[j] = s.pending_maps[order[j]];
+        if (hidden) { s.meta_h[j].row0 = (int32_t)prefix_rows; prefix_rows += m.P; longest = std::max(longest, (int)m.P); }
         S = std::max(S, (int)m.nsteps);
         for (int t = 0; t < m.nsteps; ++t) { n_active[t] += 1; sum_P[t] += m.P; }
     }
     s.pending.clear();
     s.pending_maps.clear();
+    if (hidden) {
+        // scratch for the packed hidden rows and the planes projected from them; the slot's previous
+        // batch has been retired, so a grow may free the old buffers
+        if (prefix_rows > (long)INT32_MAX / (2 * c.n_layers)) return fail(h, EBRL_ERR_UNSUPPORTED, "a batch's prefixes hold too many rows");
+        if ((size_t)prefix_rows > s.proj_cap_rows) {
+            if (s.hid_pack) cudaFree(s.hid_pack);
+            if (s.planes) cudaFree(s.planes);
+            s.hid_pack = s.planes = nullptr; s.proj_cap_rows = 0;
+            const size_t hb = (size_t)prefix_rows * c.d_ctx * h->esz, pb = (size_t)c.n_layers * 2 * prefix_rows * c.d * h->esz;
+            if (cudaMalloc(&s.hid_pack, hb) != cudaSuccess || cudaMalloc(&s.planes, pb) != cudaSuccess) {
+                cudaGetLastError();
+                if (s.hid_pack) cudaFree(s.hid_pack);
+                s.hid_pack = nullptr;
+                for (int64_t id : s.ids) h->busy_ids.erase(id);   // the batch is dropped: nothing of it was enqueued
+                s.ids.clear(); s.copies_out.clear(); s.groups_pending = 0;
+                return fail(h, EBRL_ERR_NOMEM, "projected prefix planes of %ld rows (%zu bytes) do not fit on the device", prefix_rows, hb + pb);
+            }
+            s.proj_cap_rows = (size_t)prefix_rows;
+        }
+        s.prefix_rows = (int)prefix_rows;
+        s.prefix_slices = (longest + 63) / 64;
+        for (int j = 0; j < n; ++j) {
+            EnvMeta &m = s.meta_h[j];
+            m.hid = m.kv;
+            m.kv = (const char *)s.planes + (size_t)m.row0 * c.d * h->esz;
+            // the environment's view of the planes: from its first row to the end of the last plane
+            if (with_maps && attn_mma_make_map(&maps_packed[j], m.kv, (uint64_t)2 * c.n_layers * prefix_rows - m.row0, c.d, c.n_heads, h->hd))
+                return fail(h, EBRL_ERR_CUDA, "cuTensorMapEncodeTiled failed for projected prefix planes");
+        }
+        if (h->use_tc && make_tmap_bf16(&s.t_hid, s.hid_pack, (uint64_t)c.d_ctx, (uint64_t)prefix_rows, (uint32_t)gemm_tc_box_rows_a()))
+            return fail(h, EBRL_ERR_CUDA, "cuTensorMapEncodeTiled failed for the packed hidden states");
+    }
     // SM partition: the batch runs on the partition's stream, fenced against the caller's stream by events
     cudaStream_t user = cs;
     GreenPartition *gp = nullptr;
@@ -581,6 +675,10 @@ ebrl_status_t submit_impl(ebrl_actgen *h, int32_t n, const int64_t *env_ids, con
     const size_t chunk = (size_t)c.H * c.A;
     const int K = c.K_steps;
 
+    // bytes of one environment's prefix as the caller hands it over: its planes, or its hidden states
+    auto prefix_bytes = [&](int P) {
+        return c.d_ctx > 0 ? (size_t)P * c.d_ctx * h->esz : (size_t)c.kv_layers * 2 * P * c.d * h->esz;
+    };
     const float *noise_d = noise;
     float *out_d = out;
     std::vector<const void *> kv_dev(n, nullptr);
@@ -591,7 +689,7 @@ ebrl_status_t submit_impl(ebrl_actgen *h, int32_t n, const int64_t *env_ids, con
         for (int i = 0; i < n; ++i) {
             const int P = (ext && ext->prefix_len) ? ext->prefix_len[i] : c.max_prefix_len;
             off[i] = need;
-            need += ((size_t)c.kv_layers * 2 * P * c.d * h->esz + 255) & ~(size_t)255;
+            need += (prefix_bytes(P) + 255) & ~(size_t)255;
         }
         if (!pull && s.stage_used != 0 && s.kv_stage_bytes < need) {
             // staging already referenced by queued groups: close the batch first, and remember how much
@@ -627,7 +725,7 @@ ebrl_status_t submit_impl(ebrl_actgen *h, int32_t n, const int64_t *env_ids, con
         if (!pull)
             for (int i = 0; i < n; ++i) {
                 const int P = (ext && ext->prefix_len) ? ext->prefix_len[i] : c.max_prefix_len;
-                CK(cudaMemcpyAsync(s.kv_stage + off[i], prefix_kv[i], (size_t)c.kv_layers * 2 * P * c.d * h->esz, cudaMemcpyHostToDevice, h->copy_stream));
+                CK(cudaMemcpyAsync(s.kv_stage + off[i], prefix_kv[i], prefix_bytes(P), cudaMemcpyHostToDevice, h->copy_stream));
                 kv_dev[i] = s.kv_stage + off[i];
             }
         s.stage_used = need;
@@ -643,7 +741,7 @@ ebrl_status_t submit_impl(ebrl_actgen *h, int32_t n, const int64_t *env_ids, con
 
     // descriptors of the group's planes first: a failure must leave nothing of the group queued
     std::vector<TensorMap128> group_maps;
-    if (h->use_attn_mma && !pull) {
+    if (h->use_attn_mma && !pull && c.d_ctx == 0) {   // (projected planes get theirs when the batch is launched)
         group_maps.resize(n);
         for (int i = 0; i < n; ++i) {
             const int P = (ext && ext->prefix_len) ? ext->prefix_len[i] : c.max_prefix_len;
@@ -691,6 +789,8 @@ void free_all(ebrl_actgen *h)
         if (s.meta_h) cudaFreeHost(s.meta_h);
         if (s.maps_h) cudaFreeHost(s.maps_h);
         if (s.kv_stage) cudaFree(s.kv_stage);
+        if (s.hid_pack) cudaFree(s.hid_pack);
+        if (s.planes) cudaFree(s.planes);
         for (TimedLaunch &t : s.timed) { if (t.t0) cudaEventDestroy(t.t0); if (t.t1) cudaEventDestroy(t.t1); }
     }
     for (WeightSet &ws : h->wset) {
@@ -714,6 +814,18 @@ void free_all(ebrl_actgen *h)
 extern "C" {
 
 uint32_t ebrl_actgen_abi_version(void) { return EBRL_ACTGEN_ABI_VERSION; }
+
+uint64_t ebrl_actgen_struct_size(int32_t which)
+{
+    switch (which) {
+    case 0: return sizeof(ebrl_actgen_cfg_t);
+    case 1: return sizeof(ebrl_layer_weights_t);
+    case 2: return sizeof(ebrl_actgen_weights_t);
+    case 3: return sizeof(ebrl_submit_ext_t);
+    case 4: return sizeof(ebrl_actgen_stats_t);
+    default: return 0;
+    }
+}
 
 // Host-only checks, exported so that the argument rules can be tested without a device.
 ebrl_status_t ebrl_actgen_check_cfg(const ebrl_actgen_cfg_t *cfg)

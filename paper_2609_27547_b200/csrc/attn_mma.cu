@@ -112,7 +112,8 @@ __global__ void __launch_bounds__(THREADS, 1) attn_mma_kernel(AttnArgs a, int hp
                 kgrp = (a.d + slab * W) / 64; vgrp = (2 * a.d + slab * W) / 64;
             } else {
                 tm = a.kv_maps + env; P = a.meta[env].P;
-                krow = a.kv_plane * 2 * P; vrow = krow + P;
+                const int pr = a.plane_rows ? a.plane_rows : P;
+                krow = a.kv_plane * 2 * pr; vrow = krow + pr;
                 kgrp = vgrp = slab * G;
             }
         };

@@ -335,8 +335,9 @@ __global__ void __launch_bounds__(512) attn_simt_kernel(AttnArgs a)
         } else {
             const EnvMeta m = a.meta[env];
             P = m.P; kvs = a.d;
-            kbase = (const T *)m.kv + (size_t)a.kv_plane * 2 * P * a.d + h * hd;
-            vbase = kbase + (size_t)P * a.d;
+            const int pr = a.plane_rows ? a.plane_rows : P;
+            kbase = (const T *)m.kv + (size_t)a.kv_plane * 2 * pr * a.d + h * hd;
+            vbase = kbase + (size_t)pr * a.d;
         }
         const T *qg = (const T *)a.q + (size_t)env * H * a.q_stride + h * hd;
         for (int e = t; e < H * hd; e += 128) {
@@ -441,6 +442,33 @@ static cudaError_t embed_dispatch(const EmbedArgs &a, int g, size_t smem, cudaSt
     if (a.A <= 8) return embed_launch<T, 8>(a, g, smem, st);
     if (a.A <= 16) return embed_launch<T, 16>(a, g, smem, st);
     return embed_launch<T, 32>(a, g, smem, st);
+}
+
+// Hidden-state prefixes: copy every environment's [P][d_ctx] rows to its place in the packed matrix.
+// Items are (environment, 64-row slice) over a fixed number of slices per environment (the longest
+// prefix of the batch); slices past an environment's own length are skipped.
+__global__ void __launch_bounds__(512) pack_prefix_kernel(PackArgs a)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    const int vec_per_row = a.row_bytes >> 4;
+    const int items = a.n_envs * a.slices;
+    for (int item = blockIdx.x; item < items; item += gridDim.x) {
+        const int env = item / a.slices, r0 = (item - env * a.slices) << 6;
+        const EnvMeta m = a.meta[env];
+        if (r0 >= m.P) continue;
+        const int nr = min(64, m.P - r0);
+        const uint4 *src = reinterpret_cast<const uint4 *>((const char *)m.hid + (size_t)r0 * a.row_bytes);
+        uint4 *dst = reinterpret_cast<uint4 *>((char *)a.dst + (size_t)(m.row0 + r0) * a.row_bytes);
+        const int nvec = nr * vec_per_row;
+        for (int v = threadIdx.x; v < nvec; v += blockDim.x) dst[v] = src[v];
+    }
+}
+
+cudaError_t launch_pack_prefix(const PackArgs &a, int grid, cudaStream_t st)
+{
+    if (a.n_envs == 0) return cudaSuccess;
+    return launch_kernel(pack_prefix_kernel, grid, 512, 0, st, 1, a);
 }
 
 cudaError_t launch_embed(const EmbedArgs &a, int bf16, int grid, cudaStream_t st)

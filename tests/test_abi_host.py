@@ -36,9 +36,13 @@ def test_library_exports_every_declared_symbol():
 
 
 def test_struct_sizes_match_the_header_layout():
-    assert C.sizeof(B.Cfg) == 88
-    assert C.sizeof(B.LayerWeights) == 72 and C.sizeof(B.Weights) == 40 and C.sizeof(B.SubmitExt) == 24
-    assert C.sizeof(B.Stats) == 8 * 4 + 16 + 5 * 8 * 4 + 8
+    assert C.sizeof(B.Cfg) == 96
+    assert C.sizeof(B.LayerWeights) == 88 and C.sizeof(B.Weights) == 40 and C.sizeof(B.SubmitExt) == 24
+    assert C.sizeof(B.Stats) == 8 * 4 + 16 + 6 * 8 * 4 + 8
+    # and the library, as compiled from the header, agrees with the hand-written mirrors
+    for which, mirror in enumerate((B.Cfg, B.LayerWeights, B.Weights, B.SubmitExt, B.Stats)):
+        assert B.lib().ebrl_actgen_struct_size(which) == C.sizeof(mirror), mirror.__name__
+    assert B.lib().ebrl_actgen_struct_size(5) == 0
 
 
 def _cfg(**kw):
@@ -58,6 +62,9 @@ def _cfg(**kw):
     ({"d": 192, "n_heads": 3}, B.ERR_UNSUPPORTED),   # d not a multiple of 128
     ({"n_heads": 1}, B.ERR_UNSUPPORTED),             # head_dim 256
     ({"n_layers": 0}, B.OK),
+    ({"d_ctx": 128}, B.OK),                          # hidden-state prefixes (make_cfg sets kv_layers = n_layers)
+    ({"d_ctx": 100}, B.ERR_UNSUPPORTED),             # not a multiple of 64
+    ({"d_ctx": -64}, B.ERR_INVALID_ARG),
 ])
 def test_check_cfg(kw, status):
     assert B.lib().ebrl_actgen_check_cfg(C.byref(_cfg(**kw))) == status
