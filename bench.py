@@ -73,13 +73,15 @@ def parse_args():
                     help="event-driven rollout with a synthetic simulator-latency model: chunk latency avg/P50/P99 under "
                          "group-level batching and under step-level continuous batching")
     ap.add_argument("--min-warmup", type=int, default=3, help="lower bound on warm-up steps (profiling captures use 1)")
+    ap.add_argument("--d-ctx", type=int, default=0, help="variant: prefixes are hidden states [P][d_ctx], projected to K/V per layer")
     ap.add_argument("--inflight", type=int, default=16, help="groups queued before a batch is launched")
     return ap.parse_args()
 
 
 def workload_flops(w, envs) -> float:
     """Algorithmic 2mnk FLOPs of one step (every environment from its step index to K)."""
-    return sum(w.flops_per_env_step(e.P) * (w.K - e.step) for e in envs)
+    proj = 4.0 * w.L * w.d * w.d_ctx   # hidden-state prefixes: K and V projections of one prefix row, once per chunk
+    return sum(w.flops_per_env_step(e.P) * (w.K - e.step) + proj * e.P for e in envs)
 
 
 # ------------------------------------------------------------------------------------------------
@@ -219,6 +221,8 @@ def run_ours(args):
     w = synth.WORKLOADS[args.config]
     if args.envs:
         w = synth.scaled(w, B=args.envs)
+    if args.d_ctx:
+        w = synth.scaled(w, d_ctx=args.d_ctx, name=w.name + "_hidden%d" % args.d_ctx)
     seed = args.seed or synth.DEFAULT_SEED
     quota = w.quota if args.quota < 0 else args.quota
     q_eff = quota if quota > 0 else N_SMS
@@ -368,7 +372,7 @@ def run_ours(args):
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16" if bf16 else "f32", "data": "synthetic",
             "config": {"workload": "configs[%d] %s" % (args.config, w.name), "envs_per_gpu": w.B, "H": w.H, "A": w.A, "d": w.d,
-                       "L": w.L, "heads": w.n_heads, "P": list(w.P), "K": w.K, "groups": len(groups),
+                       "L": w.L, "heads": w.n_heads, "P": list(w.P), "K": w.K, "d_ctx": w.d_ctx, "groups": len(groups),
                        "group_sizes": [min(map(len, groups)), max(map(len, groups))], "sm_quota": q_eff,
                        "inflight_groups": inflight, "corunner": bool(co_stream is not None),
                        "green_ctx": {"requested": bool(args.green_ctx), "active": bool(st0["green_ctx_active"]), "partition_sms": st0["green_ctx_sms"]},
