@@ -65,6 +65,19 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const void *tmap, uint
                  ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
 
+// 4 x 4 transpose of 32-bit words across the four lanes of a quad: on return r[c] of lane t holds what
+// lane c had in r[t].
+__device__ __forceinline__ void quad_transpose(uint32_t (&r)[4], int t)
+{
+    const bool odd = t & 1, hi = t & 2;
+    uint32_t x = __shfl_xor_sync(0xffffffffu, odd ? r[0] : r[1], 1);
+    uint32_t y = __shfl_xor_sync(0xffffffffu, odd ? r[2] : r[3], 1);
+    if (odd) { r[0] = x; r[2] = y; } else { r[1] = x; r[3] = y; }
+    x = __shfl_xor_sync(0xffffffffu, hi ? r[0] : r[2], 2);
+    y = __shfl_xor_sync(0xffffffffu, hi ? r[1] : r[3], 2);
+    if (hi) { r[0] = x; r[1] = y; } else { r[2] = x; r[3] = y; }
+}
+
 template <int HD>
 __global__ void __launch_bounds__(THREADS, 1) attn_mma_kernel(AttnArgs a, int hpc, int la_blocks, unsigned long long limit_ns, int *status)
 {
@@ -302,11 +315,22 @@ __global__ void __launch_bounds__(THREADS, 1) attn_mma_kernel(AttnArgs a, int hp
             l0 += __shfl_xor_sync(0xffffffffu, l0, 1); l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
             l1 += __shfl_xor_sync(0xffffffffu, l1, 1); l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
             const float i0 = 1.0f / l0, i1 = 1.0f / l1;
-            __nv_bfloat16 *ob = (__nv_bfloat16 *)a.out + (size_t)env * H * a.o_stride + head * HD + 2 * t;
+            // The accumulator fragment gives a lane two adjacent columns of each 8-column tile.  Four tiles
+            // at a time are transposed across the quad (lane t ends up with all 8 columns of tile 4 j + t),
+            // so that a lane stores 16 contiguous bytes and a warp instruction fills whole 32-byte sectors.
+            __nv_bfloat16 *ob = (__nv_bfloat16 *)a.out + (size_t)env * H * a.o_stride + head * HD + 8 * t;
 #pragma unroll
-            for (int n = 0; n < HD / 8; ++n) {
-                if (g < H) *reinterpret_cast<uint32_t *>(ob + (size_t)g * a.o_stride + n * 8) = pack2(o[n][0] * i0, o[n][1] * i0);
-                if (g + 8 < H) *reinterpret_cast<uint32_t *>(ob + (size_t)(g + 8) * a.o_stride + n * 8) = pack2(o[n][2] * i1, o[n][3] * i1);
+            for (int j = 0; j < HD / 32; ++j) {
+                uint32_t r0[4], r1[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    r0[k] = pack2(o[4 * j + k][0] * i0, o[4 * j + k][1] * i0);
+                    r1[k] = pack2(o[4 * j + k][2] * i1, o[4 * j + k][3] * i1);
+                }
+                quad_transpose(r0, t);
+                quad_transpose(r1, t);
+                if (g < H) *reinterpret_cast<uint4 *>(ob + (size_t)g * a.o_stride + j * 32) = make_uint4(r0[0], r0[1], r0[2], r0[3]);
+                if (g + 8 < H) *reinterpret_cast<uint4 *>(ob + (size_t)(g + 8) * a.o_stride + j * 32) = make_uint4(r1[0], r1[1], r1[2], r1[3]);
             }
         }
     }
