@@ -306,8 +306,18 @@ def run_ours(args):
         peak_note = "fp32 FFMA 148 SMs x 128 lanes x 2 x 1.965 GHz = %.1f TFLOP/s x quota %d/%d" % (FP32_ALU_TFLOPS, q_eff, N_SMS)
         bound = "alu"
     achieved = gemm["flops"] / (gemm["ms"] * 1e-3) / 1e12 if gemm["ms"] > 0 else 0.0
+    # DRAM traffic per GEMM launch from the ncu capture of one layer of this model at M = 8192 rows
+    # (profiles/gemm_tc2_cfg4_512env.md): 0.117 GB of weights per layer, which do not grow with M, plus
+    # 0.971 GB of activations, which grow in proportion to the rows; six launches per layer.
+    traffic, traffic_note = None, None
+    if bf16 and (w.d, w.L, w.H, w.mlp_mult) == (2048, 8, 16, 4) and gemm["launches"] > 0:
+        rows_per_launch = st["env_steps"] * w.H / (gemm["launches"] / 6.0 / w.L)
+        traffic = (0.117e9 + 0.971e9 * rows_per_launch / 8192.0) / 6.0
+        traffic_note = "bytes per launch, ncu capture at M=8192 scaled to M=%d (activation part in proportion)" % round(rows_per_launch)
     roofline = {"bound": bound, "kernel": "gemm", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                "frac": achieved / peak if peak else None, "traffic": None, "peak_source": peak_note,
+                "frac": achieved / peak if peak else None, "traffic": traffic, "traffic_note": traffic_note,
+                "algorithmic_bytes_per_launch": gemm["bytes"] / gemm["launches"] if gemm["launches"] else None,
+                "peak_source": peak_note,
                 "launches": gemm["launches"], "avg_launch_us": 1e3 * gemm["ms"] / max(1, gemm["launches"]),
                 "class_share": {k: round(c["ms"] / total_ms, 4) for k, c in cls.items()},
                 "class_ms_per_step": {k: round(c["ms"] / args.steps, 4) for k, c in cls.items()}}
