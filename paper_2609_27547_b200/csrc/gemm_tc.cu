@@ -110,52 +110,55 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     pdl_wait();   // set-up done; from here on the previous kernel's results are needed
 
     if (warp == 0) {
-        // ---- TMA producer
-        int stage = 0;
-        uint32_t phase = 0;
-        for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
-            const int m0 = (tile / ntn) * BM, n0 = (tile % ntn) * BN;
-            for (int kb = 0; kb < nkb; ++kb) {
-                if (!__all_sync(0xffffffffu, mbar_wait_relaxed(empty(stage), phase ^ 1u, limit_ns, abort_flag))) { ok = false; break; }
-                if (lane == 0) {
+        // ---- TMA producer: one thread (no votes, fewer instructions between a free stage and its next copies)
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
+                const int m0 = (tile / ntn) * BM, n0 = (tile % ntn) * BN;
+                for (int kb = 0; kb < nkb; ++kb) {
+                    if (!mbar_wait_relaxed(empty(stage), phase ^ 1u, limit_ns, abort_flag)) { ok = false; break; }
                     mbar_expect_tx(full(stage), A_BYTES + B_BYTES);
                     tma_load_2d(sA + stage * A_BYTES, &tmA, full(stage), kb * BK, m0);
                     tma_load_2d(sB + stage * B_BYTES, &tmB, full(stage), kb * BK, n0);   // weight rows n0 .. n0+127 (128-row boxes)
                     if (BN == 256) tma_load_2d(sB + stage * B_BYTES + B_BYTES / 2, &tmB, full(stage), kb * BK, n0 + 128);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
-                __syncwarp();
-                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
             }
         }
+        __syncwarp();
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
     } else if (warp == 1) {
-        // ---- MMA issuer
-        constexpr uint32_t idesc = instr_desc(BM, BN);
-        int stage = 0, it = 0;
-        uint32_t phase = 0;
-        for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++it) {
-            const int buf = it & 1;
-            const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
-            if (!__all_sync(0xffffffffu, mbar_wait(tempty(buf), acc_phase ^ 1u, limit_ns, abort_flag))) { ok = false; break; }
-            tc_fence_after();
-            const uint32_t d_tmem = tmem_base + (uint32_t)buf * BN;
-            for (int kb = 0; kb < nkb; ++kb) {
-                if (!__all_sync(0xffffffffu, mbar_wait(full(stage), phase, limit_ns, abort_flag))) { ok = false; break; }
+        // ---- MMA issuer: one thread
+        if (lane == 0) {
+            constexpr uint32_t idesc = instr_desc(BM, BN);
+            const uint64_t ad0 = smem_desc(sA), bd0 = smem_desc(sB);
+            int stage = 0, it = 0;
+            uint32_t phase = 0;
+            for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++it) {
+                const int buf = it & 1;
+                const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+                if (!mbar_wait(tempty(buf), acc_phase ^ 1u, limit_ns, abort_flag)) { ok = false; break; }
                 tc_fence_after();
-                if (lane == 0) {
-                    const uint64_t ad = smem_desc(sA + stage * A_BYTES), bd = smem_desc(sB + stage * B_BYTES);
+                const uint32_t d_tmem = tmem_base + (uint32_t)buf * BN;
+                for (int kb = 0; kb < nkb; ++kb) {
+                    if (!mbar_wait(full(stage), phase, limit_ns, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    // descriptors advance by whole stages and by 32 bytes per 16-wide k-slice (address field in 16-byte units)
+                    const uint64_t ad = ad0 + (uint64_t)(stage * (A_BYTES >> 4)), bd = bd0 + (uint64_t)(stage * (B_BYTES >> 4));
+                    tc_mma(d_tmem, ad, bd, idesc, kb != 0 ? 1u : 0u);
 #pragma unroll
-                    for (int k = 0; k < BK / UMMA_K; ++k)
-                        tc_mma(d_tmem, ad + (uint64_t)(k * UMMA_K * 2 / 16), bd + (uint64_t)(k * UMMA_K * 2 / 16), idesc,
-                               (kb | k) != 0 ? 1u : 0u);
+                    for (int k = 1; k < BK / UMMA_K; ++k)
+                        tc_mma(d_tmem, ad + (uint64_t)(k * UMMA_K * 2 / 16), bd + (uint64_t)(k * UMMA_K * 2 / 16), idesc, 1u);
                     tc_commit(empty(stage));
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
-                __syncwarp();
-                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                if (!ok) break;
+                tc_commit(tfull(buf));
             }
-            if (!ok) break;
-            if (lane == 0) tc_commit(tfull(buf));
-            __syncwarp();
         }
+        __syncwarp();
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
     } else {
         // ---- epilogue: warp w reads TMEM lanes 32 (w % 4) .. +31 and half of the tile's columns; one thread per row
         const int q = warp & 3, half = (warp - 2) >> 2;   // half is 0 for the 128-column shape
