@@ -254,7 +254,12 @@ __global__ void __launch_bounds__(THREADS, 1) attn_mma_kernel(AttnArgs a, int hp
             auto wait_block = [&](int b) -> bool {   // first block of a stage: wait until the copies have landed
                 if (b & bps_mask) return true;
                 const int qs = qbase + (b >> bps_sh);
-                return __all_sync(0xffffffffu, mbar_wait(full(qs % NSTAGE), (uint32_t)(qs / NSTAGE) & 1u, limit_ns, abort_flag));
+                // one lane polls the barrier (32 lanes polling the same word are 32 shared-memory operations per
+                // round, beside the copies and the ldmatrix traffic); the warp-level exchange orders the others
+                // behind it.  (The same change in the producer's sleeping wait measured 10 % slower.)
+                int landed = 1;
+                if (lane == 0) landed = mbar_wait(full(qs % NSTAGE), (uint32_t)(qs / NSTAGE) & 1u, limit_ns, abort_flag) ? 1 : 0;
+                return __shfl_sync(0xffffffffu, landed, 0) != 0;
             };
             for (int b = 0; b < nblk; ++b) {
                 // A block's Q K^T is issued when its stage is needed, not a block early: touching the next
