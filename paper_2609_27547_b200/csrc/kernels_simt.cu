@@ -138,24 +138,42 @@ __global__ void __launch_bounds__(HEAD_WARPS * 32) head_kernel(HeadArgs a)
             for (int j = 0; j < AMAX; ++j) acc[r][j] = 0.f;
         float ss[2] = {0.f, 0.f};
         if (!a.pull) {
-            for (int c = lane * 4; c < a.d; c += 128) {
-                const float4 gv = *reinterpret_cast<const float4 *>(a.gain + c);
-                float t[2][4];
+            // four 128-column steps per round: the eight row loads of a round are in flight together (one
+            // step at a time left a warp with two loads in flight and the kernel waiting on memory latency)
+            for (int c0 = lane * 4; c0 < a.d; c0 += 512) {
+                float4 xv[4][2], gv[4];
 #pragma unroll
-                for (int r = 0; r < 2; ++r) {
-                    const float4 xv = *reinterpret_cast<const float4 *>(a.x + (size_t)(row0 + (r < nr ? r : 0)) * a.d + c);
-                    ss[r] = fmaf(xv.x, xv.x, ss[r]); ss[r] = fmaf(xv.y, xv.y, ss[r]);
-                    ss[r] = fmaf(xv.z, xv.z, ss[r]); ss[r] = fmaf(xv.w, xv.w, ss[r]);
-                    t[r][0] = xv.x * gv.x; t[r][1] = xv.y * gv.y; t[r][2] = xv.z * gv.z; t[r][3] = xv.w * gv.w;
+                for (int u = 0; u < 4; ++u) {
+                    const int c = c0 + u * 128;
+                    if (c < a.d) {
+                        gv[u] = *reinterpret_cast<const float4 *>(a.gain + c);
+#pragma unroll
+                        for (int r = 0; r < 2; ++r)
+                            xv[u][r] = *reinterpret_cast<const float4 *>(a.x + (size_t)(row0 + (r < nr ? r : 0)) * a.d + c);
+                    }
                 }
 #pragma unroll
-                for (int j = 0; j < AMAX; ++j) {
-                    if (j < a.A) {
-                        const float4 w = *reinterpret_cast<const float4 *>(wO + j * a.d + c);
+                for (int u = 0; u < 4; ++u) {
+                    const int c = c0 + u * 128;
+                    if (c < a.d) {
+                        float t[2][4];
 #pragma unroll
                         for (int r = 0; r < 2; ++r) {
-                            acc[r][j] = fmaf(t[r][0], w.x, acc[r][j]); acc[r][j] = fmaf(t[r][1], w.y, acc[r][j]);
-                            acc[r][j] = fmaf(t[r][2], w.z, acc[r][j]); acc[r][j] = fmaf(t[r][3], w.w, acc[r][j]);
+                            const float4 x4 = xv[u][r];
+                            ss[r] = fmaf(x4.x, x4.x, ss[r]); ss[r] = fmaf(x4.y, x4.y, ss[r]);
+                            ss[r] = fmaf(x4.z, x4.z, ss[r]); ss[r] = fmaf(x4.w, x4.w, ss[r]);
+                            t[r][0] = x4.x * gv[u].x; t[r][1] = x4.y * gv[u].y; t[r][2] = x4.z * gv[u].z; t[r][3] = x4.w * gv[u].w;
+                        }
+#pragma unroll
+                        for (int j = 0; j < AMAX; ++j) {
+                            if (j < a.A) {
+                                const float4 w = *reinterpret_cast<const float4 *>(wO + j * a.d + c);
+#pragma unroll
+                                for (int r = 0; r < 2; ++r) {
+                                    acc[r][j] = fmaf(t[r][0], w.x, acc[r][j]); acc[r][j] = fmaf(t[r][1], w.y, acc[r][j]);
+                                    acc[r][j] = fmaf(t[r][2], w.z, acc[r][j]); acc[r][j] = fmaf(t[r][3], w.w, acc[r][j]);
+                                }
+                            }
                         }
                     }
                 }
