@@ -147,3 +147,35 @@ def test_configuration_errors():
     h = C.c_void_p()
     assert B.lib().ebrl_actgen_create(C.byref(cfg), C.byref(ws), C.byref(h)) == B.ERR_INVALID_ARG
     assert not h.value
+
+
+def test_weight_publication_replaces_the_projections_too():
+    """A published policy version carries its own W_kc / W_vc: batches launched after the update
+    project the prefixes with the new matrices, batches queued before it with the old ones."""
+    w, wA, envs = _case("bf16", 128)
+    wB = synth.make_weights(w, SEED + 7, random_gains=True)
+    ids = list(range(w.B))
+    refs = {}
+    for name, wt in (("A", wA), ("B", wB)):
+        r = Runner(w, wt, envs)
+        refs[name] = stack(r.run([ids]), ids)
+        r.close()
+    only_proj = {**wA, "layers": [{**la, "w_kc": lb["w_kc"], "w_vc": lb["w_vc"]} for la, lb in zip(wA["layers"], wB["layers"])]}
+    r = Runner(w, only_proj, envs)
+    ref_proj = stack(r.run([ids]), ids)
+    r.close()
+    assert not np.array_equal(refs["A"], ref_proj)      # the projections matter on their own
+    r = Runner(w, wA, envs, max_inflight_groups=4)
+    noise = torch.stack([r.noise[e] for e in ids])
+    out1, out2 = torch.empty_like(noise), torch.empty_like(noise)
+    kv = [r.kv[e] for e in ids]
+    sidx = [envs[e].step for e in ids]
+    r.gen.submit(ids[:4], kv[:4], noise[:4], out1[:4], step_index=sidx[:4])      # queued under version 1
+    assert r.gen.update_weights(wB) == 2
+    r.gen.submit([100 + e for e in ids], kv, noise, out2, step_index=sidx)         # runs with version 2
+    r.gen.sync()
+    assert np.array_equal(out1[:4].cpu().numpy(), refs["A"][:4])
+    assert np.array_equal(out2.cpu().numpy(), refs["B"])
+    assert r.gen.update_weights(only_proj) == 3
+    assert np.array_equal(stack(r.run([ids]), ids), ref_proj)
+    r.close()
