@@ -3,6 +3,8 @@
 #pragma once
 #include "actgen_internal.h"
 
+#include <cuda.h>
+
 namespace ebrl {
 namespace tc {
 
@@ -167,6 +169,68 @@ __device__ __forceinline__ bool epilogue_rows(const GemmArgs &g, uint32_t taddr,
         }
     }
     return true;
+}
+
+// EPI_SCALE_STORE / EPI_SCALE_GELU through the copy engine: the thread that owns a row writes its bf16 values
+// as 16-byte pieces into a [32 rows][128 B] staging tile in the 128-byte-swizzle layout (piece p of row r at
+// p ^ (r & 7): conflict-free), and one lane hands the tile to a TMA store, which also clips rows past M.
+// Per 64 columns that is 8 shared stores per thread and one copy instruction per warp, instead of 16 shared
+// stores, 16 shared loads and 16 predicated global stores -- fewer issue slots taken from the single TMA and
+// MMA threads that share the schedulers.  `stg_generic` must be 1024-byte aligned (4 KB).
+template <int EPI, int NCOLS, typename WaitF>
+__device__ __forceinline__ bool epilogue_store_tma(const GemmArgs &g, const CUtensorMap *tmC, uint32_t taddr, int row0, int n0,
+                                                   float *stg_generic, WaitF wait)
+{
+    static_assert(EPI != EPI_RESID && NCOLS % 64 == 0, "bf16 store epilogues only");
+    const int lane = threadIdx.x & 31;
+    const uint32_t stg = (uint32_t)__cvta_generic_to_shared(stg_generic);
+    float rs = 0.f;
+    if (row0 + lane < g.M) {
+        float s = 0.f;
+        const int row = row0 + lane;
+        for (int t = 0; t < g.n_ssq; ++t) s += g.ssq_in[(size_t)row * g.n_ssq + t];
+        rs = 1.0f / sqrtf(s * g.inv_d + g.eps);
+    }
+    if (!wait()) return false;
+    tc_fence_after();
+#pragma unroll 1
+    for (int h = 0; h < NCOLS / 64; ++h) {
+        // the staging tile is free once the previous copy has read it
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        __syncwarp();
+#pragma unroll
+        for (int c = 0; c < 2; ++c) {
+            uint32_t r[32];
+            tc_ld32(taddr + (uint32_t)((h * 2 + c) * 32), r);
+            tc_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                uint32_t w[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    float lo = __uint_as_float(r[8 * j + 2 * e]) * rs, hi = __uint_as_float(r[8 * j + 2 * e + 1]) * rs;
+                    if (EPI == EPI_SCALE_GELU) { lo = gelu_erf(lo); hi = gelu_erf(hi); }
+                    w[e] = pack_bf16(lo, hi);
+                }
+                const int p = c * 4 + j;
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stg + (uint32_t)(lane * 128 + ((p ^ (lane & 7)) << 4))),
+                             "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+            }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes before the copy engine reads them
+        __syncwarp();
+        if (lane == 0 && row0 < g.M) {
+            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                         ::"l"(reinterpret_cast<uint64_t>(tmC)), "r"(n0 + h * 64), "r"(row0), "r"(stg) : "memory");
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        }
+    }
+    return true;
+}
+// Before a warp that used epilogue_store_tma leaves the kernel: its copies must have completed.
+__device__ __forceinline__ void epilogue_store_drain()
+{
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }
 
 }  // namespace tc

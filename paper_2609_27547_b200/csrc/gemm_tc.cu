@@ -70,14 +70,16 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N)
 
 template <int EPI, int BN>
 __global__ void __launch_bounds__(Shape<BN>::THREADS, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmArgs g,
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const __grid_constant__ CUtensorMap tmC, GemmArgs g,
                unsigned long long limit_ns, int *status)
 {
     constexpr int STAGES = Shape<BN>::STAGES, EPI_WARPS = Shape<BN>::EPI_WARPS, B_BYTES = Shape<BN>::B_BYTES;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t sA = smem_u32(smem), sB = sA + STAGES * A_BYTES;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + STAGES * (A_BYTES + B_BYTES));
+    // after the stages: the epilogue warps' staging tiles (4 KB each, 1024-byte aligned), then the barriers
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + STAGES * (A_BYTES + B_BYTES) + EPI_WARPS * EPI_STAGE_FLOATS * 4);
     const uint32_t bar0 = smem_u32(bars);
     auto full = [&](int s) { return bar0 + 8u * s; };
     auto empty = [&](int s) { return bar0 + 8u * (STAGES + s); };
@@ -162,14 +164,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     } else {
         // ---- epilogue: warp w reads TMEM lanes 32 (w % 4) .. +31 and half of the tile's columns; one thread per row
         const int q = warp & 3, half = (warp - 2) >> 2;   // half is 0 for the 128-column shape
-        float *stg = reinterpret_cast<float *>(smem + STAGES * (A_BYTES + B_BYTES) + 256) + (warp - 2) * EPI_STAGE_FLOATS;
+        float *stg = reinterpret_cast<float *>(smem + STAGES * (A_BYTES + B_BYTES)) + (warp - 2) * EPI_STAGE_FLOATS;
         int it = 0;
         for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++it) {
             const int buf = it & 1;
             const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
             const int m0 = (tile / ntn) * BM, n0 = (tile % ntn) * BN + half * 128;
-            if (!epilogue_rows<EPI, 128>(g, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + half * 128), m0 + q * 32, n0, stg,
-                                            [&] { return __all_sync(0xffffffffu, mbar_wait_relaxed(tfull(buf), acc_phase, limit_ns, abort_flag)) != 0; })) {
+            auto acc_ready = [&] { return __all_sync(0xffffffffu, mbar_wait_relaxed(tfull(buf), acc_phase, limit_ns, abort_flag)) != 0; };
+            const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + half * 128);
+            bool done;
+            if constexpr (EPI == EPI_RESID) done = epilogue_rows<EPI, 128>(g, tacc, m0 + q * 32, n0, stg, acc_ready);
+            else done = epilogue_store_tma<EPI, 128>(g, &tmC, tacc, m0 + q * 32, n0, stg, acc_ready);
+            if (!done) {
                 ok = false;
                 break;
             }
@@ -177,6 +183,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty(buf));
         }
+        if (EPI != EPI_RESID && lane == 0) epilogue_store_drain();
     }
 
     // ---- teardown
@@ -239,8 +246,8 @@ int gemm_tc_box_rows_a() { return tc::BM; }
 int gemm_tc_box_rows_w() { return 128; }   // weight maps serve every kernel: 128-row boxes
 
 template <int EPI, int BN>
-static cudaError_t tc_launch(const TensorMap128 &ta, const TensorMap128 &tw, const GemmArgs &a, int g, unsigned long long limit_ns,
-                             int *status, cudaStream_t st)
+static cudaError_t tc_launch(const TensorMap128 &ta, const TensorMap128 &tw, const TensorMap128 &tc_, const GemmArgs &a, int g,
+                             unsigned long long limit_ns, int *status, cudaStream_t st)
 {
     static bool attr_set = false;
     if (!attr_set) {
@@ -249,7 +256,8 @@ static cudaError_t tc_launch(const TensorMap128 &ta, const TensorMap128 &tw, con
         attr_set = true;
     }
     return launch_kernel(tc::gemm_tc_kernel<EPI, BN>, g, tc::Shape<BN>::THREADS, tc::Shape<BN>::SMEM_BYTES, st, 1,
-                         *reinterpret_cast<const CUtensorMap *>(&ta), *reinterpret_cast<const CUtensorMap *>(&tw), a, limit_ns, status);
+                         *reinterpret_cast<const CUtensorMap *>(&ta), *reinterpret_cast<const CUtensorMap *>(&tw),
+                         *reinterpret_cast<const CUtensorMap *>(&tc_), a, limit_ns, status);
 }
 
 // One CTA per tile; bn = 256 or 128 columns per tile.
@@ -257,19 +265,22 @@ cudaError_t launch_gemm_tc(const TensorMap128 &ta, const TensorMap128 &tw, const
                            int *status, cudaStream_t st)
 {
     if (a.M == 0) return cudaSuccess;
+    // the store epilogues write C through the copy engine: a descriptor of C as [M][N], boxes of 32 rows x 64 columns
+    TensorMap128 tcm = ta;
+    if (a.epi != EPI_RESID && make_tmap_bf16(&tcm, a.C, (uint64_t)a.N, (uint64_t)a.M, 32)) return cudaErrorInvalidValue;
     const int tiles = ((a.M + tc::BM - 1) / tc::BM) * (a.N / bn);
     const int g = tiles < grid ? tiles : grid;
     if (bn == 256) {
         switch (a.epi) {
-        case EPI_SCALE_STORE: return tc_launch<EPI_SCALE_STORE, 256>(ta, tw, a, g, limit_ns, status, st);
-        case EPI_SCALE_GELU: return tc_launch<EPI_SCALE_GELU, 256>(ta, tw, a, g, limit_ns, status, st);
-        default: return tc_launch<EPI_RESID, 256>(ta, tw, a, g, limit_ns, status, st);
+        case EPI_SCALE_STORE: return tc_launch<EPI_SCALE_STORE, 256>(ta, tw, tcm, a, g, limit_ns, status, st);
+        case EPI_SCALE_GELU: return tc_launch<EPI_SCALE_GELU, 256>(ta, tw, tcm, a, g, limit_ns, status, st);
+        default: return tc_launch<EPI_RESID, 256>(ta, tw, tcm, a, g, limit_ns, status, st);
         }
     }
     switch (a.epi) {
-    case EPI_SCALE_STORE: return tc_launch<EPI_SCALE_STORE, 128>(ta, tw, a, g, limit_ns, status, st);
-    case EPI_SCALE_GELU: return tc_launch<EPI_SCALE_GELU, 128>(ta, tw, a, g, limit_ns, status, st);
-    default: return tc_launch<EPI_RESID, 128>(ta, tw, a, g, limit_ns, status, st);
+    case EPI_SCALE_STORE: return tc_launch<EPI_SCALE_STORE, 128>(ta, tw, tcm, a, g, limit_ns, status, st);
+    case EPI_SCALE_GELU: return tc_launch<EPI_SCALE_GELU, 128>(ta, tw, tcm, a, g, limit_ns, status, st);
+    default: return tc_launch<EPI_RESID, 128>(ta, tw, tcm, a, g, limit_ns, status, st);
     }
 }
 

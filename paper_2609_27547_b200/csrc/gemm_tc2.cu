@@ -84,7 +84,8 @@ __host__ __device__ constexpr uint32_t instr_desc_bf16(int M, int N)
 
 template <int EPI>
 __global__ void __launch_bounds__(THREADS, 1)
-gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmArgs g,
+gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                const __grid_constant__ CUtensorMap tmC, GemmArgs g,
                 unsigned long long limit_ns, int *status)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -92,7 +93,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     // address in every CTA of a kernel, so rounding up gives matching layouts
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t sA = smem_u32(smem), sB = sA + STAGES * A_BYTES;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + STAGES * (A_BYTES + B_BYTES));
+    // after the stages: the epilogue warps' staging tiles (4 KB each, 1024-byte aligned), then the barriers
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + STAGES * (A_BYTES + B_BYTES) + EPI_WARPS * EPI_STAGE_FLOATS * 4);
     const uint32_t bar0 = smem_u32(bars);
     auto full = [&](int s) { return bar0 + 8u * s; };
     auto empty = [&](int s) { return bar0 + 8u * (STAGES + s); };
@@ -182,14 +184,18 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     } else {
         // ---- epilogue (both CTAs): own 128 rows of the pair tile; each warp a lane quarter and half of the columns
         const int q = warp & 3, half = (warp - 2) >> 2;
-        float *stg = reinterpret_cast<float *>(smem + STAGES * (A_BYTES + B_BYTES) + 256) + (warp - 2) * EPI_STAGE_FLOATS;
+        float *stg = reinterpret_cast<float *>(smem + STAGES * (A_BYTES + B_BYTES)) + (warp - 2) * EPI_STAGE_FLOATS;
         int it = 0;
         for (int tile = pair; tile < ntiles && ok; tile += npairs, ++it) {
             const int buf = it & 1;
             const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
             const int m0 = (tile / ntn) * (2 * BM) + (int)rank * BM, n0 = (tile % ntn) * BN + half * (BN / 2);
-            if (!epilogue_rows<EPI, BN / 2>(g, tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + half * (BN / 2)), m0 + q * 32, n0, stg,
-                                            [&] { return __all_sync(0xffffffffu, mbar_wait_relaxed(tfull(buf), acc_phase, limit_ns, abort_flag)) != 0; })) {
+            auto acc_ready = [&] { return __all_sync(0xffffffffu, mbar_wait_relaxed(tfull(buf), acc_phase, limit_ns, abort_flag)) != 0; };
+            const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + half * (BN / 2));
+            bool done;
+            if constexpr (EPI == EPI_RESID) done = epilogue_rows<EPI, BN / 2>(g, tacc, m0 + q * 32, n0, stg, acc_ready);
+            else done = epilogue_store_tma<EPI, BN / 2>(g, &tmC, tacc, m0 + q * 32, n0, stg, acc_ready);
+            if (!done) {
                 ok = false;
                 break;
             }
@@ -197,6 +203,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(mapa(tempty(buf), 0));
         }
+        if (EPI != EPI_RESID && lane == 0) epilogue_store_drain();
     }
 
     // ---- teardown: nobody leaves while its partner may still touch its memory
@@ -221,8 +228,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 }  // namespace tc2
 
 template <int EPI>
-static cudaError_t tc2_launch(const TensorMap128 &ta, const TensorMap128 &tw, const GemmArgs &a, int g, unsigned long long limit_ns,
-                              int *status, cudaStream_t st)
+static cudaError_t tc2_launch(const TensorMap128 &ta, const TensorMap128 &tw, const TensorMap128 &tc_, const GemmArgs &a, int g,
+                              unsigned long long limit_ns, int *status, cudaStream_t st)
 {
     static bool attr_set = false;
     if (!attr_set) {
@@ -231,7 +238,7 @@ static cudaError_t tc2_launch(const TensorMap128 &ta, const TensorMap128 &tw, co
         attr_set = true;
     }
     return launch_kernel(tc2::gemm_tc2_kernel<EPI>, g, tc2::THREADS, tc2::SMEM_BYTES, st, 2, *reinterpret_cast<const CUtensorMap *>(&ta),
-                         *reinterpret_cast<const CUtensorMap *>(&tw), a, limit_ns, status);
+                         *reinterpret_cast<const CUtensorMap *>(&tw), *reinterpret_cast<const CUtensorMap *>(&tc_), a, limit_ns, status);
 }
 
 // grid = SM quota; the kernel uses floor(grid / 2) CTA pairs.  Needs grid >= 2.
@@ -239,14 +246,17 @@ cudaError_t launch_gemm_tc2(const TensorMap128 &ta, const TensorMap128 &tw, cons
                             int *status, cudaStream_t st)
 {
     if (a.M == 0) return cudaSuccess;
+    // the store epilogues write C through the copy engine: a descriptor of C as [M][N], boxes of 32 rows x 64 columns
+    TensorMap128 tcm = ta;
+    if (a.epi != EPI_RESID && make_tmap_bf16(&tcm, a.C, (uint64_t)a.N, (uint64_t)a.M, 32)) return cudaErrorInvalidValue;
     const int tiles = ((a.M + 2 * tc2::BM - 1) / (2 * tc2::BM)) * (a.N / tc2::BN);
     int pairs = grid / 2;
     if (pairs > tiles) pairs = tiles;
     const int g = 2 * pairs;
     switch (a.epi) {
-    case EPI_SCALE_STORE: return tc2_launch<EPI_SCALE_STORE>(ta, tw, a, g, limit_ns, status, st);
-    case EPI_SCALE_GELU: return tc2_launch<EPI_SCALE_GELU>(ta, tw, a, g, limit_ns, status, st);
-    default: return tc2_launch<EPI_RESID>(ta, tw, a, g, limit_ns, status, st);
+    case EPI_SCALE_STORE: return tc2_launch<EPI_SCALE_STORE>(ta, tw, tcm, a, g, limit_ns, status, st);
+    case EPI_SCALE_GELU: return tc2_launch<EPI_SCALE_GELU>(ta, tw, tcm, a, g, limit_ns, status, st);
+    default: return tc2_launch<EPI_RESID>(ta, tw, tcm, a, g, limit_ns, status, st);
     }
 }
 
