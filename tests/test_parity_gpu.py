@@ -437,3 +437,40 @@ def test_queue_semantics_flush_streams_and_timing():
     assert cls["gemm"]["launches"] == 3 * w.K * w.L * 6 and cls["gemm"]["ms"] > 0 and cls["gemm"]["flops"] > 0
     assert cls["cross_attn"]["bytes"] > 0 and cls["head"]["launches"] == 3 * w.K
     r.close()
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_two_handles_share_the_gpu_on_disjoint_quotas(dtype):
+    """Two handles (two policies co-located on one GPU, as the paper's stages are) run at the same
+    time on their own streams under complementary SM quotas; each delivers the bits it delivers alone."""
+    w = synth.scaled(synth.WORKLOADS[0], B=12, dtype=dtype, P=(30, 90), mixed_steps=True)
+    wA = synth.make_weights(w, 11, random_gains=True)
+    wB = synth.make_weights(w, 22, random_gains=True)
+    envs = [synth.make_env(w, e, SEED) for e in range(w.B)]
+    ids = list(range(w.B))
+    solo = {}
+    for name, wt in (("A", wA), ("B", wB)):
+        r = Runner(w, wt, envs)
+        solo[name] = stack(r.run([ids], quota=0), ids)
+        r.close()
+    ra, rb = Runner(w, wA, envs, max_inflight_groups=2), Runner(w, wB, envs, max_inflight_groups=2)
+    sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
+    noise = torch.stack([ra.noise[e] for e in ids])
+    outs = {"A": [], "B": []}
+    for rep in range(3):                       # interleaved submits, nothing synchronised in between
+        for name, r, st, quota in (("A", ra, sa, 100), ("B", rb, sb, 48)):
+            out = torch.empty_like(noise)
+            half = w.B // 2
+            sidx = [envs[e].step for e in ids]
+            r.gen.submit([1000 * rep + e for e in ids[:half]], [r.kv[e] for e in ids[:half]], noise[:half], out[:half],
+                         sm_quota=quota, stream=st, step_index=sidx[:half])
+            r.gen.submit([1000 * rep + e for e in ids[half:]], [r.kv[e] for e in ids[half:]], noise[half:], out[half:],
+                         sm_quota=quota, stream=st, step_index=sidx[half:])
+            outs[name].append(out)
+    ra.gen.sync()
+    rb.gen.sync()
+    for name in ("A", "B"):
+        for out in outs[name]:
+            assert np.array_equal(out.cpu().numpy(), solo[name])
+    ra.close()
+    rb.close()
