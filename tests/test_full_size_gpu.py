@@ -103,22 +103,25 @@ def test_configs3_quota_sweep_bit_identity():
 
 
 def test_configs4_full_size_sampled_one_step():
-    """configs[4]: 2048 envs, ragged groups of 32..256 at the 74-SM quota, queue depth 8 (the bench's
-    launch configuration).  One Euler step of four sampled envs against the oracle (a whole chunk
+    """configs[4]: 2048 envs, ragged groups of 32..256 at the 74-SM quota, queue depth 16 (the bench's
+    launch configuration: the whole step is one packed batch of 32768 rows); also at depth 8 (two batches).  One Euler step of four sampled envs against the oracle (a whole chunk
     of this model costs the oracle about a minute per environment), plus the whole-chunk result of
     sampled envs against running them alone."""
     w = synth.WORKLOADS[4]
     wt = synth.make_weights(w, SEED, device="cuda")
     envs = {e: synth.make_env(w, e, SEED, device="cuda") for e in range(w.B)}
     groups = synth.arrival_groups(w, SEED)
-    gen, out1, pos = _run_full(w, wt, envs, groups, w.quota, n_steps=1)
+    gen, out1, pos = _run_full(w, wt, envs, groups, w.quota, n_steps=1, inflight=16)
     sample = [groups[0][0], groups[5][-1], groups[-1][-1], 1234]
     ref = _oracle(w, wt, envs, sample, n_steps=1)
     got = np.stack([out1[pos[e]].cpu().numpy() for e in sample])
     assert chunk_rel_err(got, ref) <= TOL["bf16"]
     gen.destroy()
-    gen, out, pos = _run_full(w, wt, envs, groups, w.quota)
+    gen, out, pos = _run_full(w, wt, envs, groups, w.quota, inflight=16)
     assert torch.isfinite(out).all()
     for e in sample[:2]:
         assert torch.equal(_alone(gen, w, envs, e, 148), out[pos[e]])
+    gen.destroy()
+    gen, out8, _ = _run_full(w, wt, envs, groups, w.quota, inflight=8)     # two batches instead of one: same bits
+    assert torch.equal(out8, out)
     gen.destroy()
