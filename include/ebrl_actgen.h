@@ -193,6 +193,15 @@ ebrl_status_t ebrl_actgen_submit(ebrl_actgen_t h, int32_t n_envs, const int64_t 
                                  const void *const *prefix_kv, const float *noise, float *out,
                                  int32_t sm_quota, void *stream, const ebrl_submit_ext_t *ext);
 
+/* The same as ebrl_actgen_submit with one DEVICE pointer per environment for its state and its
+ * result ([H][A] fp32 each, 4-byte aligned; out_ptrs[i] may equal state_ptrs[i]) instead of two
+ * [n][H][A] arrays: for callers whose environments keep their buffers apart (the queue of
+ * ebrl_queue.h).  state_ptrs and out_ptrs are host arrays, copied before the call returns. */
+ebrl_status_t ebrl_actgen_submit_scattered(ebrl_actgen_t h, int32_t n_envs, const int64_t *env_ids,
+                                           const void *const *prefix_kv, const float *const *state_ptrs,
+                                           float *const *out_ptrs, int32_t sm_quota, void *stream,
+                                           const ebrl_submit_ext_t *ext);
+
 /* The same with HOST buffers: prefix_kv[i], noise and out point to host memory (pinned memory
  * makes the copies asynchronous).  The planes and the noise are copied to device staging
  * owned by the handle when the call is made -- on a copy stream of the handle, so that the
@@ -245,6 +254,9 @@ ebrl_status_t ebrl_actgen_reset_stats(ebrl_actgen_t h);
 ebrl_status_t ebrl_actgen_set_timing(ebrl_actgen_t h, int32_t on);
 
 uint32_t ebrl_actgen_abi_version(void);
+
+/* K_steps of the handle's configuration (0 for NULL). */
+int32_t ebrl_actgen_k_steps(ebrl_actgen_t h);
 
 /* sizeof of an ABI struct as this library was compiled: 0 ebrl_actgen_cfg_t, 1 ebrl_layer_weights_t,
  * 2 ebrl_actgen_weights_t, 3 ebrl_submit_ext_t, 4 ebrl_actgen_stats_t; 0 for any other index.  For

@@ -56,6 +56,29 @@ class Stats(C.Structure):
                 ("class_bytes", C.c_double * len(KC_NAMES)), ("weights_version", C.c_uint64)]
 
 
+class QueueCfg(C.Structure):
+    _fields_ = [("capacity", C.c_int32), ("max_group", C.c_int32), ("sm_quota", C.c_int32), ("step_mode", C.c_int32),
+                ("linger_us", C.c_uint32), ("reserved_", C.c_uint32)]
+
+
+QUEUE_SUBMIT_FN = C.CFUNCTYPE(C.c_int32, C.c_void_p, C.c_int32, C.POINTER(C.c_int64), C.POINTER(C.c_void_p), C.POINTER(C.c_int32),
+                              C.POINTER(C.c_void_p), C.POINTER(C.c_void_p), C.POINTER(C.c_int32), C.c_int32, C.c_int32, C.c_void_p)
+QUEUE_SYNC_FN = C.CFUNCTYPE(C.c_int32, C.c_void_p)
+
+
+class QueueBackend(C.Structure):
+    _fields_ = [("ctx", C.c_void_p), ("K_steps", C.c_int32), ("submit", QUEUE_SUBMIT_FN), ("sync", QUEUE_SYNC_FN)]
+
+
+class QueueStats(C.Structure):
+    _fields_ = [("pushed", C.c_uint64), ("completed", C.c_uint64), ("failed", C.c_uint64), ("groups", C.c_uint64),
+                ("group_envs", C.c_uint64), ("blocked_pushes", C.c_uint64), ("max_waiting", C.c_int32),
+                ("waiting", C.c_int32), ("in_service", C.c_int32), ("reserved_", C.c_int32)]
+
+
+ERR_QUEUE_FULL, ERR_CLOSED = 8, 9
+
+
 class EbrlError(RuntimeError):
     def __init__(self, status: int, text: str):
         super().__init__("ebrl_actgen status %d: %s" % (status, text))
@@ -104,6 +127,18 @@ def lib():
         L.ebrl_actgen_l0_step_noalloc.argtypes = [C.c_void_p] * 7 + [C.c_int32] * 4 + [C.c_float, C.c_int32, C.c_void_p]
         L.ebrl_actgen_wait_probe.argtypes = [C.c_int32, C.c_uint64, C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_uint64)]
         L.ebrl_sim_corunner_launch.argtypes = [C.c_void_p, C.c_uint64, C.c_int32, C.c_int32, C.c_void_p]
+        L.ebrl_actgen_k_steps.argtypes = [C.c_void_p]
+        L.ebrl_actgen_submit_scattered.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_int64), C.POINTER(C.c_void_p),
+                                                   C.POINTER(C.c_void_p), C.POINTER(C.c_void_p), C.c_int32, C.c_void_p,
+                                                   C.POINTER(SubmitExt)]
+        L.ebrl_queue_create.argtypes = [C.c_void_p, C.POINTER(QueueCfg), C.c_void_p, C.POINTER(C.c_void_p)]
+        L.ebrl_queue_create_backend.argtypes = [C.POINTER(QueueBackend), C.POINTER(QueueCfg), C.c_void_p, C.POINTER(C.c_void_p)]
+        push = [C.c_void_p, C.c_int64, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(C.c_uint64)]
+        L.ebrl_queue_push.argtypes = push
+        L.ebrl_queue_try_push.argtypes = push
+        L.ebrl_queue_wait.argtypes = [C.c_void_p, C.c_uint64, C.c_uint32]
+        L.ebrl_queue_get_stats.argtypes = [C.c_void_p, C.POINTER(QueueStats)]
+        L.ebrl_queue_destroy.argtypes = [C.c_void_p]
         _lib = L
     return _lib
 
@@ -263,6 +298,61 @@ class ActGen:
             st = self._L.ebrl_actgen_destroy(h)
             if st != OK:
                 raise EbrlError(st, "destroy failed")
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+class Queue:
+    """``ebrl_queue_*``: the bounded request queue in front of a handle (or of a test backend)."""
+
+    def __init__(self, gen: Optional["ActGen"], *, capacity: int, max_group: int, sm_quota: int = 0, step_mode: bool = False,
+                 linger_us: int = 0, stream: Optional[torch.cuda.Stream] = None, backend: Optional[QueueBackend] = None):
+        self._L = lib()
+        self._gen = gen            # keeps the handle alive
+        self._backend = backend    # keeps the callbacks alive
+        cfg = QueueCfg(capacity, max_group, sm_quota, 1 if step_mode else 0, linger_us, 0)
+        self._q = C.c_void_p()
+        sp = stream.cuda_stream if stream is not None else None
+        if backend is not None:
+            st = self._L.ebrl_queue_create_backend(C.byref(backend), C.byref(cfg), sp, C.byref(self._q))
+        else:
+            st = self._L.ebrl_queue_create(gen._h, C.byref(cfg), sp, C.byref(self._q))
+        if st != OK:
+            raise EbrlError(st, "queue create failed")
+
+    def _push(self, fn, env_id, prefix, prefix_len, state, out, step_index):
+        t = C.c_uint64(0)
+        ptr = lambda x: x.data_ptr() if torch.is_tensor(x) else int(x)
+        st = fn(self._q, int(env_id), ptr(prefix), int(prefix_len), ptr(state), ptr(out), int(step_index), C.byref(t))
+        return st, int(t.value)
+
+    def push(self, env_id, prefix, prefix_len, state, out, step_index=0) -> int:
+        """Blocks while the queue is full; returns the ticket.  Tensors (device) or raw addresses."""
+        st, t = self._push(self._L.ebrl_queue_push, env_id, prefix, prefix_len, state, out, step_index)
+        if st != OK:
+            raise EbrlError(st, "queue push failed")
+        return t
+
+    def try_push(self, env_id, prefix, prefix_len, state, out, step_index=0):
+        """(status, ticket): status ERR_QUEUE_FULL instead of blocking."""
+        return self._push(self._L.ebrl_queue_try_push, env_id, prefix, prefix_len, state, out, step_index)
+
+    def wait(self, ticket: int, timeout_ms: int = 0) -> int:
+        return int(self._L.ebrl_queue_wait(self._q, int(ticket), int(timeout_ms)))
+
+    def stats(self) -> dict:
+        s = QueueStats()
+        self._L.ebrl_queue_get_stats(self._q, C.byref(s))
+        return {k: getattr(s, k) for k, _ in QueueStats._fields_ if k != "reserved_"}
+
+    def destroy(self):
+        if self._q:
+            q, self._q = self._q, C.c_void_p()
+            self._L.ebrl_queue_destroy(q)
 
     def __del__(self):
         try:

@@ -647,8 +647,17 @@ ebrl_status_t flush_slot(ebrl_actgen *h, Slot &s)
 
 ebrl_status_t submit_impl(ebrl_actgen *h, int32_t n, const int64_t *env_ids, const void *const *prefix_kv,
                           const float *noise, float *out, int32_t sm_quota, void *stream,
-                          const ebrl_submit_ext_t *ext, bool host_buffers)
+                          const ebrl_submit_ext_t *ext, bool host_buffers,
+                          const float *const *noise_ptrs = nullptr, float *const *out_ptrs = nullptr)
 {
+    if (noise_ptrs || out_ptrs) {   // per-environment state and result pointers instead of two [n][H][A] arrays
+        if (!noise_ptrs || !out_ptrs || host_buffers || n < 1) return fail(h, EBRL_ERR_INVALID_ARG, "per-environment pointers: both arrays, device buffers, n >= 1");
+        for (int i = 0; i < n; ++i)
+            if (!noise_ptrs[i] || !out_ptrs[i] || (((uintptr_t)noise_ptrs[i] | (uintptr_t)out_ptrs[i]) & 3))
+                return fail(h, EBRL_ERR_INVALID_ARG, "state or result pointer %d is NULL or not 4-byte aligned", i);
+        noise = noise_ptrs[0];   // non-NULL stand-ins for the common checks
+        out = out_ptrs[0];
+    }
     std::string why;
     ebrl_status_t st = check_submit(&h->cfg, h->n_sms, n, env_ids, prefix_kv, noise, out, sm_quota, ext, &why);
     if (st != EBRL_OK) return fail(h, st, "%s", why.c_str());
@@ -758,8 +767,8 @@ ebrl_status_t submit_impl(ebrl_actgen *h, int32_t n, const int64_t *env_ids, con
         int ns = K - m.k0;
         if (ext && ext->n_steps > 0 && ext->n_steps < ns) ns = ext->n_steps;
         m.nsteps = ns;
-        m.noise = noise_d + (size_t)i * chunk;
-        m.out = out_d + (size_t)i * chunk;
+        m.noise = noise_ptrs ? noise_ptrs[i] : noise_d + (size_t)i * chunk;
+        m.out = out_ptrs ? out_ptrs[i] : out_d + (size_t)i * chunk;
         s.pending.push_back(m);
         if (!group_maps.empty()) s.pending_maps.push_back(group_maps[i]);
         env_steps += (uint64_t)ns;
@@ -814,6 +823,8 @@ void free_all(ebrl_actgen *h)
 extern "C" {
 
 uint32_t ebrl_actgen_abi_version(void) { return EBRL_ACTGEN_ABI_VERSION; }
+
+int32_t ebrl_actgen_k_steps(ebrl_actgen_t h) { return h ? h->cfg.K_steps : 0; }
 
 uint64_t ebrl_actgen_struct_size(int32_t which)
 {
@@ -998,6 +1009,17 @@ ebrl_status_t ebrl_actgen_submit(ebrl_actgen_t h, int32_t n, const int64_t *env_
     if (!h) return EBRL_ERR_INVALID_ARG;
     std::lock_guard<std::mutex> lk(h->mu);
     return submit_impl(h, n, env_ids, prefix_kv, noise, out, sm_quota, stream, ext, false);
+}
+
+ebrl_status_t ebrl_actgen_submit_scattered(ebrl_actgen_t h, int32_t n, const int64_t *env_ids, const void *const *prefix_kv,
+                                           const float *const *state_ptrs, float *const *out_ptrs, int32_t sm_quota, void *stream,
+                                           const ebrl_submit_ext_t *ext)
+{
+    if (!h) return EBRL_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lk(h->mu);
+    if (n == 0) return EBRL_OK;
+    if (n < 0 || !state_ptrs || !out_ptrs) return fail(h, EBRL_ERR_INVALID_ARG, "n_envs < 0, or state_ptrs / out_ptrs is NULL");
+    return submit_impl(h, n, env_ids, prefix_kv, nullptr, nullptr, sm_quota, stream, ext, false, state_ptrs, out_ptrs);
 }
 
 ebrl_status_t ebrl_actgen_submit_host(ebrl_actgen_t h, int32_t n, const int64_t *env_ids, const void *const *prefix_kv_host,
