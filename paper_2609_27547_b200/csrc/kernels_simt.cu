@@ -323,16 +323,29 @@ constexpr int AKB = 32;   // keys per block: a constant, so the arithmetic is th
 
 __device__ __forceinline__ void group_sync(int g) { asm volatile("bar.sync %0, 128;" ::"r"(g + 1) : "memory"); }
 
+template <typename T> __device__ __forceinline__ void load4(const T *p, float (&v)[4]);
+template <> __device__ __forceinline__ void load4<float>(const float *p, float (&v)[4])
+{
+    const float4 x = *reinterpret_cast<const float4 *>(p);
+    v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w;
+}
+template <> __device__ __forceinline__ void load4<__nv_bfloat16>(const __nv_bfloat16 *p, float (&v)[4])
+{
+    const uint2 x = *reinterpret_cast<const uint2 *>(p);
+    const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162 *>(&x.x), hi = *reinterpret_cast<const __nv_bfloat162 *>(&x.y);
+    v[0] = __bfloat162float(lo.x); v[1] = __bfloat162float(lo.y); v[2] = __bfloat162float(hi.x); v[3] = __bfloat162float(hi.y);
+}
+
 template <typename T, int RMAX>
 __global__ void __launch_bounds__(512) attn_simt_kernel(AttnArgs a)
 {
-    extern __shared__ float smem[];
+    extern __shared__ __align__(16) float smem[];
     const int grp = threadIdx.x >> 7, t = threadIdx.x & 127, warp = t >> 5, lane = t & 31;
     const int H = a.H, hd = a.hd;
-    const int per_group = H * hd + AKB * (hd + 1) + AKB * hd + H * AKB + 2 * H;
+    const int per_group = (H * hd + AKB * (hd + 4) + AKB * hd + H * AKB + 2 * H + 3) & ~3;   // 16-byte multiples: rows are read as float4
     float *q = smem + (size_t)grp * per_group;
     float *kb = q + H * hd;
-    float *vb = kb + AKB * (hd + 1);
+    float *vb = kb + AKB * (hd + 4);   // key rows padded by four floats: float4 reads of 32 different rows do not collide
     float *p = vb + AKB * hd;
     float *alpha = p + H * AKB;
     float *lsum = alpha + H;
@@ -371,15 +384,15 @@ __global__ void __launch_bounds__(512) attn_simt_kernel(AttnArgs a)
         for (int j0 = 0; j0 < P; j0 += AKB) {
             group_sync(grp);   // q ready; previous block's readers done
             const int nkeys = min(AKB, P - j0);
-            for (int e = t; e < AKB * hd; e += 128) {
-                const int j = e >> hd_sh, cc = e & (hd - 1);
-                float kv = 0.f, vv = 0.f;
+            for (int e = t; e < AKB * (hd >> 2); e += 128) {   // four columns per thread and turn
+                const int j = e >> (hd_sh - 2), cc = (e & ((hd >> 2) - 1)) << 2;
+                float kv[4] = {0.f, 0.f, 0.f, 0.f}, vv[4] = {0.f, 0.f, 0.f, 0.f};
                 if (j < nkeys) {
-                    kv = ldf(kbase + (size_t)(j0 + j) * kvs + cc);
-                    vv = ldf(vbase + (size_t)(j0 + j) * kvs + cc);
+                    load4(kbase + (size_t)(j0 + j) * kvs + cc, kv);
+                    load4(vbase + (size_t)(j0 + j) * kvs + cc, vv);
                 }
-                kb[j * (hd + 1) + cc] = kv;
-                vb[j * hd + cc] = vv;
+                *reinterpret_cast<float4 *>(kb + j * (hd + 4) + cc) = make_float4(kv[0], kv[1], kv[2], kv[3]);
+                *reinterpret_cast<float4 *>(vb + j * hd + cc) = make_float4(vv[0], vv[1], vv[2], vv[3]);
             }
             group_sync(grp);
             // scores and running softmax statistics: lane = key, each warp owns rows warp + 4 r
@@ -387,13 +400,19 @@ __global__ void __launch_bounds__(512) attn_simt_kernel(AttnArgs a)
             for (int r0 = 0; r0 < 8; r0 += 4) {
                 if (warp + 4 * r0 >= H) continue;   // no query row in this pass (warp-uniform)
                 float s[4] = {0.f, 0.f, 0.f, 0.f};
-                const float *krow = kb + lane * (hd + 1);
-                for (int cc = 0; cc < hd; ++cc) {
-                    const float kvv = krow[cc];
+                // four columns at a time: one 16-byte read of the key row and one broadcast read per query row
+                // feed 16 FMAs (the chain per score still runs over the columns in order)
+                const float4 *krow = reinterpret_cast<const float4 *>(kb + lane * (hd + 4));
+                for (int c4 = 0; c4 < (hd >> 2); ++c4) {
+                    const float4 k4 = krow[c4];
 #pragma unroll
                     for (int r = 0; r < 4; ++r) {
                         const int i = warp + 4 * (r0 + r);
-                        if (i < H) s[r] = fmaf(q[i * hd + cc], kvv, s[r]);
+                        if (i < H) {
+                            const float4 q4 = *reinterpret_cast<const float4 *>(q + i * hd + 4 * c4);
+                            s[r] = fmaf(q4.x, k4.x, s[r]); s[r] = fmaf(q4.y, k4.y, s[r]);
+                            s[r] = fmaf(q4.z, k4.z, s[r]); s[r] = fmaf(q4.w, k4.w, s[r]);
+                        }
                     }
                 }
 #pragma unroll
@@ -418,12 +437,17 @@ __global__ void __launch_bounds__(512) attn_simt_kernel(AttnArgs a)
                 const int i = rg + ncg * r;
                 if (i < H) acc[r] *= alpha[i];
             }
-            for (int j = 0; j < nkeys; ++j) {
-                const float vv = vb[j * hd + c];
+            // four keys at a time (weights and values of keys past the prefix are exact zeros: they add nothing)
+            for (int j = 0; j < ((nkeys + 3) & ~3); j += 4) {
+                const float v0 = vb[j * hd + c], v1 = vb[(j + 1) * hd + c], v2 = vb[(j + 2) * hd + c], v3 = vb[(j + 3) * hd + c];
 #pragma unroll
                 for (int r = 0; r < RMAX; ++r) {
                     const int i = rg + ncg * r;
-                    if (i < H) acc[r] = fmaf(p[i * AKB + j], vv, acc[r]);
+                    if (i < H) {
+                        const float4 p4 = *reinterpret_cast<const float4 *>(p + i * AKB + j);
+                        acc[r] = fmaf(p4.x, v0, acc[r]); acc[r] = fmaf(p4.y, v1, acc[r]);
+                        acc[r] = fmaf(p4.z, v2, acc[r]); acc[r] = fmaf(p4.w, v3, acc[r]);
+                    }
                 }
             }
         }
@@ -568,7 +592,7 @@ cudaError_t launch_attn_simt(const AttnArgs &a, int bf16, int grid, cudaStream_t
     if (items == 0) return cudaSuccess;
     const int need = (items + 3) / 4;
     const int g = need < grid ? need : grid;
-    const size_t per_group = (size_t)a.H * a.hd + AKB * (a.hd + 1) + AKB * a.hd + a.H * AKB + 2 * a.H;
+    const size_t per_group = ((size_t)a.H * a.hd + AKB * (a.hd + 4) + AKB * a.hd + a.H * AKB + 2 * a.H + 3) & ~(size_t)3;
     const size_t smem = 4 * per_group * sizeof(float);
     return bf16 ? attn_dispatch<__nv_bfloat16>(a, g, smem, st) : attn_dispatch<float>(a, g, smem, st);
 }
