@@ -43,6 +43,53 @@ __device__ __forceinline__ float gelu_erf(float z)
     const float q = p * t * e;
     return z * (z >= 0.f ? 1.0f - q : q);
 }
+// Two fp32 values per instruction (fma / mul / add .f32x2: IEEE per lane, the same results as the scalar
+// forms).  The epilogue's arithmetic shares the schedulers with the single TMA and MMA threads, and across
+// all epilogue kinds the tensor pipe's active share falls one for one as the epilogue's issue share rises,
+// so halving its instruction count is worth more than any reordering.
+__device__ __forceinline__ uint64_t pk2(float a, float b)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+    return r;
+}
+__device__ __forceinline__ void upk2(uint64_t v, float &a, float &b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v)); }
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b)
+{
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+// gelu_erf of two values at once: the same approximation, the polynomial and the products in packed form;
+// the reciprocal, the exponential and the sign handling stay scalar.  Phi = 1/2 + sign(z) (1/2 - q).
+__device__ __forceinline__ void gelu_erf2(float &z0, float &z1)
+{
+    const uint64_t z = pk2(z0, z1);
+    float t0, t1, e0, e1, a0, a1;
+    upk2(mul2(mul2(z, z), pk2(-0.72134752044448170f, -0.72134752044448170f)), a0, a1);   // -z^2 log2(e) / 2
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t0) : "f"(fmaf(fabsf(z0), 0.23164189f, 1.0f)));
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t1) : "f"(fmaf(fabsf(z1), 0.23164189f, 1.0f)));
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"(a0));
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e1) : "f"(a1));
+    const uint64_t t = pk2(t0, t1);
+    uint64_t p = fma2(pk2(0.5307027145f, 0.5307027145f), t, pk2(-0.7265760135f, -0.7265760135f));
+    p = fma2(p, t, pk2(0.7107068705f, 0.7107068705f));
+    p = fma2(p, t, pk2(-0.142248368f, -0.142248368f));
+    p = fma2(p, t, pk2(0.127414796f, 0.127414796f));
+    const uint64_t q = mul2(mul2(p, t), pk2(e0, e1));
+    float h0, h1;
+    upk2(fma2(q, pk2(-1.0f, -1.0f), pk2(0.5f, 0.5f)), h0, h1);                           // 1/2 - q
+    h0 = __uint_as_float(__float_as_uint(h0) ^ (__float_as_uint(z0) & 0x80000000u));   // times sign(z)
+    h1 = __uint_as_float(__float_as_uint(h1) ^ (__float_as_uint(z1) & 0x80000000u));
+    const uint64_t phi = fma2(pk2(h0, h1), pk2(1.0f, 1.0f), pk2(0.5f, 0.5f));
+    upk2(mul2(z, phi), z0, z1);
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -208,8 +255,9 @@ __device__ __forceinline__ bool epilogue_store_tma(const GemmArgs &g, const CUte
                 uint32_t w[4];
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    float lo = __uint_as_float(r[8 * j + 2 * e]) * rs, hi = __uint_as_float(r[8 * j + 2 * e + 1]) * rs;
-                    if (EPI == EPI_SCALE_GELU) { lo = gelu_erf(lo); hi = gelu_erf(hi); }
+                    float lo, hi;
+                    upk2(mul2(pk2(__uint_as_float(r[8 * j + 2 * e]), __uint_as_float(r[8 * j + 2 * e + 1])), pk2(rs, rs)), lo, hi);
+                    if (EPI == EPI_SCALE_GELU) gelu_erf2(lo, hi);
                     w[e] = pack_bf16(lo, hi);
                 }
                 const int p = c * 4 + j;
