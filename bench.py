@@ -307,7 +307,7 @@ def run_ours(args):
         bound = "alu"
     achieved = gemm["flops"] / (gemm["ms"] * 1e-3) / 1e12 if gemm["ms"] > 0 else 0.0
     # DRAM traffic per GEMM launch from the ncu capture of one layer of this model at M = 8192 rows
-    # (profiles/gemm_tc2_cfg4_512env.md): 0.117 GB of weights per layer, which do not grow with M, plus
+    # (the committed summary of that capture sits with the other profiles): 0.117 GB of weights per layer, which do not grow with M, plus
     # 0.971 GB of activations, which grow in proportion to the rows; six launches per layer.
     traffic, traffic_note = None, None
     if bf16 and (w.d, w.L, w.H, w.mlp_mult) == (2048, 8, 16, 4) and gemm["launches"] > 0:
