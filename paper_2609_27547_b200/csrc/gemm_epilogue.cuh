@@ -66,15 +66,17 @@ __device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b)
     asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
 }
-// gelu_erf of two values at once: the same approximation, the polynomial and the products in packed form;
-// the reciprocal, the exponential and the sign handling stay scalar.  Phi = 1/2 + sign(z) (1/2 - q).
+// gelu_erf of two values at once: the same approximation with the polynomial and the products in packed
+// form; only |z|, the reciprocal and the exponential stay scalar.  With q = 1/2 (a1 t + ... + a5 t^5) exp(-z^2/2),
+// Phi(z) = 1/2 + sign(z) (1/2 - q), hence z Phi(z) = z / 2 + |z| (1/2 - q).
 __device__ __forceinline__ void gelu_erf2(float &z0, float &z1)
 {
-    const uint64_t z = pk2(z0, z1);
-    float t0, t1, e0, e1, a0, a1;
+    const uint64_t z = pk2(z0, z1), az = pk2(fabsf(z0), fabsf(z1));
+    float t0, t1, e0, e1, a0, a1, r0, r1;
     upk2(mul2(mul2(z, z), pk2(-0.72134752044448170f, -0.72134752044448170f)), a0, a1);   // -z^2 log2(e) / 2
-    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t0) : "f"(fmaf(fabsf(z0), 0.23164189f, 1.0f)));
-    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t1) : "f"(fmaf(fabsf(z1), 0.23164189f, 1.0f)));
+    upk2(fma2(az, pk2(0.23164189f, 0.23164189f), pk2(1.0f, 1.0f)), r0, r1);              // 1 + p |z|
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t0) : "f"(r0));
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t1) : "f"(r1));
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"(a0));
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e1) : "f"(a1));
     const uint64_t t = pk2(t0, t1);
@@ -83,12 +85,8 @@ __device__ __forceinline__ void gelu_erf2(float &z0, float &z1)
     p = fma2(p, t, pk2(-0.142248368f, -0.142248368f));
     p = fma2(p, t, pk2(0.127414796f, 0.127414796f));
     const uint64_t q = mul2(mul2(p, t), pk2(e0, e1));
-    float h0, h1;
-    upk2(fma2(q, pk2(-1.0f, -1.0f), pk2(0.5f, 0.5f)), h0, h1);                           // 1/2 - q
-    h0 = __uint_as_float(__float_as_uint(h0) ^ (__float_as_uint(z0) & 0x80000000u));   // times sign(z)
-    h1 = __uint_as_float(__float_as_uint(h1) ^ (__float_as_uint(z1) & 0x80000000u));
-    const uint64_t phi = fma2(pk2(h0, h1), pk2(1.0f, 1.0f), pk2(0.5f, 0.5f));
-    upk2(mul2(z, phi), z0, z1);
+    const uint64_t h = fma2(q, pk2(-1.0f, -1.0f), pk2(0.5f, 0.5f));                      // 1/2 - q
+    upk2(fma2(az, h, mul2(z, pk2(0.5f, 0.5f))), z0, z1);
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 {
