@@ -102,11 +102,12 @@ def test_configs3_quota_sweep_bit_identity():
     assert chunk_rel_err(np.stack([base[e].cpu().numpy() for e in sample]), ref) <= TOL["f32"]
 
 
-def test_configs4_full_size_sampled_one_step():
+def test_configs4_full_size_sampled():
     """configs[4]: 2048 envs, ragged groups of 32..256 at the 74-SM quota, queue depth 16 (the bench's
-    launch configuration: the whole step is one packed batch of 32768 rows); also at depth 8 (two batches).  One Euler step of four sampled envs against the oracle (a whole chunk
-    of this model costs the oracle about a minute per environment), plus the whole-chunk result of
-    sampled envs against running them alone."""
+    launch configuration: the whole step is one packed batch of 32768 rows); also at depth 8 (two batches).
+    One Euler step of four sampled envs against the oracle, then the whole chunk (K = 10 steps) of six
+    envs against the oracle (about a minute of host time per environment, one thread each), plus the
+    whole-chunk result of sampled envs against running them alone."""
     w = synth.WORKLOADS[4]
     wt = synth.make_weights(w, SEED, device="cuda")
     envs = {e: synth.make_env(w, e, SEED, device="cuda") for e in range(w.B)}
@@ -119,9 +120,20 @@ def test_configs4_full_size_sampled_one_step():
     gen.destroy()
     gen, out, pos = _run_full(w, wt, envs, groups, w.quota, inflight=16)
     assert torch.isfinite(out).all()
+    # the FINAL action chunk (all K = 10 Euler steps) of six environments against the oracle.  Packed
+    # rows follow the arrival order (all environments run the same number of steps), 16 environments
+    # per 256-row pair tile: positions 0 and 15 are the first and last rows of the first pair tile,
+    # 7 and 8 the last rows of its leader CTA and the first of its peer CTA, 1000 sits mid-batch
+    # and 2047 holds the last 16 rows of the batch.
+    order = [e for g in groups for e in g]
+    chunk_sample = [order[p] for p in (0, 7, 8, 15, 1000, w.B - 1)]
+    ref_k = _oracle(w, wt, envs, chunk_sample)
+    got_k = np.stack([out[pos[e]].cpu().numpy() for e in chunk_sample])
+    assert chunk_rel_err(got_k, ref_k) <= TOL["bf16"]
     for e in sample[:2]:
         assert torch.equal(_alone(gen, w, envs, e, 148), out[pos[e]])
     gen.destroy()
     gen, out8, _ = _run_full(w, wt, envs, groups, w.quota, inflight=8)     # two batches instead of one: same bits
-    assert torch.equal(out8, out)
+    assert torch.equal(out8, out)                                          # (the first batch ends in a ragged row tile)
+    assert sum(len(g) for g in groups[:8]) * w.H % 256 != 0
     gen.destroy()

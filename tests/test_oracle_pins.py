@@ -403,9 +403,10 @@ def test_tiny_case_by_scalar_arithmetic():
 
 # ---------------------------------------------------------------- library composition
 
-def _torch_reference(w, wt, env, n_steps=0):
+def _torch_reference(w, wt, env, n_steps=0, planes=None):
     """The same network composed from torch's own fp64 routines (rms_norm, softmax, erf-GELU,
-    matmul), vectorised over tokens and heads: independent of the C loops."""
+    matmul), vectorised over tokens and heads: independent of the C loops.  ``planes`` [L][2][P][d]
+    gives every layer its own K/V pair (kv_layers = n_layers) instead of the environment's shared one."""
     F = torch.nn.functional
     D = torch.float64
     H, d, nh, hd = w.H, w.d, w.n_heads, w.head_dim
@@ -417,7 +418,7 @@ def _torch_reference(w, wt, env, n_steps=0):
         j = torch.arange(d // 2, dtype=D)
         ang = (1000.0 * k / w.K) * torch.pow(torch.tensor(10000.0, dtype=D), -j / (d // 2))
         x = a @ wt["w_in"].to(D).T + torch.cat([torch.sin(ang), torch.cos(ang)])[None, :]
-        for l in wt["layers"]:
+        for li, l in enumerate(wt["layers"]):
             y = F.rms_norm(x, (d,), l["g1"].to(D), 1e-6)
             q, kk, v = (y @ l["w_qkv"].to(D).T).split(d, dim=1)
             sh = lambda t, n: t.reshape(n, nh, hd).transpose(0, 1)
@@ -427,6 +428,8 @@ def _torch_reference(w, wt, env, n_steps=0):
             qc = y @ l["w_qc"].to(D).T
             if w.d_ctx > 0:   # this layer's keys and values from the prefix's hidden states
                 Kc, Vc = env.kv.to(D) @ l["w_kc"].to(D).T, env.kv.to(D) @ l["w_vc"].to(D).T
+            elif planes is not None:   # this layer's own cached pair
+                Kc, Vc = planes[li, 0].to(D), planes[li, 1].to(D)
             P = Kc.shape[0]
             p = torch.softmax(sh(qc, H) @ sh(Kc, P).transpose(1, 2) / math.sqrt(hd), dim=-1)
             x = x + (p @ sh(Vc, P)).transpose(0, 1).reshape(H, d) @ l["w_oc"].to(D).T
@@ -448,6 +451,90 @@ def test_against_torch_fp64_composition(dtype):
     got1 = oracle_run(w, wt, envs, n_steps=1)
     for i, e in enumerate(envs):
         assert np.abs(got1[i] - _torch_reference(w, wt, e, n_steps=1)).max() < 1e-11
+
+
+# ---------------------------------------------------------------- per-layer prefix planes (kv_layers = n_layers)
+
+def _layer_planes(w, env_id, P):
+    return synth.normal(SEED, "kv_per_layer", env_id, (w.L, 2, P, w.d), dtype=w.torch_dtype)
+
+
+def _per_layer_cfg(w):
+    oc = oracle_cfg(w)
+    oc.kv_layers = w.L
+    return oc
+
+
+def test_per_layer_planes_uniform_attention_closed_form():
+    """kv_layers = n_layers with W_qc = 0 and only the cross-attention branch alive: the softmax is
+    uniform, so layer l adds W_oc_l mean_p V_l[p] -- its OWN value plane -- to every token.  A wrong
+    plane stride, a K/V swap or a layer mix-up all change the sum."""
+    w = small(P=(6, 6), L=3)
+    wt = _only_cross(w, synth.make_weights(w, SEED, random_gains=True))
+    for l in wt["layers"]:
+        l["w_qc"].zero_()
+    e = synth.make_env(w, 2, SEED)
+    planes = _layer_planes(w, 2, e.P)
+    a = np32(e.noise).astype(np.float64)
+    x = _embed(w, wt, a, 3)
+    for li, l in enumerate(wt["layers"]):
+        vbar = np32(planes)[li, 1].astype(np.float64).mean(axis=0)
+        x = x + (np32(l["w_oc"]).astype(np.float64) @ vbar)[None, :]
+    got = oracle.velocity(_per_layer_cfg(w), oracle_weights(wt), np32(planes), a, 3)
+    assert np.abs(got - _head(w, wt, x)).max() < 1e-12
+    # the key planes play no part here, the value planes all do
+    other = np32(planes).copy()
+    other[:, 0] = 7.0
+    assert np.abs(oracle.velocity(_per_layer_cfg(w), oracle_weights(wt), other, a, 3) - got).max() < 1e-12
+    for li in range(w.L):
+        other = np32(planes).copy()
+        other[li, 1] += 1.0
+        assert np.abs(oracle.velocity(_per_layer_cfg(w), oracle_weights(wt), other, a, 3) - got).max() > 1e-3
+
+
+def test_per_layer_planes_single_token_closed_form():
+    """P = 1 and per-layer planes: layer l adds W_oc_l V_l[0] whatever the queries and keys are."""
+    w = small(P=(1, 1), L=2)
+    wt = _only_cross(w, synth.make_weights(w, SEED, random_gains=True))
+    e = synth.make_env(w, 0, SEED)
+    planes = _layer_planes(w, 0, 1)
+    a = np32(e.noise).astype(np.float64)
+    x = _embed(w, wt, a, 1)
+    for li, l in enumerate(wt["layers"]):
+        x = x + (np32(l["w_oc"]).astype(np.float64) @ np32(planes)[li, 1, 0].astype(np.float64))[None, :]
+    got = oracle.velocity(_per_layer_cfg(w), oracle_weights(wt), np32(planes), a, 1)
+    assert np.abs(got - _head(w, wt, x)).max() < 1e-12
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_per_layer_planes_against_torch_fp64_composition(dtype):
+    """The whole network with a K/V pair per layer against the torch composition, and the checks
+    that make the layout matter: swapping two layers' pairs, or K and V inside one layer, changes
+    the result; repeating one pair for every layer reproduces the shared-plane form exactly."""
+    w = synth.scaled(synth.WORKLOADS[0], B=3, dtype=dtype, L=3, P=(9, 33), mixed_steps=True)
+    wt = synth.make_weights(w, SEED, random_gains=True)
+    envs = [synth.make_env(w, e, SEED) for e in range(w.B)]
+    planes = [_layer_planes(w, e.env_id, e.P) for e in envs]
+
+    def run(pl, n_steps=0):
+        return oracle.actgen(_per_layer_cfg(w), oracle_weights(wt), [np32(p) for p in pl],
+                             np.stack([np32(e.noise) for e in envs]), step_index=[e.step for e in envs], n_steps=n_steps)
+
+    got = run(planes)
+    for i, e in enumerate(envs):
+        assert np.abs(got[i] - _torch_reference(w, wt, e, planes=planes[i])).max() < 1e-11
+    got1 = run(planes, n_steps=1)
+    for i, e in enumerate(envs):
+        assert np.abs(got1[i] - _torch_reference(w, wt, e, n_steps=1, planes=planes[i])).max() < 1e-11
+    assert np.abs(run([p[[1, 0, 2]] for p in planes]) - got).max() > 1e-4          # layers 0 and 1 exchanged
+    assert np.abs(run([p[[0, 2, 1]] for p in planes]) - got).max() > 1e-4          # layers 1 and 2 exchanged
+    kvswap = [p.clone() for p in planes]
+    for p in kvswap:
+        p[2] = p[2].flip(0)                                                        # K <-> V in the last layer only
+    assert np.abs(run(kvswap) - got).max() > 1e-4
+    shared = oracle_run(w, wt, envs)                                               # kv_layers = 1 on each env's own pair
+    rep = run([e.kv.expand(w.L, -1, -1, -1).contiguous() for e in envs])
+    assert np.array_equal(rep, shared)
 
 
 # ---------------------------------------------------------------- hidden-state prefixes

@@ -48,6 +48,33 @@ def test_small_models_parity_ragged(dtype):
     assert chunk_rel_err(got, ref) <= TOL[dtype]
 
 
+def test_every_gemm_tile_shape_every_row_against_the_oracle(monkeypatch):
+    """The three tensor-core GEMM tile shapes forced in turn (CTA pairs on 256 x 256 tiles, one CTA on
+    128 x 256, one CTA on 128 x 128) on a batch of 43 envs x H=16 = 688 rows: two full 256-row pair
+    tiles plus a tail whose leader CTA is full and whose peer CTA holds 48 rows, and 128-row tiles 5 full
+    + 48.  EVERY row is compared with the oracle, and the three shapes with each other bit for bit
+    (each output element accumulates over k in the same order whatever the tile)."""
+    w = synth.scaled(synth.WORKLOADS[0], B=43, dtype="bf16", H=16, A=14, d=512, n_heads=8, L=2, K=3, P=(5, 90),
+                     mixed_steps=True)
+    wt, envs = _setup(w)
+    ref = oracle_run(w, wt, envs)
+    ids = list(range(w.B))
+    got = {}
+    for shape in ("2", "256", "128"):
+        monkeypatch.setenv("EBRL_GEMM_SHAPE", shape)    # read when the handle is created
+        r = Runner(w, wt, envs)
+        got[shape] = stack(r.run([ids]), ids)
+        if shape == "2":
+            assert np.array_equal(stack(r.run([ids], quota=37), ids), got[shape])   # 18 pairs instead of 74
+        r.close()
+        assert chunk_rel_err(got[shape], ref) <= TOL["bf16"], "tile shape %s" % shape
+    monkeypatch.delenv("EBRL_GEMM_SHAPE")
+    assert np.array_equal(got["2"], got["256"]) and np.array_equal(got["2"], got["128"])
+    r = Runner(w, wt, envs)                              # and the shapes the library picks by itself
+    assert np.array_equal(stack(r.run([ids]), ids), got["2"])
+    r.close()
+
+
 def test_bf16_plain_alu_kernels_parity():
     """The bf16 model on the plain-ALU kernels (the path taken when d is not a multiple of 256,
     and on request)."""
@@ -320,6 +347,10 @@ def test_weight_publication_switches_versions_between_batches(dtype):
         refs[name] = stack(r.run([ids]), ids)
         r.close()
     assert not np.array_equal(refs["A"], refs["B"])
+    # each version's chunks are the oracle's for that version's weights (and not the other's)
+    assert chunk_rel_err(refs["A"], oracle_run(w, wA, envs)) <= TOL[dtype]
+    assert chunk_rel_err(refs["B"], oracle_run(w, wB, envs)) <= TOL[dtype]
+    assert chunk_rel_err(refs["A"], oracle_run(w, wB, envs)) > 10 * TOL[dtype]
     r = Runner(w, wA, envs, max_inflight_groups=4)
     assert r.gen.weights_version() == 1
     noise = torch.stack([r.noise[e] for e in ids])

@@ -6,7 +6,8 @@ control loop that must not take the allocator's lock, a worker whose memory budg
 start-up.  ``ebrl_actgen_l0_step_noalloc`` serves them with scratch that is part of the library
 image.  The test calls it through the C ABI twice in a row (the scratch keeps the first call's
 contents) and checks each result against the ordinary entry point run on the same inputs, within
-the fp32 tolerance of the parity tests.
+the fp32 tolerance of the parity tests; both are also checked against the fp64 oracle's single
+Euler step of the same layer-less model.
 """
 import math
 
@@ -16,7 +17,7 @@ import torch
 
 from paper_2609_27547_b200 import binding as B
 from paper_2609_27547_b200 import synth
-from helpers import chunk_rel_err
+from helpers import chunk_rel_err, oracle_cfg, oracle_weights
 from gpu_helpers import TOL
 
 pytestmark = pytest.mark.gpu
@@ -35,6 +36,7 @@ def test_no_alloc_step_matches_submit_on_two_calls_in_a_row():
     gen = B.ActGen(B.cfg_for(w, max_group_envs=w.B), wt)
     kv = [torch.zeros((1, 2, 4, w.d), device="cuda") for _ in range(w.B)]
     ids = list(range(w.B))
+    import oracle
     for call, (seed, k) in enumerate([(5, 0), (6, 3)]):
         a = synth.normal(seed, "state", 0, (w.B, w.H, w.A)).cuda()
         want = torch.empty_like(a)
@@ -47,6 +49,10 @@ def test_no_alloc_step_matches_submit_on_two_calls_in_a_row():
         torch.cuda.synchronize()
         assert torch.isfinite(got).all()
         assert chunk_rel_err(got.cpu().numpy(), want.cpu().numpy().astype(np.float64)) <= TOL["f32"], "call %d" % call
+        ref = oracle.actgen(oracle_cfg(w), oracle_weights(wt), [np.zeros((1, 2, 4, w.d), np.float32)] * w.B, a.cpu().numpy(),
+                            step_index=[k] * w.B, n_steps=1)
+        assert chunk_rel_err(got.cpu().numpy(), ref) <= TOL["f32"], "call %d against the oracle" % call
+        assert chunk_rel_err(want.cpu().numpy(), ref) <= TOL["f32"], "call %d, ordinary entry point against the oracle" % call
     gen.destroy()
 
 
