@@ -13,18 +13,25 @@ second (a chunk = one environment's K Euler steps).
 * ``e2e``: the same through ``ebrl_actgen_submit_host`` with pinned HOST buffers (host->device
   copies of planes and noise and the device->host copy of the chunks inside the timed region).
 * ``roofline``: the dominant kernel class (the GEMMs) timed with CUDA events around each launch
-  in a second pass of the same steps; peak from MEASURED_PEAKS.json scaled by quota/SMs.
+  in a second pass of the same steps.  ``frac`` is taken against what the quota's SMs can issue at
+  the SM clock sampled during that pass (8192 dense bf16 FLOP per clock per SM); the fractions
+  against MEASURED_PEAKS.json's burst and sustained figures scaled by quota/SMs (measured on the
+  whole, power-capped chip at a lower clock) and against the nominal 2250 TFLOP/s are beside it.
 * ``cpu_baseline``: the fp64 oracle as it stands on this machine's host cores, on a bounded sample.
 * ``--impl reference`` times that oracle alone (there is no other reference implementation).
 
-Under torchrun each rank runs the same workload shape on its own shard of environment ids
-(environments are independent: no data-path collective); ``value`` sums over ranks.
+``--gpus N`` with N > 1 starts N ranks (one per GPU, through torch.distributed.run on 127.0.0.1)
+unless the process already is one of them (RANK / WORLD_SIZE in the environment).  Each rank runs
+the same workload shape on its own shard of the job's environment ids (id mod world; environments
+are independent, so there is no data-path collective); the ranks meet only for the barriers and
+the max-over-ranks of the step time; ``value`` counts the environments of all ranks.
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
+import socket
 import statistics
 import subprocess
 import sys
@@ -38,6 +45,9 @@ UNIT = "chunks/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 N_SMS = 148
 FP32_ALU_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12   # 148 SMs x 128 FFMA lanes x 2 flop x 1965 MHz
+BF16_FLOP_PER_CLK_SM = 8192                        # dense bf16 tcgen05: 2250 TFLOP/s nominal = 148 SMs x 8192 x 1.856 GHz
+FP32_FLOP_PER_CLK_SM = 256                         # 128 FFMA lanes x 2
+NOMINAL_BF16_TFLOPS = 2250.0
 
 
 def load_peaks():
@@ -52,7 +62,7 @@ def load_peaks():
     return d
 
 
-def parse_args():
+def parse_args(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=5)
@@ -75,7 +85,13 @@ def parse_args():
     ap.add_argument("--min-warmup", type=int, default=3, help="lower bound on warm-up steps (profiling captures use 1)")
     ap.add_argument("--d-ctx", type=int, default=0, help="variant: prefixes are hidden states [P][d_ctx], projected to K/V per layer")
     ap.add_argument("--inflight", type=int, default=16, help="groups queued before a batch is launched")
-    return ap.parse_args()
+    ap.add_argument("--sweep", action="store_true",
+                    help="one line per other configuration: configs[0..2], and configs[3] at quotas 148/74/37/16 with and "
+                         "without the streaming co-runner (the committed summary of these lines sits with the profiles)")
+    ap.add_argument("--stub-step-ms", type=float, default=0.0,
+                    help="testing the rank plumbing without a GPU: every step is a sleep of this many ms (+ the rank), "
+                         "ranks talk over gloo, the line says \"data\": \"stub\" -- never a measurement")
+    return ap.parse_args(argv)
 
 
 def workload_flops(w, envs) -> float:
@@ -202,21 +218,115 @@ class ClockSampler:
                 "power_w_max": max(power), "samples": len(sm)}
 
 
-def run_ours(args):
+class RankContext:
+    """One process per GPU: which rank this is, and the only things ranks do together -- a barrier
+    and the maximum of a number (the step time).  Environments are independent (section 4.2.2), so
+    the data path has no collective; `backend` is "nccl" on GPUs and "gloo" for the CPU test of
+    this plumbing."""
+
+    def __init__(self, backend: str, device=None):
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.local = int(os.environ.get("LOCAL_RANK", "0"))
+        self.dist = None
+        if self.world > 1:
+            import torch.distributed as dist
+            os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+            if backend == "nccl":
+                dist.init_process_group("nccl", device_id=device)
+            else:
+                dist.init_process_group(backend, rank=self.rank, world_size=self.world)
+            self.dist = dist
+        self.device = device
+
+    def shard(self, envs_per_rank: int):
+        """This rank's environment ids: the job has world x envs_per_rank environments (weak scaling),
+        environment e belongs to rank e mod world."""
+        from paper_2609_27547_b200 import synth
+        return synth.shard_env_ids(self.world * envs_per_rank, self.rank, self.world)
+
+    def barrier(self):
+        if self.dist is not None:
+            self.dist.barrier()
+        if self.device is not None:
+            import torch
+            torch.cuda.synchronize(self.device)
+
+    def max_over_ranks(self, x: float) -> float:
+        if self.dist is None:
+            return float(x)
+        import torch
+        t = torch.tensor([float(x)], dtype=torch.float64, device=self.device if self.device is not None else "cpu")
+        if self.device is not None:
+            t = t.float()
+        self.dist.all_reduce(t, op=self.dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def close(self):
+        if self.dist is not None:
+            self.dist.destroy_process_group()
+
+
+def job_throughput(ctx: RankContext, envs_per_rank: int, ms_local: float, steps: int):
+    """(ms per step = the slowest rank's, whole-job chunks/s = the environments all ranks processed / that time)."""
+    ms_step = ctx.max_over_ranks(ms_local) / steps
+    return ms_step, ctx.world * envs_per_rank / (ms_step * 1e-3)
+
+
+def run_stub(args):
+    """The rank plumbing of run_ours with the GPU step replaced by a sleep (tests only)."""
+    from paper_2609_27547_b200 import synth
+    ctx = RankContext("gloo")
+    w = synth.WORKLOADS[args.config]
+    if args.envs:
+        w = synth.scaled(w, B=args.envs)
+    seed = args.seed or synth.DEFAULT_SEED
+    ids = ctx.shard(w.B)
+    groups = synth.arrival_groups(w, seed + ctx.rank, env_ids=ids)
+    assert sorted(e for g in groups for e in g) == ids
+    ctx.barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        time.sleep((args.stub_step_ms + ctx.rank) * 1e-3)
+    ms = (time.perf_counter() - t0) * 1e3
+    ctx.barrier()
+    ms_step, value = job_throughput(ctx, w.B, ms, args.steps)
+    if ctx.dist is not None:
+        gathered = [None] * ctx.world
+        ctx.dist.all_gather_object(gathered, ids)
+    else:
+        gathered = [ids]
+    if ctx.rank == 0:
+        print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": ctx.world, "steps": args.steps,
+                          "warmup": 0, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                          "data": "stub", "config": {"workload": "configs[%d] %s" % (args.config, w.name), "envs_per_gpu": w.B},
+                          "shards": gathered, "gpu_launches": 0}))
+    ctx.close()
+
+
+def launch_ranks(args):
+    """`--gpus N` outside torchrun: start N ranks of this script on this node."""
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    raise SystemExit(subprocess.call(cmd))
+
+
+def run_ours(args, emit=True):
     import torch
-    import torch.distributed as dist
     from paper_2609_27547_b200 import binding as B
     from paper_2609_27547_b200 import synth
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
+    ctx = RankContext("nccl", dev)
+    world, rank = ctx.world, ctx.rank
 
     w = synth.WORKLOADS[args.config]
     if args.envs:
@@ -229,7 +339,7 @@ def run_ours(args):
     peaks = load_peaks()
 
     # this rank's shard: the same workload shape on its own environment ids (weak scaling)
-    ids = [rank * w.B + e for e in range(w.B)]
+    ids = ctx.shard(w.B)
     wt = synth.make_weights(w, seed, device=dev)
     envs = {e: synth.make_env(w, e, seed, device=dev) for e in ids}
     groups = synth.arrival_groups(w, seed + rank, env_ids=ids)
@@ -244,11 +354,6 @@ def run_ours(args):
     gen = B.ActGen(cfg, wt)
     stream = torch.cuda.Stream(dev)
 
-    co_stream, co_buf = None, None
-    if args.corunner and q_eff < N_SMS:
-        co_stream = torch.cuda.Stream(dev)
-        co_buf = torch.zeros(1 << 29, dtype=torch.float32, device=dev)   # 2 GiB
-
     def step():
         for g in groups:
             lo = pos[g[0]]
@@ -256,68 +361,100 @@ def run_ours(args):
                        stream=stream, step_index=[envs[e].step for e in g])
         gen.sync()
 
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize(dev)
-
     n_warm = max(args.min_warmup, args.warmup)
+    tw0 = time.perf_counter()
     for _ in range(n_warm):
         step()
+    torch.cuda.synchronize(dev)
+    warm_ms_step = (time.perf_counter() - tw0) * 1e3 / max(1, n_warm)
+
+    # the synthetic simulation co-runner on the SMs outside the quota: one launch sized (from the
+    # warm-up step time and a timed pass of its own) to outlast the timed region
+    co = None
+    if args.corunner and q_eff < N_SMS:
+        co_stream = gen.rest_stream(quota) if args.green_ctx else None
+        fenced = co_stream is not None
+        if co_stream is None:
+            co_stream = torch.cuda.Stream(dev)
+        co_buf = torch.zeros(1 << 29, dtype=torch.float32, device=dev)   # 2 GiB: 4 GiB of traffic per pass
+        c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        c0.record(co_stream)
+        B.sim_corunner_launch(co_buf, 2, N_SMS - q_eff, co_stream)
+        c1.record(co_stream)
+        torch.cuda.synchronize(dev)
+        pass_ms_alone = c0.elapsed_time(c1) / 2
+        co_passes = max(4, int(3.0 * warm_ms_step * args.steps / max(pass_ms_alone, 1e-3)) + 2)
+        co = {"stream": co_stream, "buf": co_buf, "passes": co_passes, "fenced": fenced, "pass_ms_alone": pass_ms_alone,
+              "e0": torch.cuda.Event(enable_timing=True), "e1": torch.cuda.Event(enable_timing=True)}
+
     gen.reset_stats()
-    barrier()
+    ctx.barrier()
     sampler = ClockSampler(local)
-    if co_stream is not None:
-        B.sim_corunner_launch(co_buf, 8 * args.steps, N_SMS - q_eff, co_stream)
+    if co is not None:
+        co["e0"].record(co["stream"])
+        B.sim_corunner_launch(co["buf"], co["passes"], N_SMS - q_eff, co["stream"])
+        co["e1"].record(co["stream"])
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
     for _ in range(args.steps):
         step()
     e1.record(stream)
-    barrier()
+    co_outlasted = (not co["e1"].query()) if co is not None else None   # still running when the last step's sync returned
+    ctx.barrier()
     clocks = sampler.stop()
     ms = e0.elapsed_time(e1)
     st0 = gen.stats()
     launches = st0["kernel_launches"]
-    if world > 1:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    ms_step = ms / args.steps
-    value = world * w.B / (ms_step * 1e-3)
+    ms_step, value = job_throughput(ctx, w.B, ms, args.steps)
+    co_report = None
+    if co is not None:
+        torch.cuda.synchronize(dev)
+        co_ms = co["e0"].elapsed_time(co["e1"])
+        co_report = {"ctas": N_SMS - q_eff, "passes": co["passes"], "gb_per_pass": 2 * co["buf"].numel() * 4 / 1e9,
+                     "achieved_gbs": co["passes"] * 2 * co["buf"].numel() * 4 / (co_ms * 1e-3) / 1e9,
+                     "alone_gbs": 2 * co["buf"].numel() * 4 / (co["pass_ms_alone"] * 1e-3) / 1e9,
+                     "outlasted_timed_region": bool(co_outlasted),
+                     "placement": "remainder SM partition (driver-enforced)" if co["fenced"] else
+                                  "primary context: only the grid sizes keep the two apart, the driver may place its CTAs anywhere"}
 
     # ---- roofline of the dominant kernel class: a second pass with events around every launch
     gen.reset_stats()
     gen.set_timing(True)
+    sampler2 = ClockSampler(local)
     for _ in range(args.steps):
         step()
+    clocks2 = sampler2.stop()
     st = gen.stats()
     gen.set_timing(False)
     cls = st["classes"]
     total_ms = sum(c["ms"] for c in cls.values()) or 1.0
     gemm = cls["gemm"]
     bf16 = w.dtype == "bf16"
-    if bf16:
-        peak = peaks["bf16_tflops"] * q_eff / N_SMS
-        peak_note = "%s bf16 burst %.1f TFLOP/s x quota %d/%d" % (peaks["source"], peaks["bf16_tflops"], q_eff, N_SMS)
-        bound = "tensor"
-    else:
-        peak = FP32_ALU_TFLOPS * q_eff / N_SMS
-        peak_note = "fp32 FFMA 148 SMs x 128 lanes x 2 x 1.965 GHz = %.1f TFLOP/s x quota %d/%d" % (FP32_ALU_TFLOPS, q_eff, N_SMS)
-        bound = "alu"
+    use_tensor = bf16 and not args.simt
+    mhz = clocks2.get("sm_mhz") or clocks.get("sm_mhz") or 1965.0
+    per_clk = BF16_FLOP_PER_CLK_SM if use_tensor else FP32_FLOP_PER_CLK_SM
+    peak_clock = q_eff * per_clk * mhz * 1e6 / 1e12
     achieved = gemm["flops"] / (gemm["ms"] * 1e-3) / 1e12 if gemm["ms"] > 0 else 0.0
-    # DRAM traffic per GEMM launch from the ncu capture of one layer of this model at M = 8192 rows
-    # (the committed summary of that capture sits with the other profiles): 0.117 GB of weights per layer, which do not grow with M, plus
-    # 0.971 GB of activations, which grow in proportion to the rows; six launches per layer.
-    traffic, traffic_note = None, None
-    if bf16 and (w.d, w.L, w.H, w.mlp_mult) == (2048, 8, 16, 4) and gemm["launches"] > 0:
-        rows_per_launch = st["env_steps"] * w.H / (gemm["launches"] / 6.0 / w.L)
-        traffic = (0.117e9 + 0.971e9 * rows_per_launch / 8192.0) / 6.0
-        traffic_note = "bytes per launch, ncu capture at M=8192 scaled to M=%d (activation part in proportion)" % round(rows_per_launch)
-    roofline = {"bound": bound, "kernel": "gemm", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                "frac": achieved / peak if peak else None, "traffic": traffic, "traffic_note": traffic_note,
+    if use_tensor:
+        bound = "tensor"
+        alt = {"measured_burst_x_quota": peaks["bf16_tflops"] * q_eff / N_SMS,
+               "measured_sustained_x_quota": peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) * q_eff / N_SMS,
+               "nominal_2250_x_quota": NOMINAL_BF16_TFLOPS * q_eff / N_SMS}
+        peak_note = ("%d SMs x %d FLOP/clk x %.0f MHz (median SM clock sampled during the per-kernel timing pass); the %s full-chip "
+                     "figures (burst %.1f, sustained %.1f TFLOP/s, taken at a power-capped clock) scaled by %d/%d are in frac_vs"
+                     % (q_eff, per_clk, mhz, peaks["source"], peaks["bf16_tflops"],
+                        peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]), q_eff, N_SMS))
+    else:
+        bound = "alu"
+        alt = {"fp32_ffma_at_max_clock_x_quota": FP32_ALU_TFLOPS * q_eff / N_SMS}
+        peak_note = "%d SMs x 128 FFMA lanes x 2 x %.0f MHz (median SM clock sampled during the per-kernel timing pass)" % (q_eff, mhz)
+    traffic, traffic_note = gemm_traffic(w, st, gemm)
+    roofline = {"bound": bound, "kernel": "gemm", "achieved": achieved, "peak": peak_clock, "unit": "TFLOP/s",
+                "frac": achieved / peak_clock if peak_clock else None,
+                "frac_vs": {k: achieved / v for k, v in alt.items()}, "peak_alternatives": alt,
+                "traffic": traffic, "traffic_note": traffic_note,
                 "algorithmic_bytes_per_launch": gemm["bytes"] / gemm["launches"] if gemm["launches"] else None,
-                "peak_source": peak_note,
+                "peak_source": peak_note, "clocks_timing_pass": clocks2,
                 "launches": gemm["launches"], "avg_launch_us": 1e3 * gemm["ms"] / max(1, gemm["launches"]),
                 "class_share": {k: round(c["ms"] / total_ms, 4) for k, c in cls.items()},
                 "class_ms_per_step": {k: round(c["ms"] / args.steps, 4) for k, c in cls.items()}}
@@ -325,15 +462,22 @@ def run_ours(args):
     if xa["ms"] > 0:
         roofline["cross_attn_hbm"] = {"achieved_gbs": xa["bytes"] / (xa["ms"] * 1e-3) / 1e9, "peak_gbs": peaks["hbm_gbs"],
                                       "frac": xa["bytes"] / (xa["ms"] * 1e-3) / 1e9 / peaks["hbm_gbs"]}
-    # whole-path fraction of the quota-scaled roofline (the metric's second half)
+    # whole-path fraction of the quota-scaled roofline (the metric's second half): the slower of every FLOP at the
+    # tensor (or ALU) rate of the quota's SMs and the compulsory bytes at the measured HBM bandwidth, over the step time
     flops_step = workload_flops(w, [envs[e] for e in ids])
-    t_tensor = flops_step / (peak * 1e12)
     min_bytes = kv_bytes + 2 * noise.numel() * 4 + sum(t.numel() * t.element_size() for t in
                                                        [wt["w_in"], wt["w_out"]] + [v for l in wt["layers"] for v in l.values()])
     t_hbm = min_bytes / (peaks["hbm_gbs"] * 1e9)
-    path = {"flops_per_step": flops_step, "t_roof_ms": 1e3 * max(t_tensor, t_hbm), "frac": max(t_tensor, t_hbm) / (ms_step * 1e-3),
-            "frac_vs_sustained": (flops_step / (peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) * 1e12 * q_eff / N_SMS)) / (ms_step * 1e-3)
-            if bf16 else None}
+    mhz1 = clocks.get("sm_mhz") or mhz
+    path_peaks = {"clock_scaled": q_eff * per_clk * mhz1 * 1e6 / 1e12}
+    path_peaks.update(alt)
+    path = {"flops_per_step": flops_step, "min_bytes_per_step": min_bytes,
+            "frac": max(flops_step / (path_peaks["clock_scaled"] * 1e12), t_hbm) / (ms_step * 1e-3),
+            "frac_vs": {k: max(flops_step / (v * 1e12), t_hbm) / (ms_step * 1e-3) for k, v in path_peaks.items() if k != "clock_scaled"},
+            "t_roof_ms": {k: 1e3 * max(flops_step / (v * 1e12), t_hbm) for k, v in path_peaks.items()},
+            "note": "frac: against %d SMs x %d FLOP/clk x the %.0f MHz sampled during the timed steps; "
+                    "frac_vs.measured_burst_x_quota is the metric's 'quota-scaled bf16 tensor roofline' with the measured full-chip peak"
+                    % (q_eff, per_clk, mhz1)}
 
     # ---- end to end through the host-buffer entry point
     e2e = None
@@ -351,21 +495,17 @@ def run_ours(args):
 
         n_e2e = max(1, min(args.steps, 3))
         step_host()
-        barrier()
+        ctx.barrier()
         a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         t0 = time.perf_counter()
         a0.record(stream)
         for _ in range(n_e2e):
             step_host()
         a1.record(stream)
-        barrier()
+        ctx.barrier()
         wall = (time.perf_counter() - t0) / n_e2e
-        ems = a0.elapsed_time(a1) / n_e2e   # device-side span; the wall time is reported beside it
-        if world > 1:
-            t = torch.tensor([ems], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ems = float(t.item())
-        e2e = {"value": world * w.B / (ems * 1e-3), "unit": UNIT, "h2d_bytes_per_step": kv_bytes + noise.numel() * 4,
+        ems, evalue = job_throughput(ctx, w.B, a0.elapsed_time(a1), n_e2e)   # device-side span; the wall time is reported beside it
+        e2e = {"value": evalue, "unit": UNIT, "h2d_bytes_per_step": kv_bytes + noise.numel() * 4,
                "d2h_bytes_per_step": noise.numel() * 4, "ms_per_step": ems, "wall_ms_per_step": wall * 1e3, "steps": n_e2e,
                "equal_to_device_path": bool(torch.equal(h_out.to(dev), out))}
 
@@ -376,6 +516,7 @@ def run_ours(args):
         cpu = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
 
     gen.destroy()
+    line = None
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": n_warm,
@@ -384,17 +525,55 @@ def run_ours(args):
             "config": {"workload": "configs[%d] %s" % (args.config, w.name), "envs_per_gpu": w.B, "H": w.H, "A": w.A, "d": w.d,
                        "L": w.L, "heads": w.n_heads, "P": list(w.P), "K": w.K, "d_ctx": w.d_ctx, "groups": len(groups),
                        "group_sizes": [min(map(len, groups)), max(map(len, groups))], "sm_quota": q_eff,
-                       "inflight_groups": inflight, "corunner": bool(co_stream is not None),
+                       "inflight_groups": inflight, "corunner": co_report if co_report is not None else False,
                        "green_ctx": {"requested": bool(args.green_ctx), "active": bool(st0["green_ctx_active"]), "partition_sms": st0["green_ctx_sms"]},
+                       "sharding": "environment id mod %d; no data-path collective" % world,
                        "l2": ("inputs (%.2f GB of prefix planes plus weights) larger than the 126 MB L2" % (kv_bytes / 1e9))
                        if kv_bytes > 126e6 else "inputs fit in L2 and L2 is not flushed: small parity-size case, not a bench line",
                        "seed": seed},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "path_roofline": path,
             "cpu_baseline": cpu,
         }
-        print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+        if emit:
+            print(json.dumps(line))
+    ctx.close()
+    return line
+
+
+def gemm_traffic(w, st, gemm):
+    """DRAM bytes per GEMM launch from the ncu capture recorded beside the other profile summaries
+    (a capture of one layer's six GEMMs at a smaller M, scaled to this run's rows: the weight part
+    does not grow with M, the activation part grows in proportion).  None when no capture covers
+    this model."""
+    path = os.path.join(ROOT, "profiles", "gemm_dram_traffic.json")
+    if not os.path.exists(path) or gemm["launches"] <= 0:
+        return None, None
+    with open(path) as f:
+        rec = json.load(f)
+    for c in rec.get("captures", []):
+        m = c["model"]
+        if (m["d"], m["L"], m["H"], m["mlp_mult"], m["dtype"]) == (w.d, w.L, w.H, w.mlp_mult, w.dtype):
+            rows = st["env_steps"] * w.H / (gemm["launches"] / float(c["gemms_per_layer"]) / w.L)
+            per_layer = c["weight_bytes_per_layer"] + c["activation_bytes_per_layer"] * rows / c["rows"]
+            return per_layer / c["gemms_per_layer"], ("bytes per launch: %s, M=%d scaled to M=%d (activation part in proportion)"
+                                                       % (c["source"], c["rows"], round(rows)))
+    return None, None
+
+
+def run_sweep(args):
+    """One JSON line per other configuration (the bench line proper is configs[4])."""
+    import copy
+    plan = [(0, 0, False), (1, 0, False), (2, 0, False)]
+    for q in (148, 74, 37, 16):
+        plan.append((3, q, False))
+        if q < N_SMS:
+            plan.append((3, q, True))
+    for cfg_i, q, co in plan:
+        a = copy.copy(args)
+        a.config, a.corunner, a.no_cpu, a.no_e2e = cfg_i, co, True, True
+        a.quota = q if cfg_i == 3 else -1
+        a.steps = max(args.steps, 20) if cfg_i != 1 else max(args.steps, 10)
+        run_ours(a)
 
 
 def run_pgen_sweep(args):
@@ -440,6 +619,12 @@ def run_pgen_sweep(args):
 
 def main():
     args = parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        return launch_ranks(args)
+    if args.stub_step_ms > 0:
+        return run_stub(args)
+    if args.sweep:
+        return run_sweep(args)
     if args.pgen_sweep:
         return run_pgen_sweep(args)
     if args.rollout_sim:

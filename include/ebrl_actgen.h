@@ -153,7 +153,9 @@ typedef struct {
     uint64_t weights_version;             /* policy version the last launched batch ran with   */
 } ebrl_actgen_stats_t;
 
-/* Validates cfg, copies the weights to the device (re-laid-out as the kernels want), builds
+/* A generation worker for one policy (section 2.1: the action head that denoises a random tensor
+ * into an action chunk; section 4.2.1: generation is a stage of its own with its own resources).
+ * Validates cfg, copies the weights to the device (re-laid-out as the kernels want), builds
  * the timestep-embedding table, allocates max_inflight_groups workspaces of
  * max_group_envs * H rows.  Supported: d a multiple of 256 (tensor-core path) or of 64
  * (plain path), d even, H <= 32, A <= 32, head_dim in {32, 64, 128} ...; anything else
@@ -236,19 +238,38 @@ uint64_t ebrl_actgen_weights_version(ebrl_actgen_t h);
 /* Launches the queued groups now, without blocking. */
 ebrl_status_t ebrl_actgen_flush(ebrl_actgen_t h);
 
-/* Launches the queued groups, then blocks until every submitted group has completed; returns
- * the first sticky error. */
+/* The point where the consumer of the action chunks (the simulation stage of section 4.2.2, which
+ * needs an environment's chunk before it can step that environment) waits for generation: launches
+ * the queued groups, then blocks until every submitted group has completed; returns the first
+ * sticky error. */
 ebrl_status_t ebrl_actgen_sync(ebrl_actgen_t h);
 
-/* Syncs, then frees everything the handle owns. */
+/* Ends the generation worker (section 4.2.1: stages are created and retired by the scheduler as
+ * resources are re-divided): syncs, then frees everything the handle owns. */
 ebrl_status_t ebrl_actgen_destroy(ebrl_actgen_t h);
 
 /* Library-owned, NUL-terminated text of the last error on this handle (or of the last failed
  * create when h is NULL); valid until the next call on the same handle. */
 const char *ebrl_actgen_last_error(ebrl_actgen_t h);
 
+/* Counters and per-kernel-class device time since create or the last reset: the measurements the
+ * generation profile P_gen(s_g, B_g) of section 4.3.2 is built from (throughput per SM quota and
+ * batch size).  A single device_ns total is not kept; class_ms splits it by kernel class. */
 ebrl_status_t ebrl_actgen_get_stats(ebrl_actgen_t h, ebrl_actgen_stats_t *out_stats);
 ebrl_status_t ebrl_actgen_reset_stats(ebrl_actgen_t h);
+
+/* SM partitions behind the quota (sections 4.2.1 and 4.3.1: stages share a GPU under separate logical
+ * SM quotas).  With EBRL_FLAG_GREEN_CTX a submit with 0 < sm_quota < #SMs runs inside a driver
+ * partition of *out_gen_sms SMs -- the quota rounded UP to the driver's granularity (8 SMs on B200:
+ * 74 -> 80, 37 -> 40) -- while its grids stay capped at exactly sm_quota CTAs: "quota" is the number of
+ * SMs the generator keeps busy, the partition is the fence around them.  The SMs outside it form the
+ * complementary partition of *out_rest_sms SMs; *out_rest_stream is a cudaStream_t owned by the handle
+ * (valid until destroy) whose kernels can only run there, which is where a co-running stage (the
+ * simulator stand-in of the bench) belongs so that the driver keeps the two apart in both directions.
+ * All three are 0 / NULL when the flag is off, the quota is the whole chip or the driver offers no
+ * partitions; any of the out pointers may be NULL.  The partition of a quota is created on first use. */
+ebrl_status_t ebrl_actgen_partition_info(ebrl_actgen_t h, int32_t sm_quota, int32_t *out_gen_sms, int32_t *out_rest_sms,
+                                         void **out_rest_stream);
 
 /* Switches the per-kernel-class timing (EBRL_FLAG_TIMING) on or off for later submits. */
 ebrl_status_t ebrl_actgen_set_timing(ebrl_actgen_t h, int32_t on);

@@ -117,6 +117,7 @@ def lib():
         L.ebrl_actgen_get_stats.argtypes = [C.c_void_p, C.POINTER(Stats)]
         L.ebrl_actgen_reset_stats.argtypes = [C.c_void_p]
         L.ebrl_actgen_set_timing.argtypes = [C.c_void_p, C.c_int32]
+        L.ebrl_actgen_partition_info.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_int32), C.POINTER(C.c_void_p)]
         L.ebrl_actgen_check_cfg.argtypes = [C.POINTER(Cfg)]
         L.ebrl_actgen_check_submit.argtypes = [C.POINTER(Cfg), C.c_int32, C.c_int32, C.POINTER(C.c_int64),
                                                C.POINTER(C.c_void_p), C.c_void_p, C.c_void_p, C.c_int32,
@@ -285,6 +286,19 @@ class ActGen:
         out["classes"] = {n: {"ms": s.class_ms[i], "launches": s.class_launches[i], "flops": s.class_flops[i],
                               "bytes": s.class_bytes[i]} for i, n in enumerate(KC_NAMES)}
         return out
+
+    def partition_info(self, sm_quota: int):
+        """``ebrl_actgen_partition_info``: (SMs of the quota's partition, SMs of the complementary one, its stream handle or None)."""
+        g, r, st = C.c_int32(0), C.c_int32(0), C.c_void_p()
+        self._check(self._L.ebrl_actgen_partition_info(self._h, int(sm_quota), C.byref(g), C.byref(r), C.byref(st)))
+        return g.value, r.value, st.value
+
+    def rest_stream(self, sm_quota: int) -> Optional[torch.cuda.Stream]:
+        """The complementary partition's stream as a torch stream (None when there is no partition)."""
+        _, rest, st = self.partition_info(sm_quota)
+        if not st or rest < 1:
+            return None
+        return torch.cuda.ExternalStream(st, device=torch.device("cuda", self.cfg.device))
 
     def reset_stats(self):
         self._check(self._L.ebrl_actgen_reset_stats(self._h))

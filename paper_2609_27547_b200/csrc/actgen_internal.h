@@ -114,13 +114,16 @@ cudaError_t launch_gemm_tc2(const TensorMap128 &ta, const TensorMap128 &tw, cons
 // Tensor-core (mma.sync) attention over bulk-copied K/V rows, bf16 models.
 bool attn_mma_supported(int H, int n_heads, int hd);
 int attn_mma_make_map(TensorMap128 *out, const void *base, uint64_t rows, uint64_t width, int n_heads, int hd);
-cudaError_t launch_attn_mma(const AttnArgs &a, int grid, unsigned long long limit_ns, int *status, cudaStream_t st);
+cudaError_t launch_attn_mma(const AttnArgs &a, int grid, int lookahead_blocks, unsigned long long limit_ns, int *status, cudaStream_t st);
 
 // An SM partition (green context) with a stream inside it.
 struct GreenPartition {
     void *ctx = nullptr;
     cudaStream_t stream = nullptr;
     int sm_count = 0;
+    void *rest_ctx = nullptr;          // the complementary partition: every SM not in `ctx`
+    cudaStream_t rest_stream = nullptr;
+    int rest_sm_count = 0;
 };
 int green_partition_create(int device, int sm_quota, GreenPartition *out);
 void green_partition_destroy(GreenPartition *p);
@@ -132,7 +135,7 @@ void green_partition_destroy(GreenPartition *p);
 // unchanged; only the launch latency and the set-up move off the critical path.  The attribute is
 // used only for batches whose grid fills every SM their stream can reach: under a smaller SM quota
 // the early CTAs would park on SMs outside the quota (and measured slower).  pdl_set() states the
-// choice for the calling thread's next launches; EBRL_PDL=0 turns the attribute off altogether.
+// choice for the calling thread's next launches (a handle created with EBRL_PDL=0 never turns it on).
 void pdl_set(bool on);
 bool pdl_enabled();
 template <typename... KArgs, typename... Args>

@@ -23,12 +23,7 @@ using namespace ebrl;
 namespace ebrl {
 static thread_local bool t_pdl = false;
 void pdl_set(bool on) { t_pdl = on; }
-bool pdl_enabled()
-{
-    static int allowed = -1;
-    if (allowed < 0) { const char *e = getenv("EBRL_PDL"); allowed = (e && atoi(e) == 0) ? 0 : 1; }
-    return allowed != 0 && t_pdl;
-}
+bool pdl_enabled() { return t_pdl; }
 }  // namespace ebrl
 
 namespace {
@@ -106,6 +101,8 @@ struct ebrl_actgen {
     bool use_tc = false;          // tensor-core GEMMs (bf16, d a multiple of 256)
     bool use_pairs = true;        // CTA-pair GEMM allowed (EBRL_GEMM_PAIR=0 forbids it)
     int force_shape = 0;          // EBRL_GEMM_SHAPE = 2 (pairs), 256 or 128 forces one tile shape (tests, tuning)
+    bool pdl_allowed = true;      // EBRL_PDL=0 turns programmatic dependent launch off
+    int attn_lookahead = 2;       // EBRL_ATTN_LOOKAHEAD: key blocks the attention producer asks L2 for ahead of its ring
     bool use_attn_mma = false;    // tensor-core attention (bf16, H <= 16, head_dim 64/128)
     int *status_d = nullptr;      // device status word written by kernels whose waits ran out
     unsigned long long wait_ns = 0;
@@ -374,6 +371,18 @@ ebrl_status_t retire(ebrl_actgen *h, Slot &s)
     return EBRL_OK;
 }
 
+// The SM partition of a quota (created on first use, cached per quota); nullptr when the driver has none.
+GreenPartition *partition_for(ebrl_actgen *h, int quota)
+{
+    auto it = h->partitions.find(quota);
+    if (it == h->partitions.end()) {
+        GreenPartition np;
+        if (green_partition_create(h->cfg.device, quota, &np) != 0) np = GreenPartition();
+        it = h->partitions.emplace(quota, np).first;
+    }
+    return it->second.ctx ? &it->second : nullptr;
+}
+
 struct Launcher {
     ebrl_actgen *h;
     Slot *slot;
@@ -405,7 +414,7 @@ struct Launcher {
 
 cudaError_t launch_attn(ebrl_actgen *h, const AttnArgs &a, int grid, cudaStream_t st)
 {
-    if (h->use_attn_mma) return launch_attn_mma(a, grid, h->wait_ns, h->status_d, st);
+    if (h->use_attn_mma) return launch_attn_mma(a, grid, h->attn_lookahead, h->wait_ns, h->status_d, st);
     return launch_attn_simt(a, h->bf16, grid, st);
 }
 
@@ -591,15 +600,7 @@ ebrl_status_t flush_slot(ebrl_actgen *h, Slot &s)
     // SM partition: the batch runs on the partition's stream, fenced against the caller's stream by events
     cudaStream_t user = cs;
     GreenPartition *gp = nullptr;
-    if ((c.flags & EBRL_FLAG_GREEN_CTX) && s.grid < h->n_sms) {
-        auto it = h->partitions.find(s.grid);
-        if (it == h->partitions.end()) {
-            GreenPartition np;
-            if (green_partition_create(c.device, s.grid, &np) != 0) np = GreenPartition();
-            it = h->partitions.emplace(s.grid, np).first;
-        }
-        if (it->second.ctx) gp = &it->second;
-    }
+    if ((c.flags & EBRL_FLAG_GREEN_CTX) && s.grid < h->n_sms) gp = partition_for(h, s.grid);
     if (gp) {
         CK(cudaEventRecord(s.part_in, user));
         CK(cudaStreamWaitEvent(gp->stream, s.part_in, 0));
@@ -623,7 +624,7 @@ ebrl_status_t flush_slot(ebrl_actgen *h, Slot &s)
         for (int j = 0; j < n; ++j) s.maps_h[j] = maps_packed[j];
         CK(cudaMemcpyAsync(s.maps_d + 1, s.maps_h, sizeof(TensorMap128) * (size_t)n, cudaMemcpyHostToDevice, cs));
     }
-    pdl_set(s.grid >= (gp ? gp->sm_count : h->n_sms));
+    pdl_set(h->pdl_allowed && s.grid >= (gp ? gp->sm_count : h->n_sms));
     cudaError_t e = enqueue_batch(h, s, S, n_active.data(), sum_P.data(), s.grid, cs);
     pdl_set(false);
     if (e != cudaSuccess) {
@@ -908,6 +909,8 @@ ebrl_status_t ebrl_actgen_create(const ebrl_actgen_cfg_t *cfg, const ebrl_actgen
                 gemm_tc_supported(d, md) && gemm_tc_supported(3 * d, d);
     if (const char *e2 = getenv("EBRL_GEMM_PAIR")) h->use_pairs = atoi(e2) != 0;
     if (const char *e3 = getenv("EBRL_GEMM_SHAPE")) { const int v = atoi(e3); if (v == 2 || v == 256 || v == 128) h->force_shape = v; }
+    if (const char *e4 = getenv("EBRL_PDL")) h->pdl_allowed = atoi(e4) != 0;
+    if (const char *e5 = getenv("EBRL_ATTN_LOOKAHEAD")) h->attn_lookahead = std::min(64, std::max(0, atoi(e5)));
     h->use_attn_mma = h->bf16 && !(cfg->flags & EBRL_FLAG_FORCE_SIMT) && attn_mma_supported(cfg->H, cfg->n_heads, h->hd);
     if ((st = alloc_weight_set(h, h->wset[0])) != EBRL_OK) return bail(st);
     if ((st = upload_weight_set(h, h->wset[0], wts, nullptr, false)) != EBRL_OK) return bail(st);
@@ -1125,6 +1128,24 @@ uint64_t ebrl_actgen_weights_version(ebrl_actgen_t h)
     if (!h) return 0;
     std::lock_guard<std::mutex> lk(h->mu);
     return h->version;
+}
+
+ebrl_status_t ebrl_actgen_partition_info(ebrl_actgen_t h, int32_t sm_quota, int32_t *out_gen_sms, int32_t *out_rest_sms, void **out_rest_stream)
+{
+    if (!h) return EBRL_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lk(h->mu);
+    if (out_gen_sms) *out_gen_sms = 0;
+    if (out_rest_sms) *out_rest_sms = 0;
+    if (out_rest_stream) *out_rest_stream = nullptr;
+    if (sm_quota < 1 || sm_quota > h->n_sms) return fail(h, EBRL_ERR_QUOTA, "sm_quota outside 1..#SMs");
+    if (!(h->cfg.flags & EBRL_FLAG_GREEN_CTX) || sm_quota >= h->n_sms) return EBRL_OK;   // no partition is used for such submits
+    CK(cudaSetDevice(h->cfg.device));
+    const GreenPartition *gp = partition_for(h, sm_quota);
+    if (!gp) return EBRL_OK;
+    if (out_gen_sms) *out_gen_sms = gp->sm_count;
+    if (out_rest_sms) *out_rest_sms = gp->rest_sm_count;
+    if (out_rest_stream) *out_rest_stream = (void *)gp->rest_stream;
+    return EBRL_OK;
 }
 
 ebrl_status_t ebrl_actgen_set_timing(ebrl_actgen_t h, int32_t on)

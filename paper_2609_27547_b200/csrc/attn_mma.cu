@@ -405,7 +405,8 @@ int attn_mma_make_map(TensorMap128 *out, const void *base, uint64_t rows, uint64
     return r == CUDA_SUCCESS ? 0 : 2;
 }
 
-cudaError_t launch_attn_mma(const AttnArgs &a, int grid, unsigned long long limit_ns, int *status, cudaStream_t st)
+// la = L2 look-ahead of the producer in key blocks (0 disables).
+cudaError_t launch_attn_mma(const AttnArgs &a, int grid, int la, unsigned long long limit_ns, int *status, cudaStream_t st)
 {
     const int hpc = a.n_heads < am::MAXW ? a.n_heads : am::MAXW;
     const int items = a.n_envs * (a.n_heads / hpc);
@@ -413,14 +414,6 @@ cudaError_t launch_attn_mma(const AttnArgs &a, int grid, unsigned long long limi
     const int g = items < grid ? items : grid;
     const int W = hpc * a.hd;
     const size_t smem = (size_t)2 * am::NSTAGE * am::stage_keys(W) * (W / 64) * 128 + (size_t)am::MAXW * 16 * a.hd * 2 + 64 + 1024;
-    // L2 look-ahead of the producer in key blocks (EBRL_ATTN_LOOKAHEAD overrides; 0 disables)
-    static int la = -1;
-    if (la < 0) {
-        const char *env = getenv("EBRL_ATTN_LOOKAHEAD");
-        la = env ? atoi(env) : 2;
-        if (la < 0) la = 0;
-        if (la > 64) la = 64;
-    }
     cudaError_t e;
     if (a.hd == 128) {
         e = cudaFuncSetAttribute(am::attn_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

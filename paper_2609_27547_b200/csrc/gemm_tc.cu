@@ -249,11 +249,14 @@ template <int EPI, int BN>
 static cudaError_t tc_launch(const TensorMap128 &ta, const TensorMap128 &tw, const TensorMap128 &tc_, const GemmArgs &a, int g,
                              unsigned long long limit_ns, int *status, cudaStream_t st)
 {
-    static bool attr_set = false;
-    if (!attr_set) {
+    // the attribute belongs to the function on ONE device: set it once per device
+    static bool attr_set[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!attr_set[dev]) {
         cudaError_t e = cudaFuncSetAttribute(tc::gemm_tc_kernel<EPI, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::Shape<BN>::SMEM_BYTES);
         if (e != cudaSuccess) return e;
-        attr_set = true;
+        attr_set[dev] = true;
     }
     return launch_kernel(tc::gemm_tc_kernel<EPI, BN>, g, tc::Shape<BN>::THREADS, tc::Shape<BN>::SMEM_BYTES, st, 1,
                          *reinterpret_cast<const CUtensorMap *>(&ta), *reinterpret_cast<const CUtensorMap *>(&tw),

@@ -231,11 +231,14 @@ template <int EPI>
 static cudaError_t tc2_launch(const TensorMap128 &ta, const TensorMap128 &tw, const TensorMap128 &tc_, const GemmArgs &a, int g,
                               unsigned long long limit_ns, int *status, cudaStream_t st)
 {
-    static bool attr_set = false;
-    if (!attr_set) {
+    // the attribute belongs to the function on ONE device: set it once per device
+    static bool attr_set[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!attr_set[dev]) {
         cudaError_t e = cudaFuncSetAttribute(tc2::gemm_tc2_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, tc2::SMEM_BYTES);
         if (e != cudaSuccess) return e;
-        attr_set = true;
+        attr_set[dev] = true;
     }
     return launch_kernel(tc2::gemm_tc2_kernel<EPI>, g, tc2::THREADS, tc2::SMEM_BYTES, st, 2, *reinterpret_cast<const CUtensorMap *>(&ta),
                          *reinterpret_cast<const CUtensorMap *>(&tw), *reinterpret_cast<const CUtensorMap *>(&tc_), a, limit_ns, status);

@@ -49,8 +49,10 @@ const Api &api()
 }  // namespace
 
 // Creates a partition of at least `sm_quota` SMs on `device` and a stream in it.  Returns 0 on
-// success; *sm_count is the number of SMs the driver actually put in the partition (it rounds up
-// to its granularity).
+// success; sm_count is the number of SMs the driver actually put in the partition (it rounds up
+// to its granularity).  The SMs left over become a second partition with a stream of its own
+// (rest_*; absent when nothing is left or the driver refuses it): work launched there cannot
+// reach the first partition's SMs, which is how a co-running stage is fenced OUT of the quota.
 int green_partition_create(int device, int sm_quota, GreenPartition *out)
 {
     const Api &a = api();
@@ -73,6 +75,23 @@ int green_partition_create(int device, int sm_quota, GreenPartition *out)
     out->ctx = ctx;
     out->stream = (cudaStream_t)st;
     out->sm_count = (int)part.sm.smCount;
+    out->rest_ctx = nullptr;
+    out->rest_stream = nullptr;
+    out->rest_sm_count = 0;
+    if (rest.sm.smCount > 0) {
+        CUdevResourceDesc rdesc;
+        CUgreenCtx rctx;
+        if (a.generateDesc(&rdesc, &rest, 1) == CUDA_SUCCESS && a.greenCreate(&rctx, rdesc, dev, CU_GREEN_CTX_DEFAULT_STREAM) == CUDA_SUCCESS) {
+            CUstream rst;
+            if (a.streamCreate(&rst, rctx, CU_STREAM_NON_BLOCKING, 0) == CUDA_SUCCESS) {
+                out->rest_ctx = rctx;
+                out->rest_stream = (cudaStream_t)rst;
+                out->rest_sm_count = (int)rest.sm.smCount;
+            } else {
+                a.greenDestroy(rctx);
+            }
+        }
+    }
     return 0;
 }
 
@@ -81,9 +100,11 @@ void green_partition_destroy(GreenPartition *p)
     const Api &a = api();
     if (!p || !p->ctx) return;
     if (p->stream) cudaStreamDestroy(p->stream);
+    if (p->rest_stream) cudaStreamDestroy(p->rest_stream);
     if (a.ok) a.greenDestroy((CUgreenCtx)p->ctx);
-    p->ctx = nullptr;
-    p->stream = nullptr;
+    if (a.ok && p->rest_ctx) a.greenDestroy((CUgreenCtx)p->rest_ctx);
+    p->ctx = p->rest_ctx = nullptr;
+    p->stream = p->rest_stream = nullptr;
 }
 
 }  // namespace ebrl

@@ -58,3 +58,32 @@ def test_two_ranks_shard_environments_disjointly():
     w = synth.scaled(synth.WORKLOADS[2], B=50)
     total = sum(float(synth.make_env(w, e).noise.double().sum()) for e in range(50))
     assert abs(sum(g[1] for g in gathered) - total) < 1e-9   # the shards together are the whole job
+
+
+def test_bench_gpus_2_starts_two_ranks_and_aggregates_over_them():
+    """`bench.py --gpus 2` outside torchrun starts its own two ranks.  With the GPU step replaced by
+    a sleep (--stub-step-ms: rank r sleeps 30 + r ms per step) the rank plumbing runs on CPU over
+    gloo: disjoint id-mod-world shards of 2 x B environments, the step time is the slowest rank's,
+    and `value` counts the environments of both ranks."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--config", "2", "--envs", "50",
+                        "--steps", "4", "--stub-step-ms", "30"], capture_output=True, text=True, timeout=300, env=env)
+    assert p.returncode == 0, p.stderr[-2000:]
+    lines = [l for l in p.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                                   # rank 0 alone prints
+    d = json.loads(lines[0])
+    assert d["n_gpus"] == 2 and d["data"] == "stub" and d["scaling"] == "weak"
+    a, b = (set(x) for x in d["shards"])
+    assert a.isdisjoint(b) and a | b == set(range(100)) and all(e % 2 == 0 for e in a)
+    assert 31.0 <= d["ms_per_step"] < 60.0                   # the slower rank (31 ms sleeps), not the faster one
+    assert abs(d["value"] - 100 / (d["ms_per_step"] * 1e-3)) < 1e-6 * d["value"]
+
+
+def test_job_throughput_single_rank():
+    import bench
+    ctx = bench.RankContext("gloo")
+    assert ctx.world == 1 and ctx.shard(7) == list(range(7))
+    ms_step, value = bench.job_throughput(ctx, 2048, 5580.0, 10)
+    assert ms_step == 558.0 and abs(value - 2048 / 0.558) < 1e-9
