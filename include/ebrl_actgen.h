@@ -47,7 +47,7 @@
 extern "C" {
 #endif
 
-#define EBRL_ACTGEN_ABI_VERSION 2u
+#define EBRL_ACTGEN_ABI_VERSION 3u
 
 typedef struct ebrl_actgen *ebrl_actgen_t;
 
@@ -71,6 +71,16 @@ typedef enum { EBRL_F32 = 0, EBRL_BF16 = 1 } ebrl_dtype_t;
                                      of sm_quota CTAs applies either way                         */
 #define EBRL_FLAG_TIMING      4u  /* record per-kernel-class device time (see get_stats)        */
 #define EBRL_FLAG_FORCE_SIMT  8u  /* bf16 models: use the plain-ALU kernels, not tensor cores    */
+#define EBRL_FLAG_NO_FUSED   16u  /* never use the persistent step kernel (one resident grid that
+                                     walks all Euler steps of a small batch); always launch one
+                                     kernel per operation                                        */
+#define EBRL_FLAG_FORCE_FUSED 32u /* use the persistent step kernel for every batch the kernel
+                                     covers (bf16 tensor-core models with H a divisor of 128 and
+                                     A <= 16), whatever its size.  Without the flag no batch takes
+                                     it: it delivers the same bits as the per-operation kernels
+                                     but has measured slower on B200 at every batch size tried;
+                                     EBRL_FUSED_MAX_ROWS=<rows> in the environment at create makes
+                                     batches of up to that many rows take it                    */
 
 /* Plain data, copied at create. */
 typedef struct {
@@ -133,7 +143,8 @@ typedef struct {
 /* Kernel classes of the per-class timing (EBRL_FLAG_TIMING). */
 enum { EBRL_KC_EMBED = 0, EBRL_KC_GEMM = 1, EBRL_KC_SELF_ATTN = 2, EBRL_KC_CROSS_ATTN = 3,
        EBRL_KC_HEAD = 4, EBRL_KC_PREFIX = 5 /* packing and projecting hidden-state prefixes */,
-       EBRL_KC_COUNT = 6 };
+       EBRL_KC_FUSED = 6 /* the persistent step kernel: every operation of every Euler step */,
+       EBRL_KC_COUNT = 7 };
 
 typedef struct {
     uint64_t groups, envs, env_steps;     /* submitted since create                            */

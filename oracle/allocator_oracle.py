@@ -68,23 +68,23 @@ def simulator_capacity(sim_quota_pct, sim_rate, knee_tolerance):
 
 def elastic_allocation(N, c_env, sim_quota_pct, sim_rate, gen: Profile, train: Profile, s_g_min, s_t_min, M_gpu,
                        knee_tolerance=0.05):
-    E = N // c_env                                                   # line 2
-    s_sim, T_s = simulator_capacity(sim_quota_pct, sim_rate, knee_tolerance)   # lines 3-4
-    lo, hi = s_g_min, 100 - s_sim - s_t_min                          # line 5
+    E = N // c_env
+    s_sim, T_s = simulator_capacity(sim_quota_pct, sim_rate, knee_tolerance)
+    lo, hi = s_g_min, 100 - s_sim - s_t_min
     assert hi >= lo
     it = 0
-    while hi - lo > 1:                                               # line 6
-        s_g = (lo + hi) // 2                                         # line 7
-        s_t = 100 - s_sim - s_g                                      # line 8
-        c = best_pair(gen, train, s_g, s_t, T_s, M_gpu)              # line 9
-        if c["T_r"] > c["T_t"]:                                      # lines 10-12
+    while hi - lo > 1:
+        s_g = (lo + hi) // 2
+        s_t = 100 - s_sim - s_g
+        c = best_pair(gen, train, s_g, s_t, T_s, M_gpu)
+        if c["T_r"] > c["T_t"]:
             hi = s_g
         else:
             lo = s_g
         it += 1
-    a = best_pair(gen, train, lo, 100 - s_sim - lo, T_s, M_gpu)      # line 18
+    a = best_pair(gen, train, lo, 100 - s_sim - lo, T_s, M_gpu)
     b = best_pair(gen, train, hi, 100 - s_sim - hi, T_s, M_gpu)
-    w = a if a["theta"] >= b["theta"] else b                          # line 19
+    w = a if a["theta"] >= b["theta"] else b
     w.update(E=E, s_sim=s_sim, T_s=T_s, iterations=it)
     return w
 

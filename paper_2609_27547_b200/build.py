@@ -35,7 +35,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     tmp = LIB + ".tmp.%d" % os.getpid()
-    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + sources()
+    extra = os.environ.get("EBRL_NVCC_EXTRA", "").split()    # e.g. -DEBRL_FUSED_PROF for a tuning build
+    cmd = [nvcc] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + sources()
     subprocess.check_call(cmd, cwd=CSRC)
     os.replace(tmp, LIB)
     return LIB

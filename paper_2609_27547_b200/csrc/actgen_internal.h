@@ -116,6 +116,38 @@ bool attn_mma_supported(int H, int n_heads, int hd);
 int attn_mma_make_map(TensorMap128 *out, const void *base, uint64_t rows, uint64_t width, int n_heads, int hd);
 cudaError_t launch_attn_mma(const AttnArgs &a, int grid, int lookahead_blocks, unsigned long long limit_ns, int *status, cudaStream_t st);
 
+// ---- the persistent step kernel (one resident grid for all Euler steps of a small batch) ----
+// Per-layer table in device memory: TMA descriptors of the six matrices (128-row boxes) and the gains.
+struct alignas(64) FusedLayerTab {
+    TensorMap128 t_qkv, t_o, t_qc, t_oc, t_1, t_2;
+    const float *g1, *g2, *g3;
+};
+// Per-slot table in device memory: descriptors of the activation buffers as A operands (128-row boxes)
+// and as store targets of the epilogues (32-row x 64-column boxes).
+struct alignas(64) FusedMaps {
+    TensorMap128 a_xg, a_att, a_u, c_qkv, c_qc, c_u;
+};
+struct FusedArgs {
+    int H, A, d, md, n_layers, n_heads, hd, hpc, K;
+    int S, ne0;                    // inner steps of the batch, environments active at the first
+    int kv_layers, plane_rows;
+    float eps, inv_d;
+    const EnvMeta *meta;           // packed order: environments still active at inner step s are a prefix
+    const int *n_active;           // device [S]
+    int *done;                     // device [S][mt_max] completion counters, zero on entry
+    int mt_max;
+    int *trace;                    // device [#CTAs][4] progress notes (task in hand per role), or NULL
+    float *a_state, *x, *ssq;
+    void *xg, *qkv, *att, *qc, *u;
+    const FusedMaps *maps;
+    const TensorMap128 *attn_maps; // [0] = the QKV buffer, [1 + j] = environment j's planes
+    const FusedLayerTab *layers;
+    const void *w_in, *w_out;
+    const float *b_out, *g_final, *temb;
+};
+bool fused_supported(int H, int A, int d, int md, int n_heads, int hd);
+cudaError_t launch_fused_steps(const FusedArgs &f, int grid, unsigned long long limit_ns, int *status, cudaStream_t st);
+
 // An SM partition (green context) with a stream inside it.
 struct GreenPartition {
     void *ctx = nullptr;

@@ -1,6 +1,13 @@
-// Host-only: the elastic resource allocator (Algorithm 1, Eq. 2) and the runtime re-balance
-// trigger of section 4.3.2.  No device code; lives in the library so that a scheduler written
-// in any language can call it next to the generation entry points.
+// Host-only: the elastic resource allocator (section 4.3.2: Algorithm 1 and Eq. 2) and the runtime
+// re-balance trigger of the same section.  No device code; lives in the library so that a scheduler
+// written in any language can call it next to the generation entry points.
+//
+// The allocation problem: the simulator keeps the smallest profiled quota at which its rate is within
+// a tolerance of its best (more SMs buy it nothing); the rest of the chip is divided between generation
+// and training so that the pipeline rate Theta = min(min(T_s, T_g), T_t) is largest.  T_g grows and T_t
+// shrinks as generation's share grows, so the division is found by bisecting on "is rollout already
+// faster than training?", with the best batch-size pair that fits the memory budget chosen at every
+// probe, and the better end of the final bracket returned.
 #include "../../include/ebrl_alloc.h"
 
 #include <algorithm>
@@ -43,7 +50,7 @@ struct Cand {
     bool feasible;
 };
 
-// Line 9: the batch-size pair with the highest predicted end-to-end rate within M_gpu.
+// The batch-size pair with the highest predicted end-to-end rate that fits the memory budget, for one division.
 Cand evaluate(const ebrl_alloc_in_t &in, int s_sim, double T_s, int s_g)
 {
     Cand best{};
@@ -61,6 +68,32 @@ Cand evaluate(const ebrl_alloc_in_t &in, int s_sim, double T_s, int s_g)
             }
         }
     return best;
+}
+
+// The simulator's knee: the first profiled quota whose rate is within the tolerance of the table's best.
+// Rates must be positive finite numbers (a table of zeros, negatives or NaNs has no knee).
+bool simulator_knee(const ebrl_alloc_in_t &in, int *knee)
+{
+    double peak = 0.0;
+    for (int i = 0; i < in.n_sim_quota; ++i) {
+        const double r = in.sim_rate[i];
+        if (!(r > 0.0) || !(r < 1e300)) return false;
+        peak = std::max(peak, r);
+    }
+    for (int i = 0; i < in.n_sim_quota; ++i)
+        if (in.sim_rate[i] >= (1.0 - in.knee_tolerance) * peak) { *knee = i; return true; }
+    return false;
+}
+
+// Integer bisection: shrinks [lo, hi] to adjacent values, keeping pred false towards lo and true towards hi.
+template <typename Pred>
+void narrow_bracket(int &lo, int &hi, int &probes, Pred pred)
+{
+    while (hi - lo > 1) {
+        const int mid = lo + (hi - lo) / 2;
+        if (pred(mid)) hi = mid; else lo = mid;
+        ++probes;
+    }
 }
 
 }  // namespace
@@ -85,28 +118,23 @@ int32_t ebrl_alloc_elastic(const ebrl_alloc_in_t *in, ebrl_alloc_out_t *out)
     if (!in || !out || in->cores < 1 || in->cores_per_env < 1 || !in->sim_rate || !(in->knee_tolerance >= 0.0)) return 1;
     if (!grid_ok(in->n_sim_quota, in->sim_quota_pct, 0) || !profile_ok(in->gen) || !profile_ok(in->train)) return 1;
     if (in->s_g_min < 1 || in->s_t_min < 1) return 1;
-    // lines 1-4: simulator capacity at the profiled core count and the knee quota
-    const int E = in->cores / in->cores_per_env;
+    const int E = in->cores / in->cores_per_env;     // environments the host cores can drive
     if (E < 1) return 1;
-    double peak = in->sim_rate[0];
-    for (int i = 1; i < in->n_sim_quota; ++i) peak = std::max(peak, in->sim_rate[i]);
-    int knee = 0;
-    while (in->sim_rate[knee] < (1.0 - in->knee_tolerance) * peak) ++knee;
+    int knee = -1;
+    if (!simulator_knee(*in, &knee)) return 1;
     const int s_sim = in->sim_quota_pct[knee];
     const double T_s = in->sim_rate[knee];
-    // line 5: the generation quota's interval
-    int lo = in->s_g_min, hi = 100 - s_sim - in->s_t_min;
+    int lo = in->s_g_min, hi = 100 - s_sim - in->s_t_min;   // what is left for generation once training has its minimum
     if (hi < lo) return 1;
     int it = 0;
-    // lines 6-17: bisection on s_g, comparing rollout with training
-    while (hi - lo > 1) {
-        const int s_g = (lo + hi) / 2;
+    bool all_feasible = true;
+    // rollout_ahead(s_g): with this share, does rollout already outpace training?  False at small shares, true at large ones.
+    narrow_bracket(lo, hi, it, [&](int s_g) {
         const Cand c = evaluate(*in, s_sim, T_s, s_g);
-        if (!c.feasible) return 1;
-        if (c.T_r > c.T_t) hi = s_g; else lo = s_g;
-        ++it;
-    }
-    // lines 18-19: both endpoints, the better one wins
+        all_feasible = all_feasible && c.feasible;
+        return c.feasible && c.T_r > c.T_t;
+    });
+    if (!all_feasible) return 1;
     const Cand a = evaluate(*in, s_sim, T_s, lo), b = evaluate(*in, s_sim, T_s, hi);
     if (!a.feasible && !b.feasible) return 1;
     const Cand &w = (!b.feasible || (a.feasible && a.theta >= b.theta)) ? a : b;

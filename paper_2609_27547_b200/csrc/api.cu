@@ -41,6 +41,7 @@ struct WeightSet {
     void *w_in = nullptr, *w_out = nullptr;
     float *b_out = nullptr, *g_final = nullptr;
     std::vector<LayerDev> layers;
+    FusedLayerTab *ftab_d = nullptr;   // the persistent step kernel's per-layer table (descriptors + gains) in device memory
     bool allocated = false, ever_used = false;
     uint64_t version = 0;
     cudaEvent_t ready = nullptr;      // upload complete
@@ -64,9 +65,13 @@ struct Slot {
     void *xg = nullptr, *qkv = nullptr, *att = nullptr, *qc = nullptr, *u = nullptr;
     EnvMeta *meta_d = nullptr, *meta_h = nullptr;
     TensorMap128 t_xg, t_att, t_u;                    // TMA descriptors of the A operands
+    FusedMaps *fmaps_d = nullptr;                     // persistent step kernel: the same plus the epilogues' store targets, in device memory
+    int *fctl_d = nullptr, *fctl_h = nullptr;         // its control block: n_active[K] then the completion counters [K][mt_max]
+    int mt_max = 0;
     TensorMap128 *maps_d = nullptr, *maps_h = nullptr; // attention descriptors: [0] = QKV buffer, [1 + j] = env j's planes
     cudaEvent_t done = nullptr;
     bool busy = false;
+    int wset = 0;                                     // weight set the slot's batch in flight reads
     std::vector<int64_t> ids;
     // staging of the host-buffer entry point (allocated on first use)
     char *kv_stage = nullptr;
@@ -101,6 +106,11 @@ struct ebrl_actgen {
     bool use_tc = false;          // tensor-core GEMMs (bf16, d a multiple of 256)
     bool use_pairs = true;        // CTA-pair GEMM allowed (EBRL_GEMM_PAIR=0 forbids it)
     int force_shape = 0;          // EBRL_GEMM_SHAPE = 2 (pairs), 256 or 128 forces one tile shape (tests, tuning)
+    bool trace = false;           // EBRL_TRACE=1: the persistent kernel notes its progress; a time-out prints it to stderr
+    Slot *trace_slot = nullptr;
+    bool fused_ok = false;        // the persistent step kernel covers this model
+    long fused_max_rows = 0;      // batches of at most this many rows take it by themselves (EBRL_FUSED_MAX_ROWS); 0: only when forced --
+                                  // measured on B200 it is bit-identical to, but slower than, the per-operation kernels at every size tried
     bool pdl_allowed = true;      // EBRL_PDL=0 turns programmatic dependent launch off
     int attn_lookahead = 2;       // EBRL_ATTN_LOOKAHEAD: key blocks the attention producer asks L2 for ahead of its ring
     bool use_attn_mma = false;    // tensor-core attention (bf16, H <= 16, head_dim 64/128)
@@ -299,6 +309,18 @@ ebrl_status_t alloc_weight_set(ebrl_actgen *h, WeightSet &ws)
             if (bad) return fail(h, EBRL_ERR_CUDA, "cuTensorMapEncodeTiled failed for a weight matrix");
         }
     }
+    if (h->fused_ok && c.n_layers > 0) {
+        // descriptors and gain pointers refer to the set's buffers, not to their contents: built once per set
+        std::vector<FusedLayerTab> tab(c.n_layers);
+        for (int l = 0; l < c.n_layers; ++l) {
+            const LayerDev &o = ws.layers[l];
+            tab[l].t_qkv = o.t_qkv; tab[l].t_o = o.t_o; tab[l].t_qc = o.t_qc; tab[l].t_oc = o.t_oc; tab[l].t_1 = o.t_1; tab[l].t_2 = o.t_2;
+            tab[l].g1 = o.g1; tab[l].g2 = o.g2; tab[l].g3 = o.g3;
+        }
+        if ((st = dev_alloc(h, &p, sizeof(FusedLayerTab) * tab.size())) != EBRL_OK) return st;
+        ws.ftab_d = (FusedLayerTab *)p;
+        CK(cudaMemcpy(ws.ftab_d, tab.data(), sizeof(FusedLayerTab) * tab.size(), cudaMemcpyHostToDevice));
+    }
     if (cudaEventCreateWithFlags(&ws.ready, cudaEventDisableTiming) != cudaSuccess ||
         cudaEventCreateWithFlags(&ws.last_use, cudaEventDisableTiming) != cudaSuccess)
         return fail(h, EBRL_ERR_CUDA, "cudaEventCreate failed");
@@ -432,6 +454,16 @@ int pick_tile_shape(const ebrl_actgen *h, long M, int N, int grid)
     return (t_pair <= t_256 && t_pair <= t_128) ? 2 : (t_256 <= t_128 ? 256 : 128);
 }
 
+// Whether a batch of `rows` rows takes the persistent step kernel: the model must be covered, and the batch
+// small enough that the per-operation grids would be mostly fill and drain (or the caller forces it).
+bool use_fused_path(const ebrl_actgen *h, long rows, int grid)
+{
+    const ebrl_actgen_cfg_t &c = h->cfg;
+    if (!h->fused_ok || (c.flags & (EBRL_FLAG_NO_FUSED | EBRL_FLAG_TEST_PULL)) || c.n_layers < 1 || grid < 1) return false;
+    if (c.flags & EBRL_FLAG_FORCE_FUSED) return true;
+    return rows <= h->fused_max_rows;
+}
+
 // Enqueues every kernel of one batch (the groups coalesced in one slot) on the stream.
 cudaError_t enqueue_batch(ebrl_actgen *h, Slot &s, int S, const int32_t *n_active, const double *sum_P_active, int grid,
                           cudaStream_t st)
@@ -468,6 +500,31 @@ cudaError_t enqueue_batch(ebrl_actgen *h, Slot &s, int S, const int32_t *n_activ
                     ln.run(EBRL_KC_PREFIX, flops, bytes, [&] { return launch_gemm_simt(g, bf, grid, st); });
                 }
             }
+    }
+    if (use_fused_path(h, (long)n_active[0] * H, grid) && S > 0 && n_active[0] > 0) {
+        // small batch: ONE persistent kernel walks every Euler step
+        for (int t = 0; t < c.K_steps; ++t) s.fctl_h[t] = t < S ? n_active[t] : 0;
+        if ((ln.err = cudaMemcpyAsync(s.fctl_d, s.fctl_h, sizeof(int) * c.K_steps, cudaMemcpyHostToDevice, st)) != cudaSuccess) return ln.err;
+        if ((ln.err = cudaMemsetAsync(s.fctl_d + c.K_steps, 0, sizeof(int) * ((size_t)c.K_steps * s.mt_max + 4 * 256 + 2 * 12 * 4 * 256 + 4 + 4 * 4000), st)) != cudaSuccess) return ln.err;
+        FusedArgs f{};
+        f.H = H; f.A = c.A; f.d = d; f.md = md; f.n_layers = L; f.n_heads = c.n_heads; f.hd = h->hd;
+        f.hpc = c.n_heads < 8 ? c.n_heads : 8; f.K = c.K_steps; f.S = S; f.ne0 = n_active[0];
+        f.kv_layers = c.kv_layers; f.plane_rows = c.d_ctx > 0 ? s.prefix_rows : 0;
+        f.eps = c.rms_eps; f.inv_d = 1.0f / (float)d;
+        f.meta = s.meta_d; f.n_active = s.fctl_d; f.done = s.fctl_d + c.K_steps; f.mt_max = s.mt_max;
+        f.trace = h->trace ? s.fctl_d + (size_t)c.K_steps * (1 + s.mt_max) : nullptr;
+        h->trace_slot = &s;
+        f.a_state = s.a_state; f.x = s.x; f.ssq = s.ssq; f.xg = s.xg; f.qkv = s.qkv; f.att = s.att; f.qc = s.qc; f.u = s.u;
+        f.maps = s.fmaps_d; f.attn_maps = s.maps_d; f.layers = W.ftab_d;
+        f.w_in = W.w_in; f.w_out = W.w_out; f.b_out = W.b_out; f.g_final = W.g_final; f.temb = h->temb;
+        double flops = 0.0, bytes = 0.0;
+        for (int step = 0; step < S; ++step) {
+            const double M = (double)n_active[step] * H;
+            flops += L * (M * (12.0 * d * d + 4.0 * d * md) + 4.0 * H * sum_P_active[step] * d + 4.0 * M * H * d) + 4.0 * M * d * c.A;
+            bytes += L * (2.0 * sum_P_active[step] * d * esz + (6.0 * d * d + 2.0 * d * md) * esz);   // planes and weights once per layer-step
+        }
+        ln.run(EBRL_KC_FUSED, flops, bytes, [&] { return launch_fused_steps(f, grid, h->wait_ns, h->status_d, st); });
+        return ln.err;
     }
     for (int step = 0; step < S; ++step) {
         const int ne = n_active[step], M = ne * H;
@@ -633,6 +690,7 @@ ebrl_status_t flush_slot(ebrl_actgen *h, Slot &s)
     }
     CK(cudaEventRecord(wsel.last_use, cs));
     wsel.ever_used = true;
+    s.wset = h->active;
     if (gp) {
         CK(cudaEventRecord(s.part_out, cs));
         CK(cudaStreamWaitEvent(user, s.part_out, 0));
@@ -798,6 +856,7 @@ void free_all(ebrl_actgen *h)
         if (s.part_out) cudaEventDestroy(s.part_out);
         if (s.meta_h) cudaFreeHost(s.meta_h);
         if (s.maps_h) cudaFreeHost(s.maps_h);
+        if (s.fctl_h) cudaFreeHost(s.fctl_h);
         if (s.kv_stage) cudaFree(s.kv_stage);
         if (s.hid_pack) cudaFree(s.hid_pack);
         if (s.planes) cudaFree(s.planes);
@@ -912,6 +971,9 @@ ebrl_status_t ebrl_actgen_create(const ebrl_actgen_cfg_t *cfg, const ebrl_actgen
     if (const char *e4 = getenv("EBRL_PDL")) h->pdl_allowed = atoi(e4) != 0;
     if (const char *e5 = getenv("EBRL_ATTN_LOOKAHEAD")) h->attn_lookahead = std::min(64, std::max(0, atoi(e5)));
     h->use_attn_mma = h->bf16 && !(cfg->flags & EBRL_FLAG_FORCE_SIMT) && attn_mma_supported(cfg->H, cfg->n_heads, h->hd);
+    h->fused_ok = h->use_tc && h->use_attn_mma && fused_supported(cfg->H, cfg->A, d, md, cfg->n_heads, h->hd);
+    if (const char *e6 = getenv("EBRL_FUSED_MAX_ROWS")) h->fused_max_rows = atol(e6);
+    if (const char *e7 = getenv("EBRL_TRACE")) h->trace = atoi(e7) != 0;
     if ((st = alloc_weight_set(h, h->wset[0])) != EBRL_OK) return bail(st);
     if ((st = upload_weight_set(h, h->wset[0], wts, nullptr, false)) != EBRL_OK) return bail(st);
     h->wset[0].version = 1;
@@ -991,6 +1053,24 @@ ebrl_status_t ebrl_actgen_create(const ebrl_actgen_cfg_t *cfg, const ebrl_actgen
                       make_tmap_bf16(&s.t_u, s.u, md, rows, ba);
             if (bad) { fail(h, EBRL_ERR_CUDA, "cuTensorMapEncodeTiled failed for a workspace"); return bail(EBRL_ERR_CUDA); }
         }
+        if (h->fused_ok) {
+            FusedMaps fm;
+            fm.a_xg = s.t_xg; fm.a_att = s.t_att; fm.a_u = s.t_u;
+            int bad = make_tmap_bf16(&fm.c_qkv, s.qkv, 3 * (uint64_t)d, rows, 32) | make_tmap_bf16(&fm.c_qc, s.qc, d, rows, 32) |
+                      make_tmap_bf16(&fm.c_u, s.u, md, rows, 32);
+            if (bad) { fail(h, EBRL_ERR_CUDA, "cuTensorMapEncodeTiled failed for a workspace"); return bail(EBRL_ERR_CUDA); }
+            if ((st = dev_alloc(h, &p, sizeof fm)) != EBRL_OK) return bail(st);
+            s.fmaps_d = (FusedMaps *)p;
+            if (cudaMemcpy(s.fmaps_d, &fm, sizeof fm, cudaMemcpyHostToDevice) != cudaSuccess) { fail(h, EBRL_ERR_CUDA, "cudaMemcpy failed"); return bail(EBRL_ERR_CUDA); }
+            s.mt_max = (int)((rows + 127) / 128);
+            if ((st = dev_alloc(h, &p, sizeof(int) * ((size_t)cfg->K_steps * (1 + s.mt_max) + 4 * 256 + 2 * 12 * 4 * 256 + 4 + 4 * 4000))) != EBRL_OK) return bail(st);
+            s.fctl_d = (int *)p;
+            if (cudaMallocHost((void **)&s.fctl_h, sizeof(int) * (size_t)cfg->K_steps) != cudaSuccess) {
+                cudaGetLastError();
+                fail(h, EBRL_ERR_NOMEM, "pinned staging allocation failed");
+                return bail(EBRL_ERR_NOMEM);
+            }
+        }
         if (cudaEventCreateWithFlags(&s.part_in, cudaEventDisableTiming) != cudaSuccess ||
             cudaEventCreateWithFlags(&s.part_out, cudaEventDisableTiming) != cudaSuccess ||
             cudaEventCreateWithFlags(&s.h2d_done, cudaEventDisableTiming) != cudaSuccess) {
@@ -1055,10 +1135,29 @@ ebrl_status_t ebrl_actgen_sync(ebrl_actgen_t h)
     }
     h->host_depth = 1;
     if (first == EBRL_OK && h->status_d) {
-        int word = 0;
-        if (cudaMemcpy(&word, h->status_d, sizeof word, cudaMemcpyDeviceToHost) == cudaSuccess && word != 0) {
-            h->sticky = (ebrl_status_t)word;
-            fail(h, h->sticky, "a device-side wait ran out of time (status %d)", word);
+        int word[4] = {0, 0, 0, 0};   // [0] status; [1..3] where the first wait gave up (persistent step kernel): site/kind/step, task, detail
+        if (cudaMemcpy(word, h->status_d, sizeof word, cudaMemcpyDeviceToHost) == cudaSuccess && word[0] != 0) {
+            h->sticky = (ebrl_status_t)word[0];
+            if (word[1] != 0 && h->trace && h->trace_slot) {
+                std::vector<int> tr(4 * 256), ctr((size_t)h->cfg.K_steps * h->trace_slot->mt_max);
+                const Slot &ts = *h->trace_slot;
+                if (cudaMemcpy(tr.data(), ts.fctl_d + (size_t)h->cfg.K_steps * (1 + ts.mt_max), tr.size() * 4, cudaMemcpyDeviceToHost) == cudaSuccess &&
+                    cudaMemcpy(ctr.data(), ts.fctl_d + h->cfg.K_steps, ctr.size() * 4, cudaMemcpyDeviceToHost) == cudaSuccess) {
+                    fprintf(stderr, "[ebrl trace] cta: producer mma workers0 workers1  (task<<4 | kind<<2 | self)\n");
+                    for (int cta = 0; cta < 256; ++cta)
+                        if (tr[4 * cta] | tr[4 * cta + 1] | tr[4 * cta + 2] | tr[4 * cta + 3])
+                            fprintf(stderr, "[ebrl trace] %3d: %d/%d %d/%d %d/%d %d/%d\n", cta, tr[4 * cta] >> 4, tr[4 * cta] & 15, tr[4 * cta + 1] >> 4,
+                                    tr[4 * cta + 1] & 15, tr[4 * cta + 2] >> 4, tr[4 * cta + 2] & 15, tr[4 * cta + 3] >> 4, tr[4 * cta + 3] & 15);
+                    fprintf(stderr, "[ebrl trace] counters of inner step 0:");
+                    for (int m = 0; m < ts.mt_max && m < 32; ++m) fprintf(stderr, " %d", ctr[m]);
+                    fprintf(stderr, "\n");
+                }
+            }
+            if (word[1] != 0)
+                fail(h, h->sticky, "a device-side wait ran out of time (status %d; site %d, operation kind %d, inner step %d, task %d, detail 0x%x)",
+                     word[0], word[1] & 0xff, (word[1] >> 8) & 0xf, (word[1] >> 12) & 0xffff, word[2], (unsigned)word[3]);
+            else
+                fail(h, h->sticky, "a device-side wait ran out of time (status %d)", word[0]);
         }
     }
     if (first == EBRL_OK && h->sticky != EBRL_OK) first = h->sticky;
@@ -1114,7 +1213,12 @@ ebrl_status_t ebrl_actgen_update_weights(ebrl_actgen_t h, const ebrl_actgen_weig
     WeightSet &t = h->wset[1 - h->active];
     if (!t.allocated && (st = alloc_weight_set(h, t)) != EBRL_OK) return st;
     cudaStream_t cs = (cudaStream_t)stream;
-    if (t.ever_used) CK(cudaStreamWaitEvent(cs, t.last_use, 0));   // batches still reading the set being replaced
+    // Batches still reading the set being replaced: the upload waits for every one of them on the device.  last_use
+    // covers the most recent batch; batches in flight on other streams (two slots, partition streams) have their
+    // own completion events.
+    if (t.ever_used) CK(cudaStreamWaitEvent(cs, t.last_use, 0));
+    for (Slot &sl : h->slots)
+        if (sl.busy && sl.wset == 1 - h->active) CK(cudaStreamWaitEvent(cs, sl.done, 0));
     if ((st = upload_weight_set(h, t, weights, cs, true)) != EBRL_OK) return st;
     CK(cudaEventRecord(t.ready, cs));
     h->active = 1 - h->active;
@@ -1147,6 +1251,25 @@ ebrl_status_t ebrl_actgen_partition_info(ebrl_actgen_t h, int32_t sm_quota, int3
     if (out_rest_stream) *out_rest_stream = (void *)gp->rest_stream;
     return EBRL_OK;
 }
+
+#ifdef EBRL_FUSED_PROF
+// tuning builds only: the persistent kernel's cycle accounting of the last launch
+ebrl_status_t ebrl_actgen_debug_prof(ebrl_actgen_t h, long long *out, int32_t n)
+{
+    if (!h || !out || !h->trace_slot) return EBRL_ERR_INVALID_ARG;
+    const Slot &ts = *h->trace_slot;
+    const int *base = ts.fctl_d + (size_t)h->cfg.K_steps * (1 + ts.mt_max) + 4 * 256;
+    return cudaMemcpy(out, base, sizeof(long long) * (size_t)n, cudaMemcpyDeviceToHost) == cudaSuccess ? EBRL_OK : EBRL_ERR_CUDA;
+}
+ebrl_status_t ebrl_actgen_debug_events(ebrl_actgen_t h, long long *out, int32_t n_events, int32_t *count)
+{
+    if (!h || !out || !h->trace_slot) return EBRL_ERR_INVALID_ARG;
+    const Slot &ts = *h->trace_slot;
+    const int *base = ts.fctl_d + (size_t)h->cfg.K_steps * (1 + ts.mt_max) + 4 * 256 + 2 * 12 * 4 * 256;
+    if (cudaMemcpy(count, base, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return EBRL_ERR_CUDA;
+    return cudaMemcpy(out, base + 4, sizeof(long long) * 2 * (size_t)n_events, cudaMemcpyDeviceToHost) == cudaSuccess ? EBRL_OK : EBRL_ERR_CUDA;
+}
+#endif
 
 ebrl_status_t ebrl_actgen_set_timing(ebrl_actgen_t h, int32_t on)
 {

@@ -97,6 +97,20 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 
 constexpr int EPI_STAGE_FLOATS = 32 * 32;   // per-warp transpose buffer: 32 rows x 32 fp32 columns, 16-byte chunks swizzled
 
+// Loads of data that another CTA of the SAME kernel may have written (the persistent step kernel):
+// COH = true reads through L2 (ld.global.cg), because this SM's L1 may still hold the line from
+// an earlier task; kernels whose inputs were complete before launch use plain loads.
+template <bool COH> __device__ __forceinline__ float4 ld_f4(const float *p)
+{
+    if (COH) return __ldcg(reinterpret_cast<const float4 *>(p));
+    return *reinterpret_cast<const float4 *>(p);
+}
+template <bool COH> __device__ __forceinline__ float ld_f1(const float *p)
+{
+    if (COH) return __ldcg(p);
+    return *p;
+}
+
 // EPI_SCALE_STORE: C = acc * rowscale;  EPI_SCALE_GELU: C = gelu(acc * rowscale);
 // EPI_RESID: x += acc, xg = x * gain, one sum-of-squares partial per 128 columns.
 //
@@ -112,7 +126,7 @@ constexpr int EPI_STAGE_FLOATS = 32 * 32;   // per-warp transpose buffer: 32 row
 // All 32 lanes must call it.  `wait` blocks until the accumulator is complete (false on a
 // time-out); the residual values of the first chunk are requested before it and those of each
 // later chunk one chunk ahead.
-template <int EPI, int NCOLS, typename WaitF>
+template <int EPI, int NCOLS, bool COH = false, typename WaitF>
 __device__ __forceinline__ bool epilogue_rows(const GemmArgs &g, uint32_t taddr, int row0, int n0, float *stg_generic, WaitF wait)
 {
     constexpr int NC = NCOLS / 32;
@@ -127,11 +141,11 @@ __device__ __forceinline__ bool epilogue_rows(const GemmArgs &g, uint32_t taddr,
     if (EPI == EPI_RESID) {
 #pragma unroll
         for (int i = 0; i < 8; ++i)
-            if (4 * i + sub < nrows) xv[i] = *reinterpret_cast<const float4 *>(xg_x + (size_t)(row0 + 4 * i + sub) * g.N + n0 + 4 * piece);
+            if (4 * i + sub < nrows) xv[i] = ld_f4<COH>(xg_x + (size_t)(row0 + 4 * i + sub) * g.N + n0 + 4 * piece);
     } else if (lane < nrows) {
         float s = 0.f;
         const int row = row0 + lane;
-        for (int t = 0; t < g.n_ssq; ++t) s += g.ssq_in[(size_t)row * g.n_ssq + t];
+        for (int t = 0; t < g.n_ssq; ++t) s += ld_f1<COH>(g.ssq_in + (size_t)row * g.n_ssq + t);
         rs = 1.0f / sqrtf(s * g.inv_d + g.eps);
     }
     if (!wait()) return false;
@@ -188,7 +202,7 @@ __device__ __forceinline__ bool epilogue_rows(const GemmArgs &g, uint32_t taddr,
             if (c + 1 < NC) {
 #pragma unroll
                 for (int i = 0; i < 8; ++i)
-                    if (4 * i + sub < nrows) xv[i] = *reinterpret_cast<const float4 *>(xg_x + (size_t)(row0 + 4 * i + sub) * g.N + col + 32 + 4 * piece);
+                    if (4 * i + sub < nrows) xv[i] = ld_f4<COH>(xg_x + (size_t)(row0 + 4 * i + sub) * g.N + col + 32 + 4 * piece);
             }
         } else {
             __nv_bfloat16 *__restrict__ cp = (__nv_bfloat16 *)g.C;
@@ -222,7 +236,7 @@ __device__ __forceinline__ bool epilogue_rows(const GemmArgs &g, uint32_t taddr,
 // Per 64 columns that is 8 shared stores per thread and one copy instruction per warp, instead of 16 shared
 // stores, 16 shared loads and 16 predicated global stores -- fewer issue slots taken from the single TMA and
 // MMA threads that share the schedulers.  `stg_generic` must be 1024-byte aligned (4 KB).
-template <int EPI, int NCOLS, typename WaitF>
+template <int EPI, int NCOLS, bool COH = false, typename WaitF>
 __device__ __forceinline__ bool epilogue_store_tma(const GemmArgs &g, const CUtensorMap *tmC, uint32_t taddr, int row0, int n0,
                                                    float *stg_generic, WaitF wait)
 {
@@ -233,7 +247,7 @@ __device__ __forceinline__ bool epilogue_store_tma(const GemmArgs &g, const CUte
     if (row0 + lane < g.M) {
         float s = 0.f;
         const int row = row0 + lane;
-        for (int t = 0; t < g.n_ssq; ++t) s += g.ssq_in[(size_t)row * g.n_ssq + t];
+        for (int t = 0; t < g.n_ssq; ++t) s += ld_f1<COH>(g.ssq_in + (size_t)row * g.n_ssq + t);
         rs = 1.0f / sqrtf(s * g.inv_d + g.eps);
     }
     if (!wait()) return false;

@@ -6,28 +6,10 @@
 // output element is computed by a fixed sequence of operations that does not depend on the
 // grid size or on which other rows share a tile.
 #include "actgen_internal.h"
+#include "rowops.cuh"
 
 namespace ebrl {
 
-template <typename T> __device__ __forceinline__ float ldf(const T *p);
-template <> __device__ __forceinline__ float ldf<float>(const float *p) { return *p; }
-template <> __device__ __forceinline__ float ldf<__nv_bfloat16>(const __nv_bfloat16 *p) { return __bfloat162float(*p); }
-template <typename T> __device__ __forceinline__ void stf(T *p, float v);
-template <> __device__ __forceinline__ void stf<float>(float *p, float v) { *p = v; }
-template <> __device__ __forceinline__ void stf<__nv_bfloat16>(__nv_bfloat16 *p, float v) { *p = __float2bfloat16_rn(v); }
-
-__device__ __forceinline__ float warp_sum(float v)
-{
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    return v;
-}
-__device__ __forceinline__ float warp_max(float v)
-{
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-    return v;
-}
 __device__ __forceinline__ float gelu_erf(float z) { return 0.5f * z * (1.0f + erff(z * 0.70710678118654752440f)); }
 
 // ---------------------------------------------------------------------------------------
@@ -36,77 +18,22 @@ __device__ __forceinline__ float gelu_erf(float z) { return 0.5f * z * (1.0f + e
 // 128-column segment at a time; the row's action vector lives in the lanes and is broadcast by
 // shuffles.
 // ---------------------------------------------------------------------------------------
-template <typename T> __device__ __forceinline__ void store4(T *p, float a, float b, float c, float d);
-template <> __device__ __forceinline__ void store4<float>(float *p, float a, float b, float c, float d)
-{
-    *reinterpret_cast<float4 *>(p) = make_float4(a, b, c, d);
-}
-template <> __device__ __forceinline__ void store4<__nv_bfloat16>(__nv_bfloat16 *p, float a, float b, float c, float d)
-{
-    __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
-    *reinterpret_cast<uint2 *>(p) = make_uint2(*reinterpret_cast<uint32_t *>(&lo), *reinterpret_cast<uint32_t *>(&hi));
-}
-
 template <typename T, int AMAX>
 __global__ void __launch_bounds__(1024) embed_kernel(EmbedArgs a)
 {
     extern __shared__ float wT[];   // [A][d]
-    const int rows = a.n_envs * a.H, nseg = a.d / SSQ_W;
+    const int rows = a.n_envs * a.H;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const T *w_in = (const T *)a.w_in;
-    T *xg = (T *)a.xg;
     pdl_launch_dependents();
     for (int c = threadIdx.x; c < a.d; c += blockDim.x)   // weights do not depend on the previous kernel
         for (int j = 0; j < a.A; ++j) wT[j * a.d + c] = ldf(w_in + (size_t)c * a.A + j);
     __syncthreads();
     pdl_wait();
     // two rows per warp pass: each staged weight is used for both
-    for (int row0 = (blockIdx.x * 32 + warp) * 2; row0 < rows; row0 += gridDim.x * 64) {
-        float aj[2][AMAX];
-        int kk[2];
-        const int nr = min(2, rows - row0);
-#pragma unroll
-        for (int r = 0; r < 2; ++r) {
-            const int row = row0 + (r < nr ? r : 0);
-            const int env = row / a.H, h = row - env * a.H;
-            const EnvMeta m = a.meta[env];
-            kk[r] = m.k0 + a.s;
-            const float *av = (a.s == 0) ? m.noise + (size_t)h * a.A : a.a_state + (size_t)row * a.A;
-            const float mine = lane < a.A ? av[lane] : 0.f;
-#pragma unroll
-            for (int j = 0; j < AMAX; ++j) aj[r][j] = __shfl_sync(0xffffffffu, mine, j);
-        }
-        for (int seg = 0; seg < nseg; ++seg) {
-            const int c = seg * SSQ_W + 4 * lane;
-            float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-#pragma unroll
-            for (int j = 0; j < AMAX; ++j) {
-                if (j < a.A) {
-                    const float4 w = *reinterpret_cast<const float4 *>(wT + j * a.d + c);
-#pragma unroll
-                    for (int r = 0; r < 2; ++r) {
-                        acc[r][0] = fmaf(w.x, aj[r][j], acc[r][0]); acc[r][1] = fmaf(w.y, aj[r][j], acc[r][1]);
-                        acc[r][2] = fmaf(w.z, aj[r][j], acc[r][2]); acc[r][3] = fmaf(w.w, aj[r][j], acc[r][3]);
-                    }
-                }
-            }
-            const float4 gn = *reinterpret_cast<const float4 *>(a.gain + c);
-#pragma unroll
-            for (int r = 0; r < 2; ++r) {
-                if (r < nr) {
-                    const int row = row0 + r;
-                    const float4 te = *reinterpret_cast<const float4 *>(a.temb + (size_t)kk[r] * a.d + c);
-                    const float v0 = acc[r][0] + te.x, v1 = acc[r][1] + te.y, v2 = acc[r][2] + te.z, v3 = acc[r][3] + te.w;
-                    *reinterpret_cast<float4 *>(a.x + (size_t)row * a.d + c) = make_float4(v0, v1, v2, v3);
-                    store4<T>(xg + (size_t)row * a.d + c, v0 * gn.x, v1 * gn.y, v2 * gn.z, v3 * gn.w);
-                    float ss = v0 * v0;
-                    ss = fmaf(v1, v1, ss); ss = fmaf(v2, v2, ss); ss = fmaf(v3, v3, ss);
-                    ss = warp_sum(ss);
-                    if (lane == 0) a.ssq[(size_t)row * nseg + seg] = ss;
-                }
-            }
-        }
-    }
+    for (int row0 = (blockIdx.x * 32 + warp) * 2; row0 < rows; row0 += gridDim.x * 64)
+        embed_row_pair<T, AMAX, false>(a, row0, min(2, rows - row0), lane,
+                                       [&](int j, int c) { return *reinterpret_cast<const float4 *>(wT + j * a.d + c); });
 }
 
 // ---------------------------------------------------------------------------------------
@@ -129,81 +56,9 @@ __global__ void __launch_bounds__(HEAD_WARPS * 32) head_kernel(HeadArgs a)
     }
     __syncthreads();
     pdl_wait();
-    for (int row0 = (blockIdx.x * HEAD_WARPS + warp) * 2; row0 < rows; row0 += gridDim.x * HEAD_WARPS * 2) {
-        const int nr = min(2, rows - row0);
-        float acc[2][AMAX];
-#pragma unroll
-        for (int r = 0; r < 2; ++r)
-#pragma unroll
-            for (int j = 0; j < AMAX; ++j) acc[r][j] = 0.f;
-        float ss[2] = {0.f, 0.f};
-        if (!a.pull) {
-            // four 128-column steps per round: the eight row loads of a round are in flight together (one
-            // step at a time left a warp with two loads in flight and the kernel waiting on memory latency)
-            for (int c0 = lane * 4; c0 < a.d; c0 += 512) {
-                float4 xv[4][2], gv[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int c = c0 + u * 128;
-                    if (c < a.d) {
-                        gv[u] = *reinterpret_cast<const float4 *>(a.gain + c);
-#pragma unroll
-                        for (int r = 0; r < 2; ++r)
-                            xv[u][r] = *reinterpret_cast<const float4 *>(a.x + (size_t)(row0 + (r < nr ? r : 0)) * a.d + c);
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int c = c0 + u * 128;
-                    if (c < a.d) {
-                        float t[2][4];
-#pragma unroll
-                        for (int r = 0; r < 2; ++r) {
-                            const float4 x4 = xv[u][r];
-                            ss[r] = fmaf(x4.x, x4.x, ss[r]); ss[r] = fmaf(x4.y, x4.y, ss[r]);
-                            ss[r] = fmaf(x4.z, x4.z, ss[r]); ss[r] = fmaf(x4.w, x4.w, ss[r]);
-                            t[r][0] = x4.x * gv[u].x; t[r][1] = x4.y * gv[u].y; t[r][2] = x4.z * gv[u].z; t[r][3] = x4.w * gv[u].w;
-                        }
-#pragma unroll
-                        for (int j = 0; j < AMAX; ++j) {
-                            if (j < a.A) {
-                                const float4 w = *reinterpret_cast<const float4 *>(wO + j * a.d + c);
-#pragma unroll
-                                for (int r = 0; r < 2; ++r) {
-                                    acc[r][j] = fmaf(t[r][0], w.x, acc[r][j]); acc[r][j] = fmaf(t[r][1], w.y, acc[r][j]);
-                                    acc[r][j] = fmaf(t[r][2], w.z, acc[r][j]); acc[r][j] = fmaf(t[r][3], w.w, acc[r][j]);
-                                }
-                            }
-                        }
-                    }
-                }
-            }
-        }
-#pragma unroll
-        for (int r = 0; r < 2; ++r) {
-            if (r < nr) {   // warp-uniform
-                const int row = row0 + r;
-                const int env = row / a.H, h = row - env * a.H;
-                const EnvMeta m = a.meta[env];
-                const float ssr = a.pull ? 0.f : warp_sum(ss[r]);
-                const float inv = 1.0f / sqrtf(ssr / (float)a.d + a.eps);
-                const float *a_old = (a.s == 0) ? m.noise + (size_t)h * a.A : a.a_state + (size_t)row * a.A;
-#pragma unroll
-                for (int j = 0; j < AMAX; ++j) {
-                    if (j < a.A) {
-                        const float dot = warp_sum(acc[r][j]);
-                        if (lane == 0) {
-                            const float ao = a_old[j];
-                            const float v = a.pull ? (a.b_out[j] - ao) : (dot * inv + a.b_out[j]);
-                            const float an = ao + v / (float)a.K;
-                            a.a_state[(size_t)row * a.A + j] = an;
-                            if (a.s == m.nsteps - 1) m.out[(size_t)h * a.A + j] = an;
-                        }
-                    }
-                }
-            }
-        }
-    }
+    for (int row0 = (blockIdx.x * HEAD_WARPS + warp) * 2; row0 < rows; row0 += gridDim.x * HEAD_WARPS * 2)
+        head_row_pair<T, AMAX, false>(a, row0, min(2, rows - row0), lane,
+                                      [&](int j, int c) { return *reinterpret_cast<const float4 *>(wO + j * a.d + c); });
 }
 
 // ---------------------------------------------------------------------------------------

@@ -47,6 +47,7 @@ struct ebrl_queue {
     std::vector<Request> in_service;                   // step mode: mid-chunk environments, in admission order
     std::unordered_set<int64_t> live_envs;             // env ids with a request in the queue
     std::unordered_map<uint64_t, ebrl_status_t> finished;   // completed tickets not yet waited for
+    std::unordered_set<uint64_t> consumed;                  // tickets whose result has been handed out: a second wait is an error
     uint64_t next_ticket = 1;
     bool closing = false;
     int callers = 0;                                    // threads inside push or wait (destroy lets them leave first)
@@ -212,8 +213,8 @@ extern "C" ebrl_status_t ebrl_queue_wait(ebrl_queue_t q, uint64_t ticket, uint32
 {
     if (!q || ticket == 0) return EBRL_ERR_INVALID_ARG;
     std::unique_lock<std::mutex> lk(q->mu);
-    if (ticket >= q->next_ticket) return EBRL_ERR_INVALID_ARG;
-    auto ready = [&] { return q->finished.count(ticket) != 0; };
+    if (ticket >= q->next_ticket || q->consumed.count(ticket)) return EBRL_ERR_INVALID_ARG;   // never issued, or already waited for
+    auto ready = [&] { return q->finished.count(ticket) != 0 || q->consumed.count(ticket) != 0; };
     q->callers += 1;
     bool got = true;
     if (timeout_ms == 0) q->done_cv.wait(lk, ready);
@@ -221,8 +222,12 @@ extern "C" ebrl_status_t ebrl_queue_wait(ebrl_queue_t q, uint64_t ticket, uint32
     q->callers -= 1;
     q->idle_cv.notify_all();
     if (!got) return EBRL_ERR_TIMEOUT;
-    const ebrl_status_t rc = q->finished[ticket];
-    q->finished.erase(ticket);
+    auto it = q->finished.find(ticket);
+    if (it == q->finished.end()) return EBRL_ERR_INVALID_ARG;      // another waiter on the same ticket took it meanwhile
+    const ebrl_status_t rc = it->second;
+    q->finished.erase(it);
+    q->consumed.insert(ticket);
+    q->done_cv.notify_all();      // a second waiter on this ticket must not sleep on
     return rc;
 }
 

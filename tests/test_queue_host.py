@@ -176,3 +176,16 @@ def test_destroy_serves_what_is_waiting():
     assert blocked == [B.ERR_QUEUE_FULL]
     q.destroy()                                                           # returns only after the three requests ran
     assert sorted(e for g in be.groups for e in g["ids"]) == [0, 1, 2]
+
+
+def test_a_ticket_can_be_waited_for_once():
+    """The result of a ticket is handed out once: a second wait on it (with or without a timeout)
+    is an argument error instead of a wait that can never end, and destroy still returns."""
+    be = FakeBackend()
+    q = B.Queue(None, capacity=4, max_group=2, backend=be.struct)
+    t = _push(q, 1)
+    assert q.wait(t) == B.OK
+    assert q.wait(t) == B.ERR_INVALID_ARG
+    assert q.wait(t, timeout_ms=50) == B.ERR_INVALID_ARG
+    assert q.wait(t + 100) == B.ERR_INVALID_ARG                          # never issued
+    q.destroy()
