@@ -82,6 +82,15 @@ typedef enum { EBRL_F32 = 0, EBRL_BF16 = 1 } ebrl_dtype_t;
                                      EBRL_FUSED_MAX_ROWS=<rows> in the environment at create makes
                                      batches of up to that many rows take it                    */
 
+#define EBRL_FLAG_TEST_DROP_GEMM_COPIES 64u   /* tests of the give-up path only: the copy-issuing threads of
+                                     the projection kernels issue nothing, so every consumer's bounded
+                                     wait (cfg.wait_limit_ns) runs out and ebrl_actgen_sync returns
+                                     EBRL_ERR_TIMEOUT; the kernels return normally, the context stays usable */
+#define EBRL_FLAG_TEST_DROP_ATTN_COPIES 128u  /* the same for the tensor-core attention kernels                */
+#define EBRL_FLAG_DEBUG_CANARY 256u /* every device buffer the handle allocates at create gets a guard of
+                                     256 pattern bytes behind it; ebrl_actgen_sync checks the guards and
+                                     returns EBRL_ERR_CUDA naming the buffer when one was overwritten      */
+
 /* Plain data, copied at create. */
 typedef struct {
     uint32_t abi_version;        /* EBRL_ACTGEN_ABI_VERSION                                     */

@@ -33,7 +33,7 @@ typedef struct {
 
 typedef struct {
     int32_t cores;              /* N: CPU cores for simulation                                  */
-    int32_t cores_per_env;      /* c_env*: profiled per-environment core count (Alg. 1 line 1)  */
+    int32_t cores_per_env;      /* c_env*: profiled per-environment core count                  */
     /* simulator rate at (c_env*, E = floor(N / c_env*)) as a function of its SM quota; a
      * CPU-only simulator passes one grid point with quota 0                                    */
     int32_t n_sim_quota;

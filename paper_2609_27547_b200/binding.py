@@ -18,6 +18,7 @@ ABI_VERSION = 3
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_NOMEM, ERR_CUDA, ERR_ENV_BUSY, ERR_QUOTA, ERR_TIMEOUT = range(8)
 F32, BF16 = 0, 1
 FLAG_TEST_PULL, FLAG_GREEN_CTX, FLAG_TIMING, FLAG_FORCE_SIMT, FLAG_NO_FUSED, FLAG_FORCE_FUSED = 1, 2, 4, 8, 16, 32
+FLAG_TEST_DROP_GEMM_COPIES, FLAG_TEST_DROP_ATTN_COPIES, FLAG_DEBUG_CANARY = 64, 128, 256
 KC_NAMES = ("embed", "gemm", "self_attn", "cross_attn", "head", "prefix", "fused")
 
 

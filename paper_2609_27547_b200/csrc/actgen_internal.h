@@ -50,6 +50,7 @@ struct GemmArgs {
     const float *gain;     // [N] gain of the next RMSNorm
     void *xg;              // [M][N] (T)
     float *ssq_out;        // [M][N/SSQ_W]
+    int test_drop_copies;  // tests of the give-up path: the copy-issuing thread issues nothing, every consumer's bounded wait runs out
 };
 
 struct AttnArgs {
@@ -73,6 +74,7 @@ struct AttnArgs {
     // tensor-core kernel: TMA descriptors (device memory)
     const TensorMap128 *kv_maps;   // [n_envs]: the environment's planes as [kv_layers*2*P][d]
     const TensorMap128 *self_map;  // the QKV buffer as [rows][3d]
+    int test_drop_copies;          // tests of the give-up path (see GemmArgs)
 };
 
 struct EmbedArgs {
@@ -137,6 +139,7 @@ struct FusedArgs {
     int *done;                     // device [S][mt_max] completion counters, zero on entry
     int mt_max;
     int *trace;                    // device [#CTAs][4] progress notes (task in hand per role), or NULL
+    int test_drop_copies;          // tests of the give-up path: 1 = projections' copies, 2 = attention's copies are not issued
     float *a_state, *x, *ssq;
     void *xg, *qkv, *att, *qc, *u;
     const FusedMaps *maps;

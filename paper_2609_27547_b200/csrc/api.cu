@@ -131,6 +131,7 @@ struct ebrl_actgen {
     ebrl_status_t sticky = EBRL_OK;
     ebrl_actgen_stats_t stats;
     std::vector<void *> owned;   // every device allocation, for destroy
+    std::vector<std::pair<const char *, const char *>> canaries;   // EBRL_FLAG_DEBUG_CANARY: guard address and buffer name
     std::map<int, GreenPartition> partitions;   // SM partitions by quota (EBRL_FLAG_GREEN_CTX); ctx == nullptr: creation failed
     cudaStream_t copy_stream = nullptr;   // host-buffer entry point: uploads run here, beside the previous batch's kernels
 };
@@ -249,15 +250,43 @@ int plan_group(const ebrl_actgen_cfg_t *c, int n, const ebrl_submit_ext_t *ext, 
             return fail(h, EBRL_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e_));    \
     } while (0)
 
-ebrl_status_t dev_alloc(ebrl_actgen *h, void **p, size_t bytes)
+constexpr size_t CANARY_BYTES = 256;
+constexpr int CANARY_BYTE = 0xA5;
+
+// With EBRL_FLAG_DEBUG_CANARY every buffer gets a tail of CANARY_BYTES filled with a pattern that no kernel may
+// touch; ebrl_actgen_sync checks the tails (a stand-in for a memory checker: a write past a buffer's end shows up
+// as a changed tail, named in the error text).
+ebrl_status_t dev_alloc(ebrl_actgen *h, void **p, size_t bytes, const char *what = "buffer")
 {
     *p = nullptr;
-    cudaError_t e = cudaMalloc(p, bytes ? bytes : 16);
+    const bool canary = (h->cfg.flags & EBRL_FLAG_DEBUG_CANARY) != 0;
+    const size_t body = (bytes ? bytes : 16);
+    const size_t padded = (body + 15) & ~(size_t)15;
+    cudaError_t e = cudaMalloc(p, canary ? padded + CANARY_BYTES : body);
     if (e != cudaSuccess) {
         cudaGetLastError();
         return fail(h, EBRL_ERR_NOMEM, "cudaMalloc of %zu bytes failed: %s", bytes, cudaGetErrorString(e));
     }
     h->owned.push_back(*p);
+    if (canary) {
+        if (cudaMemset((char *)*p + padded, CANARY_BYTE, CANARY_BYTES) != cudaSuccess) return fail(h, EBRL_ERR_CUDA, "cudaMemset of a canary failed");
+        h->canaries.push_back({(const char *)*p + padded, what});
+    }
+    return EBRL_OK;
+}
+
+// Compares every canary tail with the pattern; names the first buffer whose tail changed.
+ebrl_status_t check_canaries(ebrl_actgen *h)
+{
+    unsigned char buf[CANARY_BYTES];
+    for (const auto &c : h->canaries) {
+        if (cudaMemcpy(buf, c.first, CANARY_BYTES, cudaMemcpyDeviceToHost) != cudaSuccess) return fail(h, EBRL_ERR_CUDA, "reading a canary failed");
+        for (size_t i = 0; i < CANARY_BYTES; ++i)
+            if (buf[i] != CANARY_BYTE) {
+                h->sticky = EBRL_ERR_CUDA;
+                return fail(h, EBRL_ERR_CUDA, "memory past the end of %s was overwritten (byte %zu of its guard)", c.second, i);
+            }
+    }
     return EBRL_OK;
 }
 
@@ -512,6 +541,7 @@ cudaError_t enqueue_batch(ebrl_actgen *h, Slot &s, int S, const int32_t *n_activ
         f.kv_layers = c.kv_layers; f.plane_rows = c.d_ctx > 0 ? s.prefix_rows : 0;
         f.eps = c.rms_eps; f.inv_d = 1.0f / (float)d;
         f.meta = s.meta_d; f.n_active = s.fctl_d; f.done = s.fctl_d + c.K_steps; f.mt_max = s.mt_max;
+        f.test_drop_copies = (c.flags & EBRL_FLAG_TEST_DROP_GEMM_COPIES) ? 1 : ((c.flags & EBRL_FLAG_TEST_DROP_ATTN_COPIES) ? 2 : 0);
         f.trace = h->trace ? s.fctl_d + (size_t)c.K_steps * (1 + s.mt_max) : nullptr;
         h->trace_slot = &s;
         f.a_state = s.a_state; f.x = s.x; f.ssq = s.ssq; f.xg = s.xg; f.qkv = s.qkv; f.att = s.att; f.qc = s.qc; f.u = s.u;
@@ -541,6 +571,7 @@ cudaError_t enqueue_batch(ebrl_actgen *h, Slot &s, int S, const int32_t *n_activ
                     g.A = A; g.W = W; g.M = M; g.N = N; g.K = K; g.epi = epi;
                     g.ssq_in = s.ssq; g.n_ssq = nseg; g.inv_d = 1.0f / (float)d; g.eps = c.rms_eps;
                     g.C = C; g.x = s.x; g.gain = gain; g.xg = s.xg; g.ssq_out = s.ssq;
+                    g.test_drop_copies = (c.flags & EBRL_FLAG_TEST_DROP_GEMM_COPIES) ? 1 : 0;
                     const double bytes = ((double)M * K + (double)N * K + (double)M * N) * esz + (epi == EPI_RESID ? 8.0 * M * N : 0.0);
                     if (h->use_tc) {
                         const int shape = pick_tile_shape(h, M, N, grid);
@@ -559,6 +590,7 @@ cudaError_t enqueue_batch(ebrl_actgen *h, Slot &s, int S, const int32_t *n_activ
                     a.q = s.qkv; a.q_stride = 3 * d; a.out = s.att; a.o_stride = d;
                     a.H = H; a.n_heads = c.n_heads; a.hd = h->hd; a.n_envs = ne; a.d = d;
                     a.self = 1;
+                    a.test_drop_copies = (c.flags & EBRL_FLAG_TEST_DROP_ATTN_COPIES) ? 1 : 0;
                     a.k_self = (const char *)s.qkv + (size_t)d * h->esz;
                     a.v_self = (const char *)s.qkv + (size_t)2 * d * h->esz;
                     a.kv_stride = 3 * d;
@@ -573,6 +605,7 @@ cudaError_t enqueue_batch(ebrl_actgen *h, Slot &s, int S, const int32_t *n_activ
                     a.q = s.qc; a.q_stride = d; a.out = s.att; a.o_stride = d;
                     a.H = H; a.n_heads = c.n_heads; a.hd = h->hd; a.n_envs = ne; a.d = d;
                     a.meta = s.meta_d; a.kv_plane = (c.kv_layers == 1) ? 0 : l; a.self = 0;
+                    a.test_drop_copies = (c.flags & EBRL_FLAG_TEST_DROP_ATTN_COPIES) ? 1 : 0;
                     a.plane_rows = c.d_ctx > 0 ? s.prefix_rows : 0;
                     a.self_map = s.maps_d; a.kv_maps = s.maps_d + 1;
                     ln.run(EBRL_KC_CROSS_ATTN, 4.0 * H * sum_P_active[step] * d,
@@ -1008,14 +1041,14 @@ ebrl_status_t ebrl_actgen_create(const ebrl_actgen_cfg_t *cfg, const ebrl_actgen
     h->slots.resize(2);
     for (Slot &s : h->slots) {
         void *p = nullptr;
-        if ((st = dev_alloc(h, &p, rows * A * 4)) != EBRL_OK) return bail(st); s.a_state = (float *)p;
-        if ((st = dev_alloc(h, &p, rows * d * 4)) != EBRL_OK) return bail(st); s.x = (float *)p;
-        if ((st = dev_alloc(h, &p, rows * (d / SSQ_W) * 4)) != EBRL_OK) return bail(st); s.ssq = (float *)p;
-        if ((st = dev_alloc(h, &s.xg, rows * d * esz)) != EBRL_OK) return bail(st);
-        if ((st = dev_alloc(h, &s.qkv, rows * 3 * d * esz)) != EBRL_OK) return bail(st);
-        if ((st = dev_alloc(h, &s.att, rows * d * esz)) != EBRL_OK) return bail(st);
-        if ((st = dev_alloc(h, &s.qc, rows * d * esz)) != EBRL_OK) return bail(st);
-        if ((st = dev_alloc(h, &s.u, rows * md * esz)) != EBRL_OK) return bail(st);
+        if ((st = dev_alloc(h, &p, rows * A * 4, "the action-state workspace")) != EBRL_OK) return bail(st); s.a_state = (float *)p;
+        if ((st = dev_alloc(h, &p, rows * d * 4, "the residual-stream workspace x")) != EBRL_OK) return bail(st); s.x = (float *)p;
+        if ((st = dev_alloc(h, &p, rows * (d / SSQ_W) * 4, "the sum-of-squares workspace")) != EBRL_OK) return bail(st); s.ssq = (float *)p;
+        if ((st = dev_alloc(h, &s.xg, rows * d * esz, "the workspace xg")) != EBRL_OK) return bail(st);
+        if ((st = dev_alloc(h, &s.qkv, rows * 3 * d * esz, "the workspace qkv")) != EBRL_OK) return bail(st);
+        if ((st = dev_alloc(h, &s.att, rows * d * esz, "the workspace att")) != EBRL_OK) return bail(st);
+        if ((st = dev_alloc(h, &s.qc, rows * d * esz, "the workspace qc")) != EBRL_OK) return bail(st);
+        if ((st = dev_alloc(h, &s.u, rows * md * esz, "the workspace u")) != EBRL_OK) return bail(st);
         if ((st = dev_alloc(h, &p, sizeof(EnvMeta) * batch_envs)) != EBRL_OK) return bail(st); s.meta_d = (EnvMeta *)p;
         if (cudaMallocHost((void **)&s.meta_h, sizeof(EnvMeta) * batch_envs) != cudaSuccess) {
             cudaGetLastError();
@@ -1134,6 +1167,7 @@ ebrl_status_t ebrl_actgen_sync(ebrl_actgen_t h)
         if (st != EBRL_OK && first == EBRL_OK) first = st;
     }
     h->host_depth = 1;
+    if (first == EBRL_OK && !h->canaries.empty()) first = check_canaries(h);
     if (first == EBRL_OK && h->status_d) {
         int word[4] = {0, 0, 0, 0};   // [0] status; [1..3] where the first wait gave up (persistent step kernel): site/kind/step, task, detail
         if (cudaMemcpy(word, h->status_d, sizeof word, cudaMemcpyDeviceToHost) == cudaSuccess && word[0] != 0) {

@@ -152,7 +152,7 @@ __global__ void __launch_bounds__(THREADS, 1) attn_mma_kernel(AttnArgs a, int hp
             locate(la_item, la_tm, la_P, la_krow, la_vrow, la_kgrp, la_vgrp);
             for (int i = 0; i < la_blocks; ++i) la_step();
         }
-        for (int item = blockIdx.x; item < items && ok; item += gridDim.x) {
+        for (int item = blockIdx.x; item < items && ok && !a.test_drop_copies; item += gridDim.x) {
             const void *tm;
             int P, krow, vrow, kgrp, vgrp;
             locate(item, tm, P, krow, vrow, kgrp, vgrp);

@@ -574,6 +574,8 @@ fused_steps_kernel(const __grid_constant__ FusedArgs f, unsigned long long limit
                 return true;
             };
             ok = walk_ops(f, [&](const OpDesc &o) -> bool {
+                if ((f.test_drop_copies == 1 && o.kind == OP_GEMM) || (f.test_drop_copies == 2 && o.kind == OP_ATTN))
+                    return false;     // tests of the give-up path: the producer walks off, the other roles' waits run out
                 if (o.kind == OP_GEMM) {
                     const int nt = o.N / BN, nkb = o.K / BK, pf = nkb < NST ? nkb : NST;
                     for (int t = first_task(o); t < o.ntasks; t += G) {

@@ -113,7 +113,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
     if (warp == 0) {
         // ---- TMA producer: one thread (no votes, fewer instructions between a free stage and its next copies)
-        if (lane == 0) {
+        if (lane == 0 && !g.test_drop_copies) {
             int stage = 0;
             uint32_t phase = 0;
             for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {

@@ -133,7 +133,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         // ---- TMA producer (both CTAs), one thread: own A rows, own half of the weight tile; bytes land on the
         // leader's barrier.  (One thread instead of a converged warp: fewer instructions between a stage
         // falling free and its next copies, and no issue slots spent on votes.)
-        if (lane == 0) {
+        if (lane == 0 && !g.test_drop_copies) {
             int stage = 0;
             uint32_t phase = 0;
             for (int tile = pair; tile < ntiles && ok; tile += npairs) {
