@@ -70,7 +70,10 @@ typedef enum { EBRL_F32 = 0, EBRL_BF16 = 1 } ebrl_dtype_t;
                                      least sm_quota SMs when the driver offers one; the grid cap
                                      of sm_quota CTAs applies either way                         */
 #define EBRL_FLAG_TIMING      4u  /* record per-kernel-class device time (see get_stats)        */
-#define EBRL_FLAG_FORCE_SIMT  8u  /* bf16 models: use the plain-ALU kernels, not tensor cores    */
+#define EBRL_FLAG_FORCE_SIMT  8u  /* use the plain-ALU kernels, not tensor cores (bf16 models: for
+                                     every operation; fp32 models: for the projections, which
+                                     otherwise run on the tensor cores as six bf16 products per
+                                     term pair of three-term operand splits, fp32-accurate)       */
 #define EBRL_FLAG_NO_FUSED   16u  /* never use the persistent step kernel (one resident grid that
                                      walks all Euler steps of a small batch); always launch one
                                      kernel per operation                                        */

@@ -118,6 +118,12 @@ bool attn_mma_supported(int H, int n_heads, int hd);
 int attn_mma_make_map(TensorMap128 *out, const void *base, uint64_t rows, uint64_t width, int n_heads, int hd);
 cudaError_t launch_attn_mma(const AttnArgs &a, int grid, int lookahead_blocks, unsigned long long limit_ns, int *status, cudaStream_t st);
 
+// fp32 GEMM on the tensor cores by splitting each operand into three bf16 terms (six products per k-slice).
+bool gemm_tc3_supported(int N, int K);
+cudaError_t launch_split3(const float *src, void *p0, void *p1, void *p2, size_t n, int grid, cudaStream_t st);
+cudaError_t launch_gemm_tc3(const TensorMap128 *ta, const TensorMap128 *tw, const GemmArgs &a, int grid, unsigned long long limit_ns,
+                            int *status, cudaStream_t st);
+
 // ---- the persistent step kernel (one resident grid for all Euler steps of a small batch) ----
 // Per-layer table in device memory: TMA descriptors of the six matrices (128-row boxes) and the gains.
 struct alignas(64) FusedLayerTab {

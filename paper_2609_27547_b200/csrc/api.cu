@@ -33,6 +33,9 @@ struct LayerDev {
     void *w_qkv = nullptr, *w_o = nullptr, *w_qc = nullptr, *w_oc = nullptr, *w_1 = nullptr, *w_2 = nullptr;
     void *w_kc = nullptr, *w_vc = nullptr;           // hidden-state prefixes (cfg.d_ctx > 0): [d][d_ctx] each
     TensorMap128 t_qkv, t_o, t_qc, t_oc, t_1, t_2, t_kc, t_vc;   // TMA descriptors of the matrices (tensor-core path)
+    // fp32 models on the tensor cores: the three bf16 terms of each matrix (0 qkv, 1 o, 2 qc, 3 oc, 4 w_1, 5 w_2) and their descriptors
+    void *w3[6][3] = {};
+    TensorMap128 t3[6][3];
 };
 
 // One complete copy of the policy's weights on the device.  The handle keeps two, so that a new
@@ -65,6 +68,8 @@ struct Slot {
     void *xg = nullptr, *qkv = nullptr, *att = nullptr, *qc = nullptr, *u = nullptr;
     EnvMeta *meta_d = nullptr, *meta_h = nullptr;
     TensorMap128 t_xg, t_att, t_u;                    // TMA descriptors of the A operands
+    void *aspl[3] = {nullptr, nullptr, nullptr};      // fp32 models on the tensor cores: the three bf16 terms of the GEMM's A operand
+    TensorMap128 t_aspl_d[3], t_aspl_md[3];           // ... seen as [rows][d] and as [rows][md]
     FusedMaps *fmaps_d = nullptr;                     // persistent step kernel: the same plus the epilogues' store targets, in device memory
     int *fctl_d = nullptr, *fctl_h = nullptr;         // its control block: n_active[K] then the completion counters [K][mt_max]
     int mt_max = 0;
@@ -104,6 +109,7 @@ struct ebrl_actgen {
     ebrl_actgen_cfg_t cfg;
     int bf16 = 0, n_sms = 0, hd = 0, md = 0;
     bool use_tc = false;          // tensor-core GEMMs (bf16, d a multiple of 256)
+    bool use_tc3 = false;         // fp32 models: projections on the tensor cores by three-term bf16 splitting
     bool use_pairs = true;        // CTA-pair GEMM allowed (EBRL_GEMM_PAIR=0 forbids it)
     int force_shape = 0;          // EBRL_GEMM_SHAPE = 2 (pairs), 256 or 128 forces one tile shape (tests, tuning)
     bool trace = false;           // EBRL_TRACE=1: the persistent kernel notes its progress; a time-out prints it to stderr
@@ -330,6 +336,15 @@ ebrl_status_t alloc_weight_set(ebrl_actgen *h, WeightSet &ws)
                     return fail(h, EBRL_ERR_CUDA, "cuTensorMapEncodeTiled failed for a weight matrix");
             }
         }
+        if (h->use_tc3) {
+            const size_t rows_n[6] = {3 * d, d, d, d, md, d}, cols_k[6] = {d, d, d, d, d, md};
+            for (int m = 0; m < 6; ++m)
+                for (int t = 0; t < 3; ++t) {
+                    if ((st = dev_alloc(h, &o.w3[m][t], rows_n[m] * cols_k[m] * 2)) != EBRL_OK) return st;
+                    if (make_tmap_bf16(&o.t3[m][t], o.w3[m][t], cols_k[m], rows_n[m], 128))
+                        return fail(h, EBRL_ERR_CUDA, "cuTensorMapEncodeTiled failed for a weight matrix");
+                }
+        }
         if (h->use_tc) {
             const uint32_t bw = (uint32_t)gemm_tc_box_rows_w();
             int bad = make_tmap_bf16(&o.t_qkv, o.w_qkv, d, 3 * d, bw) | make_tmap_bf16(&o.t_o, o.w_o, d, d, bw) |
@@ -394,6 +409,19 @@ ebrl_status_t upload_weight_set(ebrl_actgen *h, WeightSet &ws, const ebrl_actgen
         if (e == cudaSuccess && c.d_ctx > 0) e = cp(o.w_vc, w.w_vc, d * (size_t)c.d_ctx * esz);
     }
     if (e != cudaSuccess) return fail(h, EBRL_ERR_CUDA, "copying the weights failed: %s", cudaGetErrorString(e));
+    if (h->use_tc3) {
+        // the three bf16 terms of every matrix, behind the copies on the same stream
+        cudaStream_t ss = async ? st : nullptr;
+        for (int l = 0; l < c.n_layers && e == cudaSuccess; ++l) {
+            LayerDev &o = ws.layers[l];
+            const void *src[6] = {o.w_qkv, o.w_o, o.w_qc, o.w_oc, o.w_1, o.w_2};
+            const size_t n[6] = {3 * d * d, d * d, d * d, d * d, md * d, d * md};
+            for (int m = 0; m < 6 && e == cudaSuccess; ++m)
+                e = launch_split3((const float *)src[m], o.w3[m][0], o.w3[m][1], o.w3[m][2], n[m], h->n_sms, ss);
+        }
+        if (e == cudaSuccess && !async) e = cudaStreamSynchronize(ss);
+        if (e != cudaSuccess) return fail(h, EBRL_ERR_CUDA, "splitting the weights failed: %s", cudaGetErrorString(e));
+    }
     return EBRL_OK;
 }
 
@@ -566,14 +594,18 @@ cudaError_t enqueue_batch(ebrl_actgen *h, Slot &s, int S, const int32_t *n_activ
             for (int l = 0; l < L; ++l) {
                 const LayerDev &w = W.layers[l];
                 auto gemm = [&](const void *A, const TensorMap128 &tA, const void *W, const TensorMap128 &tW, int N, int K, int epi,
-                                void *C, const float *gain) {
+                                void *C, const float *gain, const TensorMap128 *w3) {
                     GemmArgs g{};
                     g.A = A; g.W = W; g.M = M; g.N = N; g.K = K; g.epi = epi;
                     g.ssq_in = s.ssq; g.n_ssq = nseg; g.inv_d = 1.0f / (float)d; g.eps = c.rms_eps;
                     g.C = C; g.x = s.x; g.gain = gain; g.xg = s.xg; g.ssq_out = s.ssq;
                     g.test_drop_copies = (c.flags & EBRL_FLAG_TEST_DROP_GEMM_COPIES) ? 1 : 0;
                     const double bytes = ((double)M * K + (double)N * K + (double)M * N) * esz + (epi == EPI_RESID ? 8.0 * M * N : 0.0);
-                    if (h->use_tc) {
+                    if (h->use_tc3) {
+                        // split the fp32 activations into their three bf16 terms, then six tensor-core products per k-slice
+                        ln.run(EBRL_KC_GEMM, 0.0, 10.0 * M * K, [&] { return launch_split3((const float *)A, s.aspl[0], s.aspl[1], s.aspl[2], (size_t)M * K, grid, st); });
+                        ln.run(EBRL_KC_GEMM, 2.0 * M * N * K, bytes, [&] { return launch_gemm_tc3(K == d ? s.t_aspl_d : s.t_aspl_md, w3, g, grid, h->wait_ns, h->status_d, st); });
+                    } else if (h->use_tc) {
                         const int shape = pick_tile_shape(h, M, N, grid);
                         if (shape == 2)
                             ln.run(EBRL_KC_GEMM, 2.0 * M * N * K, bytes, [&] { return launch_gemm_tc2(tA, tW, g, grid, h->wait_ns, h->status_d, st); });
@@ -584,7 +616,7 @@ cudaError_t enqueue_batch(ebrl_actgen *h, Slot &s, int S, const int32_t *n_activ
                         ln.run(EBRL_KC_GEMM, 2.0 * M * N * K, bytes, [&] { return launch_gemm_simt(g, bf, grid, st); });
                 };
                 // self-attention block
-                gemm(s.xg, s.t_xg, w.w_qkv, w.t_qkv, 3 * d, d, EPI_SCALE_STORE, s.qkv, nullptr);
+                gemm(s.xg, s.t_xg, w.w_qkv, w.t_qkv, 3 * d, d, EPI_SCALE_STORE, s.qkv, nullptr, w.t3[0]);
                 {
                     AttnArgs a{};
                     a.q = s.qkv; a.q_stride = 3 * d; a.out = s.att; a.o_stride = d;
@@ -597,9 +629,9 @@ cudaError_t enqueue_batch(ebrl_actgen *h, Slot &s, int S, const int32_t *n_activ
                     a.self_map = s.maps_d; a.kv_maps = s.maps_d + 1;
                     ln.run(EBRL_KC_SELF_ATTN, 4.0 * M * H * d, 4.0 * M * d * esz, [&] { return launch_attn(h, a, grid, st); });
                 }
-                gemm(s.att, s.t_att, w.w_o, w.t_o, d, d, EPI_RESID, nullptr, w.g2);
+                gemm(s.att, s.t_att, w.w_o, w.t_o, d, d, EPI_RESID, nullptr, w.g2, w.t3[1]);
                 // cross-attention block
-                gemm(s.xg, s.t_xg, w.w_qc, w.t_qc, d, d, EPI_SCALE_STORE, s.qc, nullptr);
+                gemm(s.xg, s.t_xg, w.w_qc, w.t_qc, d, d, EPI_SCALE_STORE, s.qc, nullptr, w.t3[2]);
                 {
                     AttnArgs a{};
                     a.q = s.qc; a.q_stride = d; a.out = s.att; a.o_stride = d;
@@ -611,10 +643,10 @@ cudaError_t enqueue_batch(ebrl_actgen *h, Slot &s, int S, const int32_t *n_activ
                     ln.run(EBRL_KC_CROSS_ATTN, 4.0 * H * sum_P_active[step] * d,
                            2.0 * sum_P_active[step] * d * esz + 2.0 * M * d * esz, [&] { return launch_attn(h, a, grid, st); });
                 }
-                gemm(s.att, s.t_att, w.w_oc, w.t_oc, d, d, EPI_RESID, nullptr, w.g3);
+                gemm(s.att, s.t_att, w.w_oc, w.t_oc, d, d, EPI_RESID, nullptr, w.g3, w.t3[3]);
                 // MLP block
-                gemm(s.xg, s.t_xg, w.w_1, w.t_1, md, d, EPI_SCALE_GELU, s.u, nullptr);
-                gemm(s.u, s.t_u, w.w_2, w.t_2, d, md, EPI_RESID, nullptr, (l + 1 < L) ? W.layers[l + 1].g1 : W.g_final);
+                gemm(s.xg, s.t_xg, w.w_1, w.t_1, md, d, EPI_SCALE_GELU, s.u, nullptr, w.t3[4]);
+                gemm(s.u, s.t_u, w.w_2, w.t_2, d, md, EPI_RESID, nullptr, (l + 1 < L) ? W.layers[l + 1].g1 : W.g_final, w.t3[5]);
             }
         }
         HeadArgs ha{s.meta_d, ne, H, c.A, d, step, c.K_steps, s.a_state, s.x, W.g_final, W.w_out, W.b_out, c.rms_eps, pull ? 1 : 0};
@@ -1004,6 +1036,8 @@ ebrl_status_t ebrl_actgen_create(const ebrl_actgen_cfg_t *cfg, const ebrl_actgen
     if (const char *e4 = getenv("EBRL_PDL")) h->pdl_allowed = atoi(e4) != 0;
     if (const char *e5 = getenv("EBRL_ATTN_LOOKAHEAD")) h->attn_lookahead = std::min(64, std::max(0, atoi(e5)));
     h->use_attn_mma = h->bf16 && !(cfg->flags & EBRL_FLAG_FORCE_SIMT) && attn_mma_supported(cfg->H, cfg->n_heads, h->hd);
+    h->use_tc3 = !h->bf16 && !(cfg->flags & EBRL_FLAG_FORCE_SIMT) && gemm_tc3_supported(d, d) && gemm_tc3_supported(md, d) &&
+                 gemm_tc3_supported(d, md) && gemm_tc3_supported(3 * d, d);
     h->fused_ok = h->use_tc && h->use_attn_mma && fused_supported(cfg->H, cfg->A, d, md, cfg->n_heads, h->hd);
     if (const char *e6 = getenv("EBRL_FUSED_MAX_ROWS")) h->fused_max_rows = atol(e6);
     if (const char *e7 = getenv("EBRL_TRACE")) h->trace = atoi(e7) != 0;
@@ -1085,6 +1119,16 @@ ebrl_status_t ebrl_actgen_create(const ebrl_actgen_cfg_t *cfg, const ebrl_actgen
             int bad = make_tmap_bf16(&s.t_xg, s.xg, d, rows, ba) | make_tmap_bf16(&s.t_att, s.att, d, rows, ba) |
                       make_tmap_bf16(&s.t_u, s.u, md, rows, ba);
             if (bad) { fail(h, EBRL_ERR_CUDA, "cuTensorMapEncodeTiled failed for a workspace"); return bail(EBRL_ERR_CUDA); }
+        }
+        if (h->use_tc3) {
+            for (int t = 0; t < 3; ++t) {
+                if ((st = dev_alloc(h, &s.aspl[t], rows * md * 2, "a split-operand workspace")) != EBRL_OK) return bail(st);
+                if (cudaMemset(s.aspl[t], 0, rows * md * 2) != cudaSuccess) { fail(h, EBRL_ERR_CUDA, "cudaMemset of the workspace failed"); return bail(EBRL_ERR_CUDA); }
+                if (make_tmap_bf16(&s.t_aspl_d[t], s.aspl[t], d, rows, 128) | make_tmap_bf16(&s.t_aspl_md[t], s.aspl[t], md, rows, 128)) {
+                    fail(h, EBRL_ERR_CUDA, "cuTensorMapEncodeTiled failed for a workspace");
+                    return bail(EBRL_ERR_CUDA);
+                }
+            }
         }
         if (h->fused_ok) {
             FusedMaps fm;

@@ -126,7 +126,18 @@ template <bool COH> __device__ __forceinline__ float ld_f1(const float *p)
 // All 32 lanes must call it.  `wait` blocks until the accumulator is complete (false on a
 // time-out); the residual values of the first chunk are requested before it and those of each
 // later chunk one chunk ahead.
-template <int EPI, int NCOLS, bool COH = false, typename WaitF>
+// Four consecutive outputs of a row in the activations' type: bf16 (8 bytes) or fp32 (16 bytes).
+template <typename OT> __device__ __forceinline__ void store_out4(OT *p, float a, float b, float c, float d);
+template <> __device__ __forceinline__ void store_out4<__nv_bfloat16>(__nv_bfloat16 *p, float a, float b, float c, float d)
+{
+    *reinterpret_cast<uint2 *>(p) = make_uint2(pack_bf16(a, b), pack_bf16(c, d));
+}
+template <> __device__ __forceinline__ void store_out4<float>(float *p, float a, float b, float c, float d)
+{
+    *reinterpret_cast<float4 *>(p) = make_float4(a, b, c, d);
+}
+
+template <int EPI, int NCOLS, bool COH = false, typename OT = __nv_bfloat16, typename WaitF>
 __device__ __forceinline__ bool epilogue_rows(const GemmArgs &g, uint32_t taddr, int row0, int n0, float *stg_generic, WaitF wait)
 {
     constexpr int NC = NCOLS / 32;
@@ -185,7 +196,7 @@ __device__ __forceinline__ bool epilogue_rows(const GemmArgs &g, uint32_t taddr,
         __syncwarp();
         if (EPI == EPI_RESID) {
             const float4 gn = *reinterpret_cast<const float4 *>(g.gain + col + 4 * piece);
-            __nv_bfloat16 *__restrict__ xg = (__nv_bfloat16 *)g.xg;
+            OT *__restrict__ xg = (OT *)g.xg;
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const int rr = 4 * i + sub;
@@ -194,7 +205,7 @@ __device__ __forceinline__ bool epilogue_rows(const GemmArgs &g, uint32_t taddr,
                     float4 xn;
                     xn.x = xv[i].x + acc[i].x; xn.y = xv[i].y + acc[i].y; xn.z = xv[i].z + acc[i].z; xn.w = xv[i].w + acc[i].w;
                     *reinterpret_cast<float4 *>(xg_x + off) = xn;
-                    *reinterpret_cast<uint2 *>(xg + off) = make_uint2(pack_bf16(xn.x * gn.x, xn.y * gn.y), pack_bf16(xn.z * gn.z, xn.w * gn.w));
+                    store_out4<OT>(xg + off, xn.x * gn.x, xn.y * gn.y, xn.z * gn.z, xn.w * gn.w);
                     ssp[i] = fmaf(xn.x, xn.x, ssp[i]); ssp[i] = fmaf(xn.y, xn.y, ssp[i]);
                     ssp[i] = fmaf(xn.z, xn.z, ssp[i]); ssp[i] = fmaf(xn.w, xn.w, ssp[i]);
                 }
@@ -205,13 +216,11 @@ __device__ __forceinline__ bool epilogue_rows(const GemmArgs &g, uint32_t taddr,
                     if (4 * i + sub < nrows) xv[i] = ld_f4<COH>(xg_x + (size_t)(row0 + 4 * i + sub) * g.N + col + 32 + 4 * piece);
             }
         } else {
-            __nv_bfloat16 *__restrict__ cp = (__nv_bfloat16 *)g.C;
+            OT *__restrict__ cp = (OT *)g.C;
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const int rr = 4 * i + sub;
-                if (rr < nrows)
-                    *reinterpret_cast<uint2 *>(cp + (size_t)(row0 + rr) * g.N + col + 4 * piece) =
-                        make_uint2(pack_bf16(acc[i].x, acc[i].y), pack_bf16(acc[i].z, acc[i].w));
+                if (rr < nrows) store_out4<OT>(cp + (size_t)(row0 + rr) * g.N + col + 4 * piece, acc[i].x, acc[i].y, acc[i].z, acc[i].w);
             }
         }
     }

@@ -25,15 +25,15 @@ SEED = synth.DEFAULT_SEED
 LIMIT_NS = 50_000_000
 
 
-def _tiny():
-    w = synth.scaled(synth.WORKLOADS[0], B=4, dtype="bf16", d=256, n_heads=4, L=1, K=1, P=(16, 40))
+def _tiny(dtype="bf16"):
+    w = synth.scaled(synth.WORKLOADS[0], B=4, dtype=dtype, d=256, n_heads=4, L=1, K=1, P=(16, 40))
     wt = synth.make_weights(w, SEED, random_gains=True)
     envs = [synth.make_env(w, e, SEED) for e in range(w.B)]
     return w, wt, envs
 
 
-def _expect_timeout_then_recover(flags, monkeypatch=None, shape=None):
-    w, wt, envs = _tiny()
+def _expect_timeout_then_recover(flags, monkeypatch=None, shape=None, dtype="bf16"):
+    w, wt, envs = _tiny(dtype)
     ids = list(range(w.B))
     if shape is not None:
         monkeypatch.setenv("EBRL_GEMM_SHAPE", shape)
@@ -60,7 +60,12 @@ def _expect_timeout_then_recover(flags, monkeypatch=None, shape=None):
     r = Runner(w, wt, envs)
     got = stack(r.run([ids]), ids)
     r.close()
-    assert chunk_rel_err(got, oracle_run(w, wt, envs)) <= TOL["bf16"]
+    assert chunk_rel_err(got, oracle_run(w, wt, envs)) <= TOL[dtype]
+
+
+def test_fp32_tensor_core_projection_kernel_gives_up_cleanly():
+    """The split-operand kernel of the fp32 models (six operand tiles per stage)."""
+    _expect_timeout_then_recover(B.FLAG_TEST_DROP_GEMM_COPIES, dtype="f32")
 
 
 @pytest.mark.parametrize("shape", ["128", "256", "2"])

@@ -75,6 +75,29 @@ def test_every_gemm_tile_shape_every_row_against_the_oracle(monkeypatch):
     r.close()
 
 
+def test_fp32_projections_on_tensor_cores_and_on_the_plain_alus():
+    """fp32 models run their projections on the tensor cores (every operand the exact sum of three
+    bf16 terms, six products per term pair) unless told to use the FFMA kernels.  Both must stay
+    within the fp32 bound of the oracle on a model with long reductions (d = 512, MLP width 2048),
+    several row tiles and a ragged tail; the tensor-core path must also be quota-independent."""
+    w = synth.scaled(synth.WORKLOADS[0], B=37, dtype="f32", d=512, n_heads=8, L=3, K=4, P=(1, 97), mixed_steps=True)
+    wt, envs = _setup(w)
+    ref = oracle_run(w, wt, envs)
+    ids = list(range(w.B))
+    r = Runner(w, wt, envs)
+    got = stack(r.run([ids]), ids)
+    assert chunk_rel_err(got, ref) <= TOL["f32"]
+    for q in (16, 37, 74):
+        assert np.array_equal(stack(r.run([ids], quota=q), ids), got)
+    assert np.array_equal(stack(r.run([ids[:9], ids[9:]]), ids), got)
+    r.close()
+    r = Runner(w, wt, envs, flags=B.FLAG_FORCE_SIMT)
+    alu = stack(r.run([ids]), ids)
+    r.close()
+    assert chunk_rel_err(alu, ref) <= TOL["f32"]
+    print("fp32 max chunk-relative error: tensor cores %.2e, FFMA %.2e" % (chunk_rel_err(got, ref), chunk_rel_err(alu, ref)))
+
+
 def test_bf16_plain_alu_kernels_parity():
     """The bf16 model on the plain-ALU kernels (the path taken when d is not a multiple of 256,
     and on request)."""
@@ -453,7 +476,9 @@ def test_queue_semantics_flush_streams_and_timing():
     s1.synchronize()
     assert np.array_equal(out_a.cpu().numpy(), base)
     n1 = r.gen.stats()["kernel_launches"]
-    assert n1 == w.K * (w.L * 8 + 2)                                        # one batch, not two
+    # one batch, not two: per Euler step embed + head, per layer six projections and two attentions -- and for an
+    # fp32 model six more launches that split the projections' fp32 operands into bf16 terms for the tensor cores
+    assert n1 == w.K * (w.L * (8 + (6 if w.dtype == "f32" else 0)) + 2)
     r.gen.sync()                                                             # retire: the ids may be used again
     r.gen.submit(ids[:5], kv[:5], noise[:5], out_b[:5], stream=s1, sm_quota=37)
     r.gen.submit(ids[5:], kv[5:], noise[5:], out_c[5:], stream=s2, sm_quota=37)   # other stream: closes the first batch
@@ -465,7 +490,8 @@ def test_queue_semantics_flush_streams_and_timing():
     assert stt["kernel_launches"] == 3 * n1 and stt["groups"] == 4
     cls = stt["classes"]
     assert sum(c["launches"] for c in cls.values()) == stt["kernel_launches"]
-    assert cls["gemm"]["launches"] == 3 * w.K * w.L * 6 and cls["gemm"]["ms"] > 0 and cls["gemm"]["flops"] > 0
+    assert cls["gemm"]["launches"] == 3 * w.K * w.L * (12 if w.dtype == "f32" else 6)    # fp32: operand split + projection
+    assert cls["gemm"]["ms"] > 0 and cls["gemm"]["flops"] > 0
     assert cls["cross_attn"]["bytes"] > 0 and cls["head"]["launches"] == 3 * w.K
     r.close()
 
