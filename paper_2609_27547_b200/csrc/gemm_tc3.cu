@@ -12,9 +12,12 @@
 // Weights are split once, when they are copied into the handle; activations are split by
 // split3_kernel right before the GEMM that reads them.  The GEMM is the single-CTA 128 x 128
 // tensor-core kernel with six operand tiles per 64-wide k-block (96 KB per stage, two stages) and
-// the same fused epilogues on fp32 outputs.  Every output element is the sum over k in order of its
-// six products in the order above, whatever the grid size: results do not depend on the SM quota
-// or on which rows share a tile.  Every wait is bounded (status word, as in the other kernels).
+// the same fused epilogues on fp32 outputs.  With K of a few hundred the epilogue of a tile takes
+// longer than its mainloop, so two groups of four epilogue warps drain the two accumulators in
+// turn (tile i by group i mod 2): two epilogues run while the next tile accumulates.  Every output
+// element is the sum over k in order of its six products in the order above, whatever the grid
+// size: results do not depend on the SM quota or on which rows share a tile.  Every wait is
+// bounded (status word, as in the other kernels).
 #include "actgen_internal.h"
 #include "ptx_helpers.cuh"
 #include "gemm_epilogue.cuh"
@@ -27,7 +30,7 @@ namespace tc3 {
 using namespace ptx;
 using namespace tc;
 
-constexpr int BM = 128, BN = 128, BK = 64, UMMA_K = 16, STAGES = 2, EPI_WARPS = 4;
+constexpr int BM = 128, BN = 128, BK = 64, UMMA_K = 16, STAGES = 2, EPI_WARPS = 8;   // two groups of four
 constexpr int TILE_BYTES = BM * BK * 2;                 // one bf16 operand tile
 constexpr int STAGE_BYTES = 6 * TILE_BYTES;             // A0 A1 A2 W0 W1 W2
 constexpr int THREADS = 64 + 32 * EPI_WARPS;
@@ -88,7 +91,7 @@ gemm_tc3_kernel(const __grid_constant__ Maps6 tm, GemmArgs g, unsigned long long
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(tfull(b), 1); mbar_init(tempty(b), EPI_WARPS); }
+        for (int b = 0; b < 2; ++b) { mbar_init(tfull(b), 1); mbar_init(tempty(b), EPI_WARPS / 2); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         for (int i = 0; i < 3; ++i) {
@@ -169,12 +172,14 @@ gemm_tc3_kernel(const __grid_constant__ Maps6 tm, GemmArgs g, unsigned long long
         __syncwarp();
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
     } else {
-        // ---- epilogue: warp w reads TMEM lanes 32 (w % 4) .. +31; one thread per row; fp32 outputs
-        const int q = warp & 3;
+        // ---- epilogue: warp w reads TMEM lanes 32 (w % 4) .. +31; one thread per row; fp32 outputs;
+        // group (w - 2) / 4 owns accumulator (w - 2) / 4, i.e. every other tile of this CTA
+        const int q = warp & 3, grp = (warp - 2) >> 2;
         float *stg = reinterpret_cast<float *>(smem + STAGES * STAGE_BYTES) + (warp - 2) * EPI_STAGE_FLOATS;
         int it = 0;
         for (int tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++it) {
             const int buf = it & 1;
+            if (buf != grp) continue;
             const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
             const int m0 = (tile / ntn) * BM, n0 = (tile % ntn) * BN;
             auto acc_ready = [&] { return __all_sync(0xffffffffu, mbar_wait_relaxed(tfull(buf), acc_phase, limit_ns, abort_flag)) != 0; };

@@ -191,8 +191,11 @@ template <> __device__ __forceinline__ void load4<__nv_bfloat16>(const __nv_bflo
     v[0] = __bfloat162float(lo.x); v[1] = __bfloat162float(lo.y); v[2] = __bfloat162float(hi.x); v[3] = __bfloat162float(hi.y);
 }
 
-template <typename T, int RMAX>
-__global__ void __launch_bounds__(512) attn_simt_kernel(AttnArgs a)
+// GROUPS items are in flight per CTA (one per 128 threads).  With head_dim <= 64 a thread's share of the next key
+// block (four 16-byte pieces of K and of V) is requested into registers while the current block is computed, so the
+// global-memory latency of a block hides behind the arithmetic of the one before it.
+template <typename T, int RMAX, int GROUPS>
+__global__ void __launch_bounds__(GROUPS * 128) attn_simt_kernel(AttnArgs a)
 {
     extern __shared__ __align__(16) float smem[];
     const int grp = threadIdx.x >> 7, t = threadIdx.x & 127, warp = t >> 5, lane = t & 31;
@@ -210,7 +213,8 @@ __global__ void __launch_bounds__(512) attn_simt_kernel(AttnArgs a)
     const int items = a.n_envs * a.n_heads;
     pdl_launch_dependents();
     pdl_wait();
-    for (int item = blockIdx.x * 4 + grp; item < items; item += gridDim.x * 4) {
+    const bool ahead = hd <= 64;     // 32 * (hd / 4) / 128 <= 4 pieces per thread and plane
+    for (int item = blockIdx.x * GROUPS + grp; item < items; item += gridDim.x * GROUPS) {
         const int env = item / a.n_heads, h = item - env * a.n_heads;
         const T *kbase, *vbase;
         int P, kvs;
@@ -236,18 +240,48 @@ __global__ void __launch_bounds__(512) attn_simt_kernel(AttnArgs a)
         float mrun[8], lrun[8];   // rows warp, warp+4, ... (H <= 32)
 #pragma unroll
         for (int r = 0; r < 8; ++r) { mrun[r] = -INFINITY; lrun[r] = 0.f; }
+        // this thread's pieces of a key block: piece u is key j = e >> (hd_sh - 2), columns cc .. cc + 3, e = t + 128 u
+        float kreg[4][4], vreg[4][4];
+        auto fetch_block = [&](int j0) {
+            const int nk = min(AKB, P - j0);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int e = t + 128 * u;
+                const int j = e >> (hd_sh - 2), cc = (e & ((hd >> 2) - 1)) << 2;
+#pragma unroll
+                for (int x = 0; x < 4; ++x) kreg[u][x] = vreg[u][x] = 0.f;
+                if (e < AKB * (hd >> 2) && j < nk) {
+                    load4(kbase + (size_t)(j0 + j) * kvs + cc, kreg[u]);
+                    load4(vbase + (size_t)(j0 + j) * kvs + cc, vreg[u]);
+                }
+            }
+        };
+        if (ahead) fetch_block(0);
         for (int j0 = 0; j0 < P; j0 += AKB) {
             group_sync(grp);   // q ready; previous block's readers done
             const int nkeys = min(AKB, P - j0);
-            for (int e = t; e < AKB * (hd >> 2); e += 128) {   // four columns per thread and turn
-                const int j = e >> (hd_sh - 2), cc = (e & ((hd >> 2) - 1)) << 2;
-                float kv[4] = {0.f, 0.f, 0.f, 0.f}, vv[4] = {0.f, 0.f, 0.f, 0.f};
-                if (j < nkeys) {
-                    load4(kbase + (size_t)(j0 + j) * kvs + cc, kv);
-                    load4(vbase + (size_t)(j0 + j) * kvs + cc, vv);
+            if (ahead) {
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int e = t + 128 * u;
+                    if (e < AKB * (hd >> 2)) {
+                        const int j = e >> (hd_sh - 2), cc = (e & ((hd >> 2) - 1)) << 2;
+                        *reinterpret_cast<float4 *>(kb + j * (hd + 4) + cc) = make_float4(kreg[u][0], kreg[u][1], kreg[u][2], kreg[u][3]);
+                        *reinterpret_cast<float4 *>(vb + j * hd + cc) = make_float4(vreg[u][0], vreg[u][1], vreg[u][2], vreg[u][3]);
+                    }
                 }
-                *reinterpret_cast<float4 *>(kb + j * (hd + 4) + cc) = make_float4(kv[0], kv[1], kv[2], kv[3]);
-                *reinterpret_cast<float4 *>(vb + j * hd + cc) = make_float4(vv[0], vv[1], vv[2], vv[3]);
+                if (j0 + AKB < P) fetch_block(j0 + AKB);   // lands while this block is computed
+            } else {
+                for (int e = t; e < AKB * (hd >> 2); e += 128) {   // four columns per thread and turn
+                    const int j = e >> (hd_sh - 2), cc = (e & ((hd >> 2) - 1)) << 2;
+                    float kv[4] = {0.f, 0.f, 0.f, 0.f}, vv[4] = {0.f, 0.f, 0.f, 0.f};
+                    if (j < nkeys) {
+                        load4(kbase + (size_t)(j0 + j) * kvs + cc, kv);
+                        load4(vbase + (size_t)(j0 + j) * kvs + cc, vv);
+                    }
+                    *reinterpret_cast<float4 *>(kb + j * (hd + 4) + cc) = make_float4(kv[0], kv[1], kv[2], kv[3]);
+                    *reinterpret_cast<float4 *>(vb + j * hd + cc) = make_float4(vv[0], vv[1], vv[2], vv[3]);
+                }
             }
             group_sync(grp);
             // scores and running softmax statistics: lane = key, each warp owns rows warp + 4 r
@@ -422,34 +456,34 @@ cudaError_t launch_gemm_simt(const GemmArgs &a, int bf16, int grid, cudaStream_t
     return bf16 ? gemm_simt_dispatch<__nv_bfloat16>(a, g, st) : gemm_simt_dispatch<float>(a, g, st);
 }
 
-template <typename T, int RMAX>
-static cudaError_t attn_launch(const AttnArgs &a, int g, size_t smem, cudaStream_t st)
+template <typename T, int RMAX, int GROUPS>
+static cudaError_t attn_launch(const AttnArgs &a, int grid, cudaStream_t st)
 {
-    cudaError_t e = cudaFuncSetAttribute(attn_simt_kernel<T, RMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const int items = a.n_envs * a.n_heads;
+    const int need = (items + GROUPS - 1) / GROUPS;
+    const int g = need < grid ? need : grid;
+    const size_t per_group = ((size_t)a.H * a.hd + AKB * (a.hd + 4) + AKB * a.hd + a.H * AKB + 2 * a.H + 3) & ~(size_t)3;
+    const size_t smem = GROUPS * per_group * sizeof(float);
+    cudaError_t e = cudaFuncSetAttribute(attn_simt_kernel<T, RMAX, GROUPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    return launch_kernel(attn_simt_kernel<T, RMAX>, g, 512, smem, st, 1, a);
+    return launch_kernel(attn_simt_kernel<T, RMAX, GROUPS>, g, GROUPS * 128, smem, st, 1, a);
 }
 
 template <typename T>
-static cudaError_t attn_dispatch(const AttnArgs &a, int g, size_t smem, cudaStream_t st)
+static cudaError_t attn_dispatch(const AttnArgs &a, int grid, cudaStream_t st)
 {
     const int ncg = 128 / a.hd;
     const int R = (a.H + ncg - 1) / ncg;
-    if (R <= 4) return attn_launch<T, 4>(a, g, smem, st);
-    if (R <= 8) return attn_launch<T, 8>(a, g, smem, st);
-    if (R <= 16) return attn_launch<T, 16>(a, g, smem, st);
-    return attn_launch<T, 32>(a, g, smem, st);
+    if (R <= 4) return attn_launch<T, 4, 4>(a, grid, st);
+    if (R <= 8) return attn_launch<T, 8, 4>(a, grid, st);
+    if (R <= 16) return attn_launch<T, 16, 4>(a, grid, st);
+    return attn_launch<T, 32, 4>(a, grid, st);
 }
 
 cudaError_t launch_attn_simt(const AttnArgs &a, int bf16, int grid, cudaStream_t st)
 {
-    const int items = a.n_envs * a.n_heads;
-    if (items == 0) return cudaSuccess;
-    const int need = (items + 3) / 4;
-    const int g = need < grid ? need : grid;
-    const size_t per_group = ((size_t)a.H * a.hd + AKB * (a.hd + 4) + AKB * a.hd + a.H * AKB + 2 * a.H + 3) & ~(size_t)3;
-    const size_t smem = 4 * per_group * sizeof(float);
-    return bf16 ? attn_dispatch<__nv_bfloat16>(a, g, smem, st) : attn_dispatch<float>(a, g, smem, st);
+    if (a.n_envs * a.n_heads == 0) return cudaSuccess;
+    return bf16 ? attn_dispatch<__nv_bfloat16>(a, grid, st) : attn_dispatch<float>(a, grid, st);
 }
 
 }  // namespace ebrl
