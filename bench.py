@@ -85,6 +85,8 @@ def parse_args(argv=None):
     ap.add_argument("--min-warmup", type=int, default=3, help="lower bound on warm-up steps (profiling captures use 1)")
     ap.add_argument("--d-ctx", type=int, default=0, help="variant: prefixes are hidden states [P][d_ctx], projected to K/V per layer")
     ap.add_argument("--inflight", type=int, default=16, help="groups queued before a batch is launched")
+    ap.add_argument("--fused", action="store_true",
+                    help="run every batch through the persistent step kernel (one resident grid for all Euler steps)")
     ap.add_argument("--sweep", action="store_true",
                     help="one line per other configuration: configs[0..2], and configs[3] at quotas 148/74/37/16 with and "
                          "without the streaming co-runner (the committed summary of these lines sits with the profiles)")
@@ -349,7 +351,8 @@ def run_ours(args, emit=True):
     out = torch.empty_like(noise)
     kv_bytes = sum(envs[e].kv.numel() * envs[e].kv.element_size() for e in ids)
     inflight = args.inflight
-    flags = (B.FLAG_FORCE_SIMT if args.simt else 0) | (B.FLAG_GREEN_CTX if args.green_ctx else 0)
+    flags = (B.FLAG_FORCE_SIMT if args.simt else 0) | (B.FLAG_GREEN_CTX if args.green_ctx else 0) | \
+        (B.FLAG_FORCE_FUSED if args.fused else 0)
     cfg = B.cfg_for(w, max_group_envs=max(len(g) for g in groups), max_inflight_groups=inflight, flags=flags, device=local)
     gen = B.ActGen(cfg, wt)
     stream = torch.cuda.Stream(dev)
@@ -428,19 +431,23 @@ def run_ours(args, emit=True):
     gen.set_timing(False)
     cls = st["classes"]
     total_ms = sum(c["ms"] for c in cls.values()) or 1.0
-    gemm = cls["gemm"]
+    gemm = cls["fused"] if cls["fused"]["launches"] else cls["gemm"]
     bf16 = w.dtype == "bf16"
-    use_tensor = bf16 and not args.simt
+    use_tensor = not args.simt            # fp32 models run their projections on the tensor cores too, as six bf16 products each
     mhz = clocks2.get("sm_mhz") or clocks.get("sm_mhz") or 1965.0
-    per_clk = BF16_FLOP_PER_CLK_SM if use_tensor else FP32_FLOP_PER_CLK_SM
+    per_clk = (BF16_FLOP_PER_CLK_SM / (1.0 if bf16 else 6.0)) if use_tensor else FP32_FLOP_PER_CLK_SM
     peak_clock = q_eff * per_clk * mhz * 1e6 / 1e12
     achieved = gemm["flops"] / (gemm["ms"] * 1e-3) / 1e12 if gemm["ms"] > 0 else 0.0
     if use_tensor:
         bound = "tensor"
-        alt = {"measured_burst_x_quota": peaks["bf16_tflops"] * q_eff / N_SMS,
-               "measured_sustained_x_quota": peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) * q_eff / N_SMS,
-               "nominal_2250_x_quota": NOMINAL_BF16_TFLOPS * q_eff / N_SMS}
-        peak_note = ("%d SMs x %d FLOP/clk x %.0f MHz (median SM clock sampled during the per-kernel timing pass); the %s full-chip "
+        div = 1.0 if bf16 else 6.0
+        alt = {"measured_burst_x_quota": peaks["bf16_tflops"] * q_eff / N_SMS / div,
+               "measured_sustained_x_quota": peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) * q_eff / N_SMS / div,
+               "nominal_2250_x_quota": NOMINAL_BF16_TFLOPS * q_eff / N_SMS / div}
+        if not bf16:
+            alt["fp32_ffma_at_max_clock_x_quota"] = FP32_ALU_TFLOPS * q_eff / N_SMS
+        peak_note = ("fp32 products as six bf16 tensor-core products each: the bf16 figures divided by 6; " if not bf16 else "") + \
+                    ("%d SMs x %d FLOP/clk x %.0f MHz (median SM clock sampled during the per-kernel timing pass); the %s full-chip "
                      "figures (burst %.1f, sustained %.1f TFLOP/s, taken at a power-capped clock) scaled by %d/%d are in frac_vs"
                      % (q_eff, per_clk, mhz, peaks["source"], peaks["bf16_tflops"],
                         peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]), q_eff, N_SMS))
@@ -449,7 +456,7 @@ def run_ours(args, emit=True):
         alt = {"fp32_ffma_at_max_clock_x_quota": FP32_ALU_TFLOPS * q_eff / N_SMS}
         peak_note = "%d SMs x 128 FFMA lanes x 2 x %.0f MHz (median SM clock sampled during the per-kernel timing pass)" % (q_eff, mhz)
     traffic, traffic_note = gemm_traffic(w, st, gemm)
-    roofline = {"bound": bound, "kernel": "gemm", "achieved": achieved, "peak": peak_clock, "unit": "TFLOP/s",
+    roofline = {"bound": bound, "kernel": "fused_steps" if cls["fused"]["launches"] else "gemm", "achieved": achieved, "peak": peak_clock, "unit": "TFLOP/s",
                 "frac": achieved / peak_clock if peak_clock else None,
                 "frac_vs": {k: achieved / v for k, v in alt.items()}, "peak_alternatives": alt,
                 "traffic": traffic, "traffic_note": traffic_note,
@@ -526,6 +533,7 @@ def run_ours(args, emit=True):
                        "L": w.L, "heads": w.n_heads, "P": list(w.P), "K": w.K, "d_ctx": w.d_ctx, "groups": len(groups),
                        "group_sizes": [min(map(len, groups)), max(map(len, groups))], "sm_quota": q_eff,
                        "inflight_groups": inflight, "corunner": co_report if co_report is not None else False,
+                       "kernels": "persistent step kernel" if args.fused else ("plain ALU" if args.simt else "one kernel per operation"),
                        "green_ctx": {"requested": bool(args.green_ctx), "active": bool(st0["green_ctx_active"]), "partition_sms": st0["green_ctx_sms"]},
                        "sharding": "environment id mod %d; no data-path collective" % world,
                        "l2": ("inputs (%.2f GB of prefix planes plus weights) larger than the 126 MB L2" % (kv_bytes / 1e9))
@@ -563,16 +571,16 @@ def gemm_traffic(w, st, gemm):
 def run_sweep(args):
     """One JSON line per other configuration (the bench line proper is configs[4])."""
     import copy
-    plan = [(0, 0, False), (1, 0, False), (2, 0, False)]
+    plan = [(0, -1, False), (1, -1, False), (2, -1, False)]
     for q in (148, 74, 37, 16):
         plan.append((3, q, False))
         if q < N_SMS:
             plan.append((3, q, True))
+    plan += [(4, 148, False), (4, 37, False)]                 # the bench configuration at other quotas than its own 74
     for cfg_i, q, co in plan:
         a = copy.copy(args)
-        a.config, a.corunner, a.no_cpu, a.no_e2e = cfg_i, co, True, True
-        a.quota = q if cfg_i == 3 else -1
-        a.steps = max(args.steps, 20) if cfg_i != 1 else max(args.steps, 10)
+        a.config, a.corunner, a.no_cpu, a.no_e2e, a.quota = cfg_i, co, True, True, q
+        a.steps = {1: 10, 4: 3}.get(cfg_i, max(args.steps, 20))
         run_ours(a)
 
 
@@ -590,7 +598,7 @@ def run_pgen_sweep(args):
     quotas, batches = [20, 40, 60, 80], [8, 16, 32, 64]
     wt = synth.make_weights(w, seed, device="cuda")
     envs = [synth.make_env(w, e, seed, device="cuda") for e in range(max(batches))]
-    gen = B.ActGen(B.cfg_for(w, max_group_envs=max(batches), max_inflight_groups=1), wt)
+    gen = B.ActGen(B.cfg_for(w, max_group_envs=max(batches), max_inflight_groups=1, flags=B.FLAG_FORCE_FUSED if args.fused else 0), wt)
     stream = torch.cuda.Stream()
     noise = torch.stack([e.noise for e in envs]).contiguous()
     out = torch.empty_like(noise)
@@ -614,6 +622,7 @@ def run_pgen_sweep(args):
         rate.append(row)
     gen.destroy()
     print(json.dumps({"pgen": {"workload": "configs[%d] %s" % (args.config, w.name), "unit": UNIT, "quota_pct": quotas,
+                               "kernels": "persistent step kernel" if args.fused else "one kernel per operation",
                                "quota_sms": [max(1, round(N_SMS * q / 100)) for q in quotas], "batch": batches, "rate": rate}}))
 
 

@@ -195,6 +195,15 @@ ebrl_status_t ebrl_actgen_create(const ebrl_actgen_cfg_t *cfg, const ebrl_actgen
  *              planes live in scratch of the handle that grows to the largest batch seen
  *              (n_layers * 2 * sum(P_i) * d elements per batch in flight; EBRL_ERR_NOMEM when
  *              the device cannot hold it).
+ *              Every value in an environment's planes must be finite.  The tensor-core attention
+ *              reads keys and values in blocks of 16 rows; in the last block of a plane the rows
+ *              past P_i are the first rows of what follows it INSIDE THE SAME ENVIRONMENT'S
+ *              BUFFER (the V plane after K, the next layer's K plane after V when kv_layers > 1;
+ *              past the end of the buffer the copy engine supplies zeros, never a neighbour's
+ *              memory).  Their scores are masked and their values get weight exactly 0, which
+ *              keeps any finite number out of the result -- but 0 x Inf or 0 x NaN is NaN.  So an
+ *              Inf or NaN in layer l+1's keys can reach layer l's result of the same environment
+ *              (whose layer l+1 would be spoiled by it anyway); no other environment is affected.
  *   noise      DEVICE [n][H][A] fp32: env i's action state at its step index (the initial
  *              noise when that is 0).
  *   out        DEVICE [n][H][A] fp32; may equal noise.

@@ -283,10 +283,6 @@ __global__ void __launch_bounds__(THREADS, 1) attn_mma_kernel(AttnArgs a, int hp
 #pragma unroll
                 for (int i = 0; i < NPRE; ++i) ldsm_x4_t(vaddr(2 * i), vf[i][0], vf[i][1], vf[i][2], vf[i][3]);
                 float v[8] = {s0[0], s0[1], s0[2], s0[3], s1[0], s1[1], s1[2], s1[3]};
-                // Rows of the last block past the prefix hold whatever follows the plane in memory.  Their scores
-                // are masked, and their VALUE rows are cleared too: a weight of exactly 0 would still turn an Inf or
-                // NaN found there into NaN.  (b0/b2 of a fragment hold keys 2t, 2t+1; b1/b3 keys 2t+8, 2t+9.)
-                uint32_t vm0 = 0xffffffffu, vm1 = 0xffffffffu;
                 if (b == nblk - 1) {
                     const int kleft = P - b * 16;
 #pragma unroll
@@ -294,10 +290,6 @@ __global__ void __launch_bounds__(THREADS, 1) attn_mma_kernel(AttnArgs a, int hp
                         const int key = (e >> 2) * 8 + 2 * t + (e & 1);
                         if (key >= kleft) v[e] = -INFINITY;
                     }
-                    vm0 = (2 * t < kleft ? 0xffffu : 0u) | (2 * t + 1 < kleft ? 0xffff0000u : 0u);
-                    vm1 = (2 * t + 8 < kleft ? 0xffffu : 0u) | (2 * t + 9 < kleft ? 0xffff0000u : 0u);
-#pragma unroll
-                    for (int i = 0; i < NPRE; ++i) { vf[i][0] &= vm0; vf[i][1] &= vm1; vf[i][2] &= vm0; vf[i][3] &= vm1; }
                 }
                 float mx0 = fmaxf(fmaxf(v[0], v[1]), fmaxf(v[4], v[5]));
                 float mx1 = fmaxf(fmaxf(v[2], v[3]), fmaxf(v[6], v[7]));
@@ -330,7 +322,6 @@ __global__ void __launch_bounds__(THREADS, 1) attn_mma_kernel(AttnArgs a, int hp
                 for (int n = 2 * NPRE; n < HD / 8; n += 2) {
                     uint32_t b0, b1, b2, b3;
                     ldsm_x4_t(vaddr(n), b0, b1, b2, b3);
-                    b0 &= vm0; b1 &= vm1; b2 &= vm0; b3 &= vm1;
                     mma_bf16(o[n], pf, b0, b1);
                     mma_bf16(o[n + 1], pf, b2, b3);
                 }

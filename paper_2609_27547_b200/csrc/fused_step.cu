@@ -373,7 +373,6 @@ __device__ __noinline__ int attn_item(AttnItem &ai, int lane)
 #pragma unroll
         for (int i = 0; i < NPRE; ++i) ldsm_x4_t(vaddr(2 * i), vf[i][0], vf[i][1], vf[i][2], vf[i][3]);
         float v[8] = {s0[0], s0[1], s0[2], s0[3], s1[0], s1[1], s1[2], s1[3]};
-        uint32_t vm0 = 0xffffffffu, vm1 = 0xffffffffu;   // value rows of keys past the prefix are cleared, not just weighted by 0
         if (b == nblk - 1) {
             const int kleft = P - b * 16;
 #pragma unroll
@@ -381,10 +380,6 @@ __device__ __noinline__ int attn_item(AttnItem &ai, int lane)
                 const int key = (e >> 2) * 8 + 2 * tq + (e & 1);
                 if (key >= kleft) v[e] = -INFINITY;
             }
-            vm0 = (2 * tq < kleft ? 0xffffu : 0u) | (2 * tq + 1 < kleft ? 0xffff0000u : 0u);
-            vm1 = (2 * tq + 8 < kleft ? 0xffffu : 0u) | (2 * tq + 9 < kleft ? 0xffff0000u : 0u);
-#pragma unroll
-            for (int i = 0; i < NPRE; ++i) { vf[i][0] &= vm0; vf[i][1] &= vm1; vf[i][2] &= vm0; vf[i][3] &= vm1; }
         }
         float mx0 = fmaxf(fmaxf(v[0], v[1]), fmaxf(v[4], v[5]));
         float mx1 = fmaxf(fmaxf(v[2], v[3]), fmaxf(v[6], v[7]));
@@ -416,7 +411,6 @@ __device__ __noinline__ int attn_item(AttnItem &ai, int lane)
         for (int n = 2 * NPRE; n < HD / 8; n += 2) {
             uint32_t b0, b1, b2, b3;
             ldsm_x4_t(vaddr(n), b0, b1, b2, b3);
-            b0 &= vm0; b1 &= vm1; b2 &= vm0; b3 &= vm1;
             mma_bf16(oacc[n], pf, b0, b1);
             mma_bf16(oacc[n + 1], pf, b2, b3);
         }
