@@ -1331,14 +1331,7 @@ ebrl_status_t ebrl_actgen_partition_info(ebrl_actgen_t h, int32_t sm_quota, int3
 }
 
 #ifdef EBRL_FUSED_PROF
-// tuning builds only: the persistent kernel's cycle accounting of the last launch
-ebrl_status_t ebrl_actgen_debug_prof(ebrl_actgen_t h, long long *out, int32_t n)
-{
-    if (!h || !out || !h->trace_slot) return EBRL_ERR_INVALID_ARG;
-    const Slot &ts = *h->trace_slot;
-    const int *base = ts.fctl_d + (size_t)h->cfg.K_steps * (1 + ts.mt_max) + 4 * 256;
-    return cudaMemcpy(out, base, sizeof(long long) * (size_t)n, cudaMemcpyDeviceToHost) == cudaSuccess ? EBRL_OK : EBRL_ERR_CUDA;
-}
+// tuning builds only: the persistent kernel's event log of the last launch (read by fused_timeline.py)
 ebrl_status_t ebrl_actgen_debug_events(ebrl_actgen_t h, long long *out, int32_t n_events, int32_t *count)
 {
     if (!h || !out || !h->trace_slot) return EBRL_ERR_INVALID_ARG;
