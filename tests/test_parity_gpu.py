@@ -317,6 +317,14 @@ def test_sm_partition_gives_the_same_bits(dtype):
         assert st["granted_sms"] == q
         if st["green_ctx_active"]:
             assert q <= st["green_ctx_sms"] <= 148
+            # the complementary partition: the other SMs, with a stream a co-runner can be fenced into
+            gen_sms, rest_sms, rest_stream = r.gen.partition_info(q)
+            assert gen_sms == st["green_ctx_sms"] and gen_sms + rest_sms == 148 and rest_stream
+            buf = torch.zeros(1 << 20, device="cuda")
+            B.sim_corunner_launch(buf, 2, rest_sms, r.gen.rest_stream(q))      # runs there beside nothing: just must work
+            r.gen.rest_stream(q).synchronize()
+            assert torch.allclose(buf, torch.full_like(buf, 0.001 * 0.999 + 0.001))
+    assert r.gen.partition_info(148) == (0, 0, None)  # the whole chip needs no partition
     got = stack(r.run([ids], quota=0), ids)          # full chip: no partition needed
     assert np.array_equal(got, base) and r.gen.stats()["green_ctx_active"] == 0
     r.close()
