@@ -51,6 +51,9 @@ struct GemmArgs {
     void *xg;              // [M][N] (T)
     float *ssq_out;        // [M][N/SSQ_W]
     int test_drop_copies;  // tests of the give-up path: the copy-issuing thread issues nothing, every consumer's bounded wait runs out
+    // fp32 models on the tensor cores: outputs that are the next projection's A operand (xg of the residual epilogue, C of
+    // the GELU epilogue) are written as three bf16 term planes instead of one fp32 array; xg / C then name plane 0
+    void *out_t1, *out_t2;
 };
 
 struct AttnArgs {
@@ -75,6 +78,8 @@ struct AttnArgs {
     const TensorMap128 *kv_maps;   // [n_envs]: the environment's planes as [kv_layers*2*P][d]
     const TensorMap128 *self_map;  // the QKV buffer as [rows][3d]
     int test_drop_copies;          // tests of the give-up path (see GemmArgs)
+    void *out_t1, *out_t2;         // fp32 models on the tensor cores: out, out_t1, out_t2 = the three bf16 term planes of the result
+    int split_out;
 };
 
 struct EmbedArgs {
@@ -87,6 +92,8 @@ struct EmbedArgs {
     float *x;                      // [rows][d]
     void *xg;                      // [rows][d] (T)
     float *ssq;                    // [rows][d/SSQ_W]
+    void *xg_t1, *xg_t2;           // fp32 models on the tensor cores: xg, xg_t1, xg_t2 = the three bf16 term planes of x * gain
+    int split_xg;
 };
 
 struct HeadArgs {

@@ -68,8 +68,9 @@ struct Slot {
     void *xg = nullptr, *qkv = nullptr, *att = nullptr, *qc = nullptr, *u = nullptr;
     EnvMeta *meta_d = nullptr, *meta_h = nullptr;
     TensorMap128 t_xg, t_att, t_u;                    // TMA descriptors of the A operands
-    void *aspl[3] = {nullptr, nullptr, nullptr};      // fp32 models on the tensor cores: the three bf16 terms of the GEMM's A operand
-    TensorMap128 t_aspl_d[3], t_aspl_md[3];           // ... seen as [rows][d] and as [rows][md]
+    // fp32 models on the tensor cores: the projections' A operands as three bf16 term planes each, written by their producers
+    void *xg3[3] = {}, *att3[3] = {}, *u3[3] = {};
+    TensorMap128 t_xg3[3], t_att3[3], t_u3[3];
     FusedMaps *fmaps_d = nullptr;                     // persistent step kernel: the same plus the epilogues' store targets, in device memory
     int *fctl_d = nullptr, *fctl_h = nullptr;         // its control block: n_active[K] then the completion counters [K][mt_max]
     int mt_max = 0;
@@ -590,6 +591,7 @@ cudaError_t enqueue_batch(ebrl_actgen *h, Slot &s, int S, const int32_t *n_activ
         if (!pull) {
             EmbedArgs ea{s.meta_d, ne, H, c.A, d, step, s.a_state, W.w_in, h->temb,
                          L > 0 ? W.layers[0].g1 : W.g_final, s.x, s.xg, s.ssq};
+            if (h->use_tc3) { ea.xg = s.xg3[0]; ea.xg_t1 = s.xg3[1]; ea.xg_t2 = s.xg3[2]; ea.split_xg = 1; }
             ln.run(EBRL_KC_EMBED, 2.0 * M * d * c.A, (double)M * d * (4 + esz), [&] { return launch_embed(ea, bf, grid, st); });
             for (int l = 0; l < L; ++l) {
                 const LayerDev &w = W.layers[l];
@@ -602,9 +604,12 @@ cudaError_t enqueue_batch(ebrl_actgen *h, Slot &s, int S, const int32_t *n_activ
                     g.test_drop_copies = (c.flags & EBRL_FLAG_TEST_DROP_GEMM_COPIES) ? 1 : 0;
                     const double bytes = ((double)M * K + (double)N * K + (double)M * N) * esz + (epi == EPI_RESID ? 8.0 * M * N : 0.0);
                     if (h->use_tc3) {
-                        // split the fp32 activations into their three bf16 terms, then six tensor-core products per k-slice
-                        ln.run(EBRL_KC_GEMM, 0.0, 10.0 * M * K, [&] { return launch_split3((const float *)A, s.aspl[0], s.aspl[1], s.aspl[2], (size_t)M * K, grid, st); });
-                        ln.run(EBRL_KC_GEMM, 2.0 * M * N * K, bytes, [&] { return launch_gemm_tc3(K == d ? s.t_aspl_d : s.t_aspl_md, w3, g, grid, h->wait_ns, h->status_d, st); });
+                        // the A operand exists as three bf16 term planes (its producer wrote them); the residual epilogue's xg and
+                        // the GELU epilogue's C go out as term planes in turn; six tensor-core products per k-slice
+                        const TensorMap128 *ta3 = A == s.xg ? s.t_xg3 : (A == s.att ? s.t_att3 : s.t_u3);
+                        if (epi == EPI_RESID) { g.xg = s.xg3[0]; g.out_t1 = s.xg3[1]; g.out_t2 = s.xg3[2]; }
+                        if (epi == EPI_SCALE_GELU) { g.C = s.u3[0]; g.out_t1 = s.u3[1]; g.out_t2 = s.u3[2]; }
+                        ln.run(EBRL_KC_GEMM, 2.0 * M * N * K, bytes, [&] { return launch_gemm_tc3(ta3, w3, g, grid, h->wait_ns, h->status_d, st); });
                     } else if (h->use_tc) {
                         const int shape = pick_tile_shape(h, M, N, grid);
                         if (shape == 2)
@@ -627,6 +632,7 @@ cudaError_t enqueue_batch(ebrl_actgen *h, Slot &s, int S, const int32_t *n_activ
                     a.v_self = (const char *)s.qkv + (size_t)2 * d * h->esz;
                     a.kv_stride = 3 * d;
                     a.self_map = s.maps_d; a.kv_maps = s.maps_d + 1;
+                    if (h->use_tc3) { a.out = s.att3[0]; a.out_t1 = s.att3[1]; a.out_t2 = s.att3[2]; a.split_out = 1; }
                     ln.run(EBRL_KC_SELF_ATTN, 4.0 * M * H * d, 4.0 * M * d * esz, [&] { return launch_attn(h, a, grid, st); });
                 }
                 gemm(s.att, s.t_att, w.w_o, w.t_o, d, d, EPI_RESID, nullptr, w.g2, w.t3[1]);
@@ -640,6 +646,7 @@ cudaError_t enqueue_batch(ebrl_actgen *h, Slot &s, int S, const int32_t *n_activ
                     a.test_drop_copies = (c.flags & EBRL_FLAG_TEST_DROP_ATTN_COPIES) ? 1 : 0;
                     a.plane_rows = c.d_ctx > 0 ? s.prefix_rows : 0;
                     a.self_map = s.maps_d; a.kv_maps = s.maps_d + 1;
+                    if (h->use_tc3) { a.out = s.att3[0]; a.out_t1 = s.att3[1]; a.out_t2 = s.att3[2]; a.split_out = 1; }
                     ln.run(EBRL_KC_CROSS_ATTN, 4.0 * H * sum_P_active[step] * d,
                            2.0 * sum_P_active[step] * d * esz + 2.0 * M * d * esz, [&] { return launch_attn(h, a, grid, st); });
                 }
@@ -1122,11 +1129,16 @@ ebrl_status_t ebrl_actgen_create(const ebrl_actgen_cfg_t *cfg, const ebrl_actgen
         }
         if (h->use_tc3) {
             for (int t = 0; t < 3; ++t) {
-                if ((st = dev_alloc(h, &s.aspl[t], rows * md * 2, "a split-operand workspace")) != EBRL_OK) return bail(st);
-                if (cudaMemset(s.aspl[t], 0, rows * md * 2) != cudaSuccess) { fail(h, EBRL_ERR_CUDA, "cudaMemset of the workspace failed"); return bail(EBRL_ERR_CUDA); }
-                if (make_tmap_bf16(&s.t_aspl_d[t], s.aspl[t], d, rows, 128) | make_tmap_bf16(&s.t_aspl_md[t], s.aspl[t], md, rows, 128)) {
-                    fail(h, EBRL_ERR_CUDA, "cuTensorMapEncodeTiled failed for a workspace");
-                    return bail(EBRL_ERR_CUDA);
+                void **bufs[3] = {&s.xg3[t], &s.att3[t], &s.u3[t]};
+                TensorMap128 *maps[3] = {&s.t_xg3[t], &s.t_att3[t], &s.t_u3[t]};
+                const size_t width[3] = {(size_t)d, (size_t)d, (size_t)md};
+                for (int b = 0; b < 3; ++b) {
+                    if ((st = dev_alloc(h, bufs[b], rows * width[b] * 2, "a split-operand workspace")) != EBRL_OK) return bail(st);
+                    if (cudaMemset(*bufs[b], 0, rows * width[b] * 2) != cudaSuccess) { fail(h, EBRL_ERR_CUDA, "cudaMemset of the workspace failed"); return bail(EBRL_ERR_CUDA); }
+                    if (make_tmap_bf16(maps[b], *bufs[b], width[b], rows, 128)) {
+                        fail(h, EBRL_ERR_CUDA, "cuTensorMapEncodeTiled failed for a workspace");
+                        return bail(EBRL_ERR_CUDA);
+                    }
                 }
             }
         }

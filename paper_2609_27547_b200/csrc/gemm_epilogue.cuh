@@ -2,6 +2,7 @@
 // row of the tile and walks its accumulator columns 32 at a time out of tensor memory.
 #pragma once
 #include "actgen_internal.h"
+#include "split3.cuh"
 
 #include <cuda.h>
 
@@ -137,7 +138,9 @@ template <> __device__ __forceinline__ void store_out4<float>(float *p, float a,
     *reinterpret_cast<float4 *>(p) = make_float4(a, b, c, d);
 }
 
-template <int EPI, int NCOLS, bool COH = false, typename OT = __nv_bfloat16, typename WaitF>
+// SPLIT (fp32 models on the tensor cores): what feeds the next projection -- xg of the residual epilogue, C of the
+// GELU epilogue -- is written as three bf16 term planes; the scale/store epilogue's C (queries, keys, values) stays fp32.
+template <int EPI, int NCOLS, bool COH = false, typename OT = __nv_bfloat16, bool SPLIT = false, typename WaitF>
 __device__ __forceinline__ bool epilogue_rows(const GemmArgs &g, uint32_t taddr, int row0, int n0, float *stg_generic, WaitF wait)
 {
     constexpr int NC = NCOLS / 32;
@@ -205,7 +208,8 @@ __device__ __forceinline__ bool epilogue_rows(const GemmArgs &g, uint32_t taddr,
                     float4 xn;
                     xn.x = xv[i].x + acc[i].x; xn.y = xv[i].y + acc[i].y; xn.z = xv[i].z + acc[i].z; xn.w = xv[i].w + acc[i].w;
                     *reinterpret_cast<float4 *>(xg_x + off) = xn;
-                    store_out4<OT>(xg + off, xn.x * gn.x, xn.y * gn.y, xn.z * gn.z, xn.w * gn.w);
+                    if (SPLIT) store_split4(g.xg, g.out_t1, g.out_t2, off, xn.x * gn.x, xn.y * gn.y, xn.z * gn.z, xn.w * gn.w);
+                    else store_out4<OT>(xg + off, xn.x * gn.x, xn.y * gn.y, xn.z * gn.z, xn.w * gn.w);
                     ssp[i] = fmaf(xn.x, xn.x, ssp[i]); ssp[i] = fmaf(xn.y, xn.y, ssp[i]);
                     ssp[i] = fmaf(xn.z, xn.z, ssp[i]); ssp[i] = fmaf(xn.w, xn.w, ssp[i]);
                 }
@@ -220,7 +224,11 @@ __device__ __forceinline__ bool epilogue_rows(const GemmArgs &g, uint32_t taddr,
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const int rr = 4 * i + sub;
-                if (rr < nrows) store_out4<OT>(cp + (size_t)(row0 + rr) * g.N + col + 4 * piece, acc[i].x, acc[i].y, acc[i].z, acc[i].w);
+                if (rr < nrows) {
+                    const size_t off = (size_t)(row0 + rr) * g.N + col + 4 * piece;
+                    if (SPLIT && EPI == EPI_SCALE_GELU) store_split4(g.C, g.out_t1, g.out_t2, off, acc[i].x, acc[i].y, acc[i].z, acc[i].w);
+                    else store_out4<OT>(cp + off, acc[i].x, acc[i].y, acc[i].z, acc[i].w);
+                }
             }
         }
     }

@@ -9,8 +9,9 @@
 // leave the FFMA pipe (2 x 128 FLOP per clock per SM) for the tensor pipe (six products still run
 // several times faster).
 //
-// Weights are split once, when they are copied into the handle; activations are split by
-// split3_kernel right before the GEMM that reads them.  The GEMM is the single-CTA 128 x 128
+// Weights are split once (split3_kernel), when they are copied into the handle; activations are
+// written as their three term planes by whatever produces them (the embedding, the residual and
+// GELU epilogues below, the attention kernel).  The GEMM is the single-CTA 128 x 128
 // tensor-core kernel with six operand tiles per 64-wide k-block (96 KB per stage, two stages) and
 // the same fused epilogues on fp32 outputs.  With K of a few hundred the epilogue of a tile takes
 // longer than its mainloop, so two groups of four epilogue warps drain the two accumulators in
@@ -184,7 +185,7 @@ gemm_tc3_kernel(const __grid_constant__ Maps6 tm, GemmArgs g, unsigned long long
             const int m0 = (tile / ntn) * BM, n0 = (tile % ntn) * BN;
             auto acc_ready = [&] { return __all_sync(0xffffffffu, mbar_wait_relaxed(tfull(buf), acc_phase, limit_ns, abort_flag)) != 0; };
             const uint32_t tacc = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN);
-            if (!epilogue_rows<EPI, 128, false, float>(g, tacc, m0 + q * 32, n0, stg, acc_ready)) { ok = false; break; }
+            if (!epilogue_rows<EPI, 128, false, float, true>(g, tacc, m0 + q * 32, n0, stg, acc_ready)) { ok = false; break; }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty(buf));
@@ -221,13 +222,7 @@ __global__ void __launch_bounds__(512) split3_kernel(const float4 *__restrict__ 
         const float a[4] = {v.x, v.y, v.z, v.w};
         __nv_bfloat16 t0[4], t1[4], t2[4];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            t0[e] = __float2bfloat16_rn(a[e]);
-            const float r1 = a[e] - __bfloat162float(t0[e]);      // exact
-            t1[e] = __float2bfloat16_rn(r1);
-            const float r2 = r1 - __bfloat162float(t1[e]);        // exact
-            t2[e] = __float2bfloat16_rn(r2);
-        }
+        for (int e = 0; e < 4; ++e) split3(a[e], t0[e], t1[e], t2[e]);
         p0[i] = *reinterpret_cast<const uint2 *>(t0);
         p1[i] = *reinterpret_cast<const uint2 *>(t1);
         p2[i] = *reinterpret_cast<const uint2 *>(t2);

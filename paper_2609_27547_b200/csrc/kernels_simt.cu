@@ -7,6 +7,7 @@
 // grid size or on which other rows share a tile.
 #include "actgen_internal.h"
 #include "rowops.cuh"
+#include "split3.cuh"
 
 namespace ebrl {
 
@@ -350,7 +351,17 @@ __global__ void __launch_bounds__(GROUPS * 128) attn_simt_kernel(AttnArgs a)
 #pragma unroll
         for (int r = 0; r < RMAX; ++r) {
             const int i = rg + ncg * r;
-            if (i < H) stf(og + (size_t)i * a.o_stride, acc[r] / lsum[i]);
+            if (i < H) {
+                const float val = acc[r] / lsum[i];
+                if (a.split_out) {   // the three bf16 terms of the result, for the tensor-core projection that follows
+                    const size_t off = (size_t)env * H * a.o_stride + h * hd + c + (size_t)i * a.o_stride;
+                    __nv_bfloat16 t0, t1, t2;
+                    split3(val, t0, t1, t2);
+                    ((__nv_bfloat16 *)a.out)[off] = t0; ((__nv_bfloat16 *)a.out_t1)[off] = t1; ((__nv_bfloat16 *)a.out_t2)[off] = t2;
+                } else {
+                    stf(og + (size_t)i * a.o_stride, val);
+                }
+            }
         }
         group_sync(grp);   // lsum, q are reused by the next item
     }

@@ -4,6 +4,7 @@
 // same bits: a row's result is one fixed sequence of operations whoever calls it.
 #pragma once
 #include "actgen_internal.h"
+#include "split3.cuh"
 
 namespace ebrl {
 
@@ -88,7 +89,8 @@ __device__ __forceinline__ void embed_row_pair(const EmbedArgs &a, int row0, int
                 const float4 te = *reinterpret_cast<const float4 *>(a.temb + (size_t)kk[r] * a.d + c);
                 const float v0 = acc[r][0] + te.x, v1 = acc[r][1] + te.y, v2 = acc[r][2] + te.z, v3 = acc[r][3] + te.w;
                 *reinterpret_cast<float4 *>(a.x + (size_t)row * a.d + c) = make_float4(v0, v1, v2, v3);
-                store4<T>(xg + (size_t)row * a.d + c, v0 * gn.x, v1 * gn.y, v2 * gn.z, v3 * gn.w);
+                if (a.split_xg) store_split4(a.xg, a.xg_t1, a.xg_t2, (size_t)row * a.d + c, v0 * gn.x, v1 * gn.y, v2 * gn.z, v3 * gn.w);
+                else store4<T>(xg + (size_t)row * a.d + c, v0 * gn.x, v1 * gn.y, v2 * gn.z, v3 * gn.w);
                 float ss = v0 * v0;
                 ss = fmaf(v1, v1, ss); ss = fmaf(v2, v2, ss); ss = fmaf(v3, v3, ss);
                 ss = warp_sum(ss);
