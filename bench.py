@@ -165,7 +165,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * sum(times) / len(times),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "configs[%d] %s" % (args.config, w.name), "note": "fp64 CPU oracle on host cores; each step is a bounded sample"},
+        "config": {"workload": synth.workload_label(args.config), "note": "fp64 CPU oracle on host cores; each step is a bounded sample"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -301,7 +301,7 @@ def run_stub(args):
     if ctx.rank == 0:
         print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": ctx.world, "steps": args.steps,
                           "warmup": 0, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-                          "data": "stub", "config": {"workload": "configs[%d] %s" % (args.config, w.name), "envs_per_gpu": w.B},
+                          "data": "stub", "config": {"workload": synth.workload_label(args.config), "envs_per_gpu": w.B},
                           "shards": gathered, "gpu_launches": 0}))
     ctx.close()
 
@@ -529,7 +529,7 @@ def run_ours(args, emit=True):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": n_warm,
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16" if bf16 else "f32", "data": "synthetic",
-            "config": {"workload": "configs[%d] %s" % (args.config, w.name), "envs_per_gpu": w.B, "H": w.H, "A": w.A, "d": w.d,
+            "config": {"workload": synth.workload_label(args.config), "envs_per_gpu": w.B, "H": w.H, "A": w.A, "d": w.d,
                        "L": w.L, "heads": w.n_heads, "P": list(w.P), "K": w.K, "d_ctx": w.d_ctx, "groups": len(groups),
                        "group_sizes": [min(map(len, groups)), max(map(len, groups))], "sm_quota": q_eff,
                        "inflight_groups": inflight, "corunner": co_report if co_report is not None else False,
@@ -577,10 +577,15 @@ def run_sweep(args):
         if q < N_SMS:
             plan.append((3, q, True))
     plan += [(4, 148, False), (4, 37, False)]                 # the bench configuration at other quotas than its own 74
+    plan.append((12, -1, False))                              # configurations 2 and 3 on the configs[1] model
+    for q in (148, 74, 37, 16):
+        plan.append((13, q, False))
+        if q < N_SMS:
+            plan.append((13, q, True))
     for cfg_i, q, co in plan:
         a = copy.copy(args)
         a.config, a.corunner, a.no_cpu, a.no_e2e, a.quota = cfg_i, co, True, True, q
-        a.steps = {1: 10, 4: 3}.get(cfg_i, max(args.steps, 20))
+        a.steps = {1: 10, 4: 3, 12: 10, 13: 5}.get(cfg_i, max(args.steps, 20))
         run_ours(a)
 
 
@@ -621,7 +626,7 @@ def run_pgen_sweep(args):
             row.append(b * args.steps / (e0.elapsed_time(e1) * 1e-3))
         rate.append(row)
     gen.destroy()
-    print(json.dumps({"pgen": {"workload": "configs[%d] %s" % (args.config, w.name), "unit": UNIT, "quota_pct": quotas,
+    print(json.dumps({"pgen": {"workload": synth.workload_label(args.config), "unit": UNIT, "quota_pct": quotas,
                                "kernels": "persistent step kernel" if args.fused else "one kernel per operation",
                                "quota_sms": [max(1, round(N_SMS * q / 100)) for q in quotas], "batch": batches, "rate": rate}}))
 
@@ -647,7 +652,7 @@ def main():
         quota = w.quota if args.quota < 0 else args.quota
         out = [R.run(w, wt, n, max(1, args.steps), pol, quota=quota, max_group=64, sim_steps_per_chunk=w.H).summary()
                for pol in ("chunk", "step")]
-        print(json.dumps({"rollout_sim": {"workload": "configs[%d] %s" % (args.config, w.name), "envs": n, "chunks_per_env": max(1, args.steps),
+        print(json.dumps({"rollout_sim": {"workload": synth.workload_label(args.config), "envs": n, "chunks_per_env": max(1, args.steps),
                                           "sm_quota": quota or N_SMS, "simulator": "log-normal step time, mean 40 ms, P99 60 ms, H steps per chunk",
                                           "policies": out}}))
         return

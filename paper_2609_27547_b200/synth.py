@@ -136,7 +136,19 @@ WORKLOADS: Dict[int, Workload] = {
                 mixed_steps=True),
     3: Workload("cfg3_quota_sweep_f32", "f32", 1024, 8, 7, 256, 2, 4, 4, (256, 256), None, 0),
     4: Workload("cfg4_large_bf16", "bf16", 2048, 16, 14, 2048, 8, 16, 10, (768, 768), (32, 256), 74),
+    # The other reading of "the config-1 model" in configurations 2 and 3 (counting from zero: the
+    # bf16 mid-size head of WORKLOADS[1] instead of the tiny fp32 one); same arrivals and quotas.
+    12: Workload("cfg2_ragged_mid_bf16", "bf16", 512, 8, 7, 1024, 4, 16, 10, (64, 512), (1, 64), 0,
+                 mixed_steps=True),
+    13: Workload("cfg3_quota_sweep_mid_bf16", "bf16", 1024, 8, 7, 1024, 4, 16, 10, (256, 256), None, 0),
 }
+
+
+def workload_label(i: int) -> str:
+    """The name a result line carries: ``configs[i] <name>`` (12 and 13 are configurations 2 and 3 on
+    the WORKLOADS[1] model)."""
+    w = WORKLOADS[i]
+    return "configs[%d] %s" % (i - 10, w.name) if i >= 10 else "configs[%d] %s" % (i, w.name)
 
 
 def scaled(w: Workload, **kw) -> Workload:

@@ -102,6 +102,41 @@ def test_configs3_quota_sweep_bit_identity():
     assert chunk_rel_err(np.stack([base[e].cpu().numpy() for e in sample]), ref) <= TOL["f32"]
 
 
+def test_configs2_and_3_on_the_mid_size_bf16_model():
+    """The other reading of "the config-1 model" (the bf16 mid-size head of configs[1]): the ragged
+    arrivals of configs[2] against the oracle and alone, the quota sweep of configs[3] bit-identical."""
+    w = synth.WORKLOADS[12]
+    wt = synth.make_weights(w, SEED, device="cuda")
+    envs = {e: synth.make_env(w, e, SEED, device="cuda") for e in range(w.B)}
+    groups = synth.arrival_groups(w, SEED)
+    gen, out, pos = _run_full(w, wt, envs, groups, 0, inflight=4)
+    sample = [groups[0][0], groups[3][0], groups[-1][-1], 100, 101, 102]
+    ref = _oracle(w, wt, envs, sample)
+    got = np.stack([out[pos[e]].cpu().numpy() for e in sample])
+    assert chunk_rel_err(got, ref) <= TOL["bf16"]
+    for e in sample[:3]:
+        assert torch.equal(_alone(gen, w, envs, e, 16), out[pos[e]])
+    gen.destroy()
+    del envs
+    w = synth.WORKLOADS[13]
+    envs = {e: synth.make_env(w, e, SEED, device="cuda") for e in range(w.B)}
+    ids = list(range(w.B))
+    base = None
+    for q in (148, 74, 37, 16):
+        gen, out, pos = _run_full(w, wt, envs, [ids], q)
+        gen.destroy()
+        if base is None:
+            base = out.clone()
+        else:
+            assert torch.equal(out, base), "quota %d" % q
+    gen, out, pos = _run_full(w, wt, envs, [ids[i:i + 128] for i in range(0, w.B, 128)], 74)
+    gen.destroy()
+    assert torch.equal(out, base)
+    sample = [0, 1023]
+    ref = _oracle(w, wt, envs, sample)
+    assert chunk_rel_err(np.stack([base[e].cpu().numpy() for e in sample]), ref) <= TOL["bf16"]
+
+
 def test_configs4_full_size_sampled():
     """configs[4]: 2048 envs, ragged groups of 32..256 at the 74-SM quota, queue depth 16 (the bench's
     launch configuration: the whole step is one packed batch of 32768 rows); also at depth 8 (two batches).
