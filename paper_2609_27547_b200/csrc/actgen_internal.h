@@ -234,5 +234,8 @@ cudaError_t launch_embed(const EmbedArgs &a, int bf16, int grid, cudaStream_t st
 cudaError_t launch_head(const HeadArgs &a, int bf16, int grid, cudaStream_t st);
 cudaError_t launch_gemm_simt(const GemmArgs &a, int bf16, int grid, cudaStream_t st);
 cudaError_t launch_attn_simt(const AttnArgs &a, int bf16, int grid, cudaStream_t st);
+// fp32 models, head_dim 64, H <= 8: one warp per (environment, head), operands in registers (attn_f32.cu)
+bool attn_f32_supported(int H, int hd);
+cudaError_t launch_attn_f32(const AttnArgs &a, int grid, cudaStream_t st);
 
 }  // namespace ebrl

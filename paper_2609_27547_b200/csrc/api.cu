@@ -121,6 +121,7 @@ struct ebrl_actgen {
     bool pdl_allowed = true;      // EBRL_PDL=0 turns programmatic dependent launch off
     int attn_lookahead = 2;       // EBRL_ATTN_LOOKAHEAD: key blocks the attention producer asks L2 for ahead of its ring
     bool use_attn_mma = false;    // tensor-core attention (bf16, H <= 16, head_dim 64/128)
+    bool use_attn_f32 = false;    // warp-per-item fp32 attention (head_dim 64, H <= 8)
     int *status_d = nullptr;      // device status word written by kernels whose waits ran out
     unsigned long long wait_ns = 0;
     size_t esz = 4;   // bytes per element of matrices / activations / planes
@@ -495,6 +496,7 @@ struct Launcher {
 cudaError_t launch_attn(ebrl_actgen *h, const AttnArgs &a, int grid, cudaStream_t st)
 {
     if (h->use_attn_mma) return launch_attn_mma(a, grid, h->attn_lookahead, h->wait_ns, h->status_d, st);
+    if (h->use_attn_f32) return launch_attn_f32(a, grid, st);
     return launch_attn_simt(a, h->bf16, grid, st);
 }
 
@@ -1043,6 +1045,7 @@ ebrl_status_t ebrl_actgen_create(const ebrl_actgen_cfg_t *cfg, const ebrl_actgen
     if (const char *e4 = getenv("EBRL_PDL")) h->pdl_allowed = atoi(e4) != 0;
     if (const char *e5 = getenv("EBRL_ATTN_LOOKAHEAD")) h->attn_lookahead = std::min(64, std::max(0, atoi(e5)));
     h->use_attn_mma = h->bf16 && !(cfg->flags & EBRL_FLAG_FORCE_SIMT) && attn_mma_supported(cfg->H, cfg->n_heads, h->hd);
+    h->use_attn_f32 = !h->bf16 && !(cfg->flags & EBRL_FLAG_FORCE_SIMT) && attn_f32_supported(cfg->H, h->hd);
     h->use_tc3 = !h->bf16 && !(cfg->flags & EBRL_FLAG_FORCE_SIMT) && gemm_tc3_supported(d, d) && gemm_tc3_supported(md, d) &&
                  gemm_tc3_supported(d, md) && gemm_tc3_supported(3 * d, d);
     h->fused_ok = h->use_tc && h->use_attn_mma && fused_supported(cfg->H, cfg->A, d, md, cfg->n_heads, h->hd);

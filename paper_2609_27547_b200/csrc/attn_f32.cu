@@ -1,0 +1,260 @@
+// Softmax attention for the fp32 models (head_dim 64, up to 8 query tokens): one WARP per
+// (environment, head) item, no shared state between warps and no block-wide barrier.
+//
+// The contraction is tiny -- 8 query rows against P keys of 64 columns -- so what decides the
+// speed is how many operand fetches an FMA costs.  Here the query block lives in registers for
+// the whole item and every key / value element fetched from shared memory feeds 8 FMAs:
+//
+//   lane = (key slot k4 = lane / 8, column group cq = lane % 8); a lane owns the 8 columns
+//   4 cq .. 4 cq + 3 and 32 + 4 cq .. 32 + 4 cq + 3 of every row it touches;
+//   q[8 rows][8 columns]   registers, scaled by 1 / sqrt(head_dim), loaded once per item
+//   o[8 rows][8 columns]   registers, this lane's share of the output over ITS keys
+//   scores: 8 partial dot products per lane and key (64 FMAs on two 16-byte reads of the key),
+//   folded across the 8 column groups by a halving exchange (7 shuffles) that leaves the score
+//   of row rho(cq) with lane cq; values: the 8 weights of the key are gathered back (8
+//   shuffles) for 64 FMAs on two 16-byte reads.
+//
+// Keys and values stream through a per-warp ring of 16-key stages filled by cp.async (zero fill
+// past the prefix), so a warp's global-memory latency hides behind its own arithmetic and the
+// eight warps of a CTA never wait on one another.  Keys are visited in blocks of 16 in index
+// order with a running maximum and sum; an item's arithmetic involves nothing but the item, so
+// the result does not depend on the grid size or on what else is in the batch.
+#include "actgen_internal.h"
+#include "split3.cuh"
+
+#include <cuda_runtime.h>
+#include <math.h>
+
+namespace ebrl {
+namespace af {
+
+constexpr int HD = 64;            // head_dim
+constexpr int ROWS = 8;           // query rows held per item
+constexpr int WARPS = 8;          // items in flight per CTA
+constexpr int SK = 16;            // keys per stage
+constexpr int NST = 3;            // stages per warp
+constexpr int PLANE_FLOATS = SK * HD;
+constexpr int STAGE_FLOATS = 2 * PLANE_FLOATS;                 // keys, then values
+constexpr int SMEM_BYTES = WARPS * NST * STAGE_FLOATS * 4;     // 192 KB
+constexpr unsigned FULL = 0xffffffffu;
+
+__device__ __forceinline__ void cp16(uint32_t dst, const void *src, uint32_t nbytes)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(nbytes) : "memory");
+}
+__device__ __forceinline__ void cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// Sum of v[r] over the 8 lanes that differ in lane bits 0..2, for all 8 r at once: each exchange halves the
+// number of rows a lane still carries (4 + 2 + 1 shuffles).  On return the lane holds the total of row
+// rho(lane % 8) = 4 bit0 + 2 bit1 + bit2 (the bit reversal of its column group).
+__device__ __forceinline__ float fold8(const float (&v)[8], int lane)
+{
+    const bool b0 = lane & 1, b1 = lane & 2, b2 = lane & 4;
+    float w[4], x[2];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float send = b0 ? v[i] : v[i + 4], keep = b0 ? v[i + 4] : v[i];
+        w[i] = keep + __shfl_xor_sync(FULL, send, 1);
+    }
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const float send = b1 ? w[i] : w[i + 2], keep = b1 ? w[i + 2] : w[i];
+        x[i] = keep + __shfl_xor_sync(FULL, send, 2);
+    }
+    const float send = b2 ? x[0] : x[1], keep = b2 ? x[1] : x[0];
+    return keep + __shfl_xor_sync(FULL, send, 4);
+}
+// rho is its own inverse: the column group whose lane holds row r
+__device__ __forceinline__ int rho(int r) { return ((r >> 2) & 1) | (r & 2) | ((r & 1) << 2); }
+
+__global__ void __launch_bounds__(WARPS * 32, 1) attn_f32_kernel(AttnArgs a)
+{
+    extern __shared__ __align__(16) float smem[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int k4 = lane >> 3, cq = lane & 7, kgrp = lane & 24;
+    float *ring = smem + (size_t)warp * NST * STAGE_FLOATS;
+    const uint32_t ring_u = (uint32_t)__cvta_generic_to_shared(ring);
+    const int H = a.H;
+    const float scale = 1.0f / sqrtf((float)HD);
+    const int items = a.n_envs * a.n_heads;
+    pdl_launch_dependents();
+    pdl_wait();
+    for (int item = blockIdx.x * WARPS + warp; item < items; item += gridDim.x * WARPS) {
+        const int env = item / a.n_heads, h = item - env * a.n_heads;
+        const float *kbase, *vbase;
+        int P, kvs;
+        if (a.self) {
+            kbase = (const float *)a.k_self + (size_t)env * H * a.kv_stride + h * HD;
+            vbase = (const float *)a.v_self + (size_t)env * H * a.kv_stride + h * HD;
+            P = H; kvs = a.kv_stride;
+        } else {
+            const EnvMeta m = a.meta[env];
+            P = m.P; kvs = a.d;
+            const int pr = a.plane_rows ? a.plane_rows : P;
+            kbase = (const float *)m.kv + (size_t)a.kv_plane * 2 * pr * a.d + h * HD;
+            vbase = kbase + (size_t)pr * a.d;
+        }
+        const int nblk = (P + SK - 1) / SK;
+        __syncwarp();   // the previous item's last stage has been read by every lane
+        // stage b of the item: 16 keys x 256 bytes of each plane, 16 bytes per copy, two keys per warp instruction
+        auto issue = [&](int b) {
+            if (b < nblk) {
+                const uint32_t dst = ring_u + (uint32_t)((b % NST) * STAGE_FLOATS * 4);
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int c = lane + 32 * u, key = c >> 4, col = (c & 15) << 2;
+                    const bool in = b * SK + key < P;
+                    const size_t src = (size_t)(in ? b * SK + key : 0) * kvs + col;
+                    cp16(dst + (uint32_t)((key * HD + col) * 4), kbase + src, in ? 16u : 0u);
+                    cp16(dst + (uint32_t)((PLANE_FLOATS + key * HD + col) * 4), vbase + src, in ? 16u : 0u);
+                }
+            }
+            cp_commit();   // one group per call, empty past the last block: the wait below counts groups
+        };
+#pragma unroll
+        for (int b = 0; b < NST - 1; ++b) issue(b);
+
+        float q[ROWS][8];
+        const float *qg = (const float *)a.q + (size_t)env * H * a.q_stride + h * HD;
+#pragma unroll
+        for (int r = 0; r < ROWS; ++r) {
+            float4 lo = make_float4(0.f, 0.f, 0.f, 0.f), hi = lo;
+            if (r < H) {
+                lo = *reinterpret_cast<const float4 *>(qg + (size_t)r * a.q_stride + 4 * cq);
+                hi = *reinterpret_cast<const float4 *>(qg + (size_t)r * a.q_stride + 32 + 4 * cq);
+            }
+            q[r][0] = lo.x * scale; q[r][1] = lo.y * scale; q[r][2] = lo.z * scale; q[r][3] = lo.w * scale;
+            q[r][4] = hi.x * scale; q[r][5] = hi.y * scale; q[r][6] = hi.z * scale; q[r][7] = hi.w * scale;
+        }
+        float o[ROWS][8];
+#pragma unroll
+        for (int r = 0; r < ROWS; ++r)
+#pragma unroll
+            for (int c = 0; c < 8; ++c) o[r][c] = 0.f;
+        float mrun = -INFINITY, lrun = 0.f;   // running maximum and (this lane's keys') sum of row rho(cq)
+
+        for (int b = 0; b < nblk; ++b) {
+            __syncwarp();            // every lane is done with the stage the next copies overwrite
+            issue(b + NST - 1);
+            cp_wait<NST - 1>();      // this lane's copies of stage b have landed ...
+            __syncwarp();            // ... and so have the other lanes'
+            const float *ks = ring + (b % NST) * STAGE_FLOATS, *vs = ks + PLANE_FLOATS;
+            float s[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int key = 4 * j + k4;
+                const float4 klo = *reinterpret_cast<const float4 *>(ks + key * HD + 4 * cq);
+                const float4 khi = *reinterpret_cast<const float4 *>(ks + key * HD + 32 + 4 * cq);
+                float part[ROWS];
+#pragma unroll
+                for (int r = 0; r < ROWS; ++r) {
+                    float t = q[r][0] * klo.x;
+                    t = fmaf(q[r][1], klo.y, t); t = fmaf(q[r][2], klo.z, t); t = fmaf(q[r][3], klo.w, t);
+                    t = fmaf(q[r][4], khi.x, t); t = fmaf(q[r][5], khi.y, t); t = fmaf(q[r][6], khi.z, t); t = fmaf(q[r][7], khi.w, t);
+                    part[r] = t;
+                }
+                const float sc = fold8(part, lane);
+                s[j] = (b * SK + key < P) ? sc : -INFINITY;
+            }
+            // running softmax statistics of row rho(cq): the block's maximum over this lane's four keys and the
+            // four key slots (the block's first key always exists, so the maximum is finite)
+            float bm = fmaxf(fmaxf(s[0], s[1]), fmaxf(s[2], s[3]));
+            bm = fmaxf(bm, __shfl_xor_sync(FULL, bm, 8));
+            bm = fmaxf(bm, __shfl_xor_sync(FULL, bm, 16));
+            const float mnew = fmaxf(mrun, bm);
+            const float al = expf(mrun - mnew);
+            float p[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) p[j] = expf(s[j] - mnew);
+            lrun = lrun * al + ((p[0] + p[1]) + (p[2] + p[3]));
+            mrun = mnew;
+            if (__any_sync(FULL, al != 1.0f)) {   // once the maxima have settled every factor is exactly 1
+#pragma unroll
+                for (int r = 0; r < ROWS; ++r) {
+                    const float ar = __shfl_sync(FULL, al, kgrp | rho(r));
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) o[r][c] *= ar;
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int key = 4 * j + k4;
+                const float4 vlo = *reinterpret_cast<const float4 *>(vs + key * HD + 4 * cq);
+                const float4 vhi = *reinterpret_cast<const float4 *>(vs + key * HD + 32 + 4 * cq);
+#pragma unroll
+                for (int r = 0; r < ROWS; ++r) {
+                    const float pr = __shfl_sync(FULL, p[j], kgrp | rho(r));   // weight of (row r, this lane's key)
+                    o[r][0] = fmaf(pr, vlo.x, o[r][0]); o[r][1] = fmaf(pr, vlo.y, o[r][1]);
+                    o[r][2] = fmaf(pr, vlo.z, o[r][2]); o[r][3] = fmaf(pr, vlo.w, o[r][3]);
+                    o[r][4] = fmaf(pr, vhi.x, o[r][4]); o[r][5] = fmaf(pr, vhi.y, o[r][5]);
+                    o[r][6] = fmaf(pr, vhi.z, o[r][6]); o[r][7] = fmaf(pr, vhi.w, o[r][7]);
+                }
+            }
+        }
+        cp_wait<0>();   // only empty groups are left
+        // totals over the four key slots (lane bits 3 and 4): the row sums everywhere, the outputs by two
+        // halving exchanges that leave rows 4 bit3 + 2 bit4 + {0, 1} with the lane
+        lrun += __shfl_xor_sync(FULL, lrun, 8);
+        lrun += __shfl_xor_sync(FULL, lrun, 16);
+        const bool b3 = lane & 8, b4 = lane & 16;
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const float send = b3 ? o[i][c] : o[i + 4][c], keep = b3 ? o[i + 4][c] : o[i][c];
+                o[i][c] = keep + __shfl_xor_sync(FULL, send, 8);
+            }
+#pragma unroll
+        for (int i = 0; i < 2; ++i)
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const float send = b4 ? o[i][c] : o[i + 2][c], keep = b4 ? o[i + 2][c] : o[i][c];
+                o[i][c] = keep + __shfl_xor_sync(FULL, send, 16);
+            }
+        const int rbase = (b3 ? 4 : 0) + (b4 ? 2 : 0);
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const int r = rbase + i;
+            const float lr = __shfl_sync(FULL, lrun, rho(r));
+            if (r < H) {
+                const size_t off = (size_t)(env * H + r) * a.o_stride + h * HD + 4 * cq;
+                float v[8];
+#pragma unroll
+                for (int c = 0; c < 8; ++c) v[c] = o[i][c] / lr;
+                if (a.split_out) {   // the three bf16 terms of the result, for the tensor-core projection that follows
+                    store_split4(a.out, a.out_t1, a.out_t2, off, v[0], v[1], v[2], v[3]);
+                    store_split4(a.out, a.out_t1, a.out_t2, off + 32, v[4], v[5], v[6], v[7]);
+                } else {
+                    *reinterpret_cast<float4 *>((float *)a.out + off) = make_float4(v[0], v[1], v[2], v[3]);
+                    *reinterpret_cast<float4 *>((float *)a.out + off + 32) = make_float4(v[4], v[5], v[6], v[7]);
+                }
+            }
+        }
+    }
+}
+
+}  // namespace af
+
+// Shapes the warp-per-item kernel covers (fp32 planes and activations).
+bool attn_f32_supported(int H, int hd) { return hd == af::HD && H >= 1 && H <= af::ROWS; }
+
+// grid = SM quota; each CTA keeps eight items in flight.
+cudaError_t launch_attn_f32(const AttnArgs &a, int grid, cudaStream_t st)
+{
+    const int items = a.n_envs * a.n_heads;
+    if (items == 0) return cudaSuccess;
+    static bool attr_set[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    if (!attr_set[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(af::attn_f32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, af::SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        attr_set[dev] = true;
+    }
+    const int need = (items + af::WARPS - 1) / af::WARPS;
+    const int g = need < grid ? need : grid;
+    return launch_kernel(af::attn_f32_kernel, g, af::WARPS * 32, af::SMEM_BYTES, st, 1, a);
+}
+
+}  // namespace ebrl
