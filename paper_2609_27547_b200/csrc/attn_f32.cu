@@ -12,7 +12,8 @@
 //   scores: 8 partial dot products per lane and key (64 FMAs on two 16-byte reads of the key),
 //   folded across the 8 column groups by a halving exchange (7 shuffles) that leaves the score
 //   of row rho(cq) with lane cq; values: the 8 weights of the key are gathered back (8
-//   shuffles) for 64 FMAs on two 16-byte reads.
+//   shuffles) for 64 FMAs on two 16-byte reads.  The FMAs are issued two per instruction
+//   (f32x2 on column pairs): the kernel is bound by issue slots, not by the FMA pipe.
 //
 // Keys and values stream through a per-warp ring of 16-key stages filled by cp.async (zero fill
 // past the prefix), so a warp's global-memory latency hides behind its own arithmetic and the
@@ -21,6 +22,7 @@
 // the result does not depend on the grid size or on what else is in the batch.
 #include "actgen_internal.h"
 #include "split3.cuh"
+#include "f32x2.cuh"
 
 #include <cuda_runtime.h>
 #include <math.h>
@@ -45,34 +47,18 @@ __device__ __forceinline__ void cp16(uint32_t dst, const void *src, uint32_t nby
 __device__ __forceinline__ void cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-// Sum of v[r] over the 8 lanes that differ in lane bits 0..2, for all 8 r at once: each exchange halves the
-// number of rows a lane still carries (4 + 2 + 1 shuffles).  On return the lane holds the total of row
-// rho(lane % 8) = 4 bit0 + 2 bit1 + bit2 (the bit reversal of its column group).
-__device__ __forceinline__ float fold8(const float (&v)[8], int lane)
-{
-    const bool b0 = lane & 1, b1 = lane & 2, b2 = lane & 4;
-    float w[4], x[2];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const float send = b0 ? v[i] : v[i + 4], keep = b0 ? v[i + 4] : v[i];
-        w[i] = keep + __shfl_xor_sync(FULL, send, 1);
-    }
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-        const float send = b1 ? w[i] : w[i + 2], keep = b1 ? w[i + 2] : w[i];
-        x[i] = keep + __shfl_xor_sync(FULL, send, 2);
-    }
-    const float send = b2 ? x[0] : x[1], keep = b2 ? x[1] : x[0];
-    return keep + __shfl_xor_sync(FULL, send, 4);
-}
-// rho is its own inverse: the column group whose lane holds row r
+// The score fold: 8 partial sums per lane (one per query row) are added over the 8 lanes that differ in lane
+// bits 0..2 by three halving exchanges (4 + 2 + 1 shuffles): with lane ^ 1 a lane hands over four rows and keeps
+// four, with lane ^ 2 two and two, with lane ^ 4 one and one.  Which rows a lane keeps follows its bits: it ends
+// with the total of row rho(lane % 8) = 4 bit0 + 2 bit1 + bit2 (the bit reversal of its column group).
+// rho is its own inverse (the column group whose lane holds row r) and distributes over xor
 __device__ __forceinline__ int rho(int r) { return ((r >> 2) & 1) | (r & 2) | ((r & 1) << 2); }
 
 __global__ void __launch_bounds__(WARPS * 32, 1) attn_f32_kernel(AttnArgs a)
 {
     extern __shared__ __align__(16) float smem[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int k4 = lane >> 3, cq = lane & 7, kgrp = lane & 24;
+    const int k4 = lane >> 3, cq = lane & 7;
     float *ring = smem + (size_t)warp * NST * STAGE_FLOATS;
     const uint32_t ring_u = (uint32_t)__cvta_generic_to_shared(ring);
     const int H = a.H;
@@ -99,7 +85,16 @@ __global__ void __launch_bounds__(WARPS * 32, 1) attn_f32_kernel(AttnArgs a)
         __syncwarp();   // the previous item's last stage has been read by every lane
         // stage b of the item: 16 keys x 256 bytes of each plane, 16 bytes per copy, two keys per warp instruction
         auto issue = [&](int b) {
-            if (b < nblk) {
+            if (b < nblk && b * SK + SK <= P) {   // a whole stage: no predicates
+                const uint32_t dst = ring_u + (uint32_t)((b % NST) * STAGE_FLOATS * 4);
+                const size_t row0 = (size_t)b * SK * kvs;
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int c = lane + 32 * u, key = c >> 4, col = (c & 15) << 2;
+                    cp16(dst + (uint32_t)((key * HD + col) * 4), kbase + row0 + (size_t)key * kvs + col, 16u);
+                    cp16(dst + (uint32_t)((PLANE_FLOATS + key * HD + col) * 4), vbase + row0 + (size_t)key * kvs + col, 16u);
+                }
+            } else if (b < nblk) {                 // the last, partial stage: keys past the prefix are filled with zeros
                 const uint32_t dst = ring_u + (uint32_t)((b % NST) * STAGE_FLOATS * 4);
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
@@ -115,23 +110,29 @@ __global__ void __launch_bounds__(WARPS * 32, 1) attn_f32_kernel(AttnArgs a)
 #pragma unroll
         for (int b = 0; b < NST - 1; ++b) issue(b);
 
-        float q[ROWS][8];
+        // rows in a lane-dependent order: register i holds row i ^ perm.  The halving exchanges of the score fold then
+        // keep the low registers and send the high ones in EVERY lane (no selects), and the lane that owns the
+        // weight of register i's row is simply lane ^ rho(i).
+        const int perm = rho(cq);
+        const float qs = scale * 1.4426950408889634f;   // scores in units of log 2: the weights are exp2
+        uint64_t q2[ROWS][4];
         const float *qg = (const float *)a.q + (size_t)env * H * a.q_stride + h * HD;
 #pragma unroll
-        for (int r = 0; r < ROWS; ++r) {
+        for (int i = 0; i < ROWS; ++i) {
+            const int r = i ^ perm;
             float4 lo = make_float4(0.f, 0.f, 0.f, 0.f), hi = lo;
             if (r < H) {
                 lo = *reinterpret_cast<const float4 *>(qg + (size_t)r * a.q_stride + 4 * cq);
                 hi = *reinterpret_cast<const float4 *>(qg + (size_t)r * a.q_stride + 32 + 4 * cq);
             }
-            q[r][0] = lo.x * scale; q[r][1] = lo.y * scale; q[r][2] = lo.z * scale; q[r][3] = lo.w * scale;
-            q[r][4] = hi.x * scale; q[r][5] = hi.y * scale; q[r][6] = hi.z * scale; q[r][7] = hi.w * scale;
+            q2[i][0] = pk2(lo.x * qs, lo.y * qs); q2[i][1] = pk2(lo.z * qs, lo.w * qs);
+            q2[i][2] = pk2(hi.x * qs, hi.y * qs); q2[i][3] = pk2(hi.z * qs, hi.w * qs);
         }
-        float o[ROWS][8];
+        uint64_t o2[ROWS][4];
 #pragma unroll
-        for (int r = 0; r < ROWS; ++r)
+        for (int i = 0; i < ROWS; ++i)
 #pragma unroll
-            for (int c = 0; c < 8; ++c) o[r][c] = 0.f;
+            for (int c = 0; c < 4; ++c) o2[i][c] = 0ull;
         float mrun = -INFINITY, lrun = 0.f;   // running maximum and (this lane's keys') sum of row rho(cq)
 
         for (int b = 0; b < nblk; ++b) {
@@ -144,17 +145,23 @@ __global__ void __launch_bounds__(WARPS * 32, 1) attn_f32_kernel(AttnArgs a)
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const int key = 4 * j + k4;
-                const float4 klo = *reinterpret_cast<const float4 *>(ks + key * HD + 4 * cq);
-                const float4 khi = *reinterpret_cast<const float4 *>(ks + key * HD + 32 + 4 * cq);
+                const ulonglong2 klo = *reinterpret_cast<const ulonglong2 *>(ks + key * HD + 4 * cq);
+                const ulonglong2 khi = *reinterpret_cast<const ulonglong2 *>(ks + key * HD + 32 + 4 * cq);
                 float part[ROWS];
 #pragma unroll
-                for (int r = 0; r < ROWS; ++r) {
-                    float t = q[r][0] * klo.x;
-                    t = fmaf(q[r][1], klo.y, t); t = fmaf(q[r][2], klo.z, t); t = fmaf(q[r][3], klo.w, t);
-                    t = fmaf(q[r][4], khi.x, t); t = fmaf(q[r][5], khi.y, t); t = fmaf(q[r][6], khi.z, t); t = fmaf(q[r][7], khi.w, t);
-                    part[r] = t;
+                for (int i = 0; i < ROWS; ++i) {
+                    uint64_t t = mul2(q2[i][0], klo.x);
+                    t = fma2(q2[i][1], klo.y, t); t = fma2(q2[i][2], khi.x, t); t = fma2(q2[i][3], khi.y, t);
+                    float te, to;
+                    upk2(t, te, to);
+                    part[i] = te + to;
                 }
-                const float sc = fold8(part, lane);
+                // fold across the eight column groups: 4 + 2 + 1 exchanges, register 0 ends as the score of row rho(cq)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) part[i] += __shfl_xor_sync(FULL, part[i + 4], 1);
+#pragma unroll
+                for (int i = 0; i < 2; ++i) part[i] += __shfl_xor_sync(FULL, part[i + 2], 2);
+                const float sc = part[0] + __shfl_xor_sync(FULL, part[1], 4);
                 s[j] = (b * SK + key < P) ? sc : -INFINITY;
             }
             // running softmax statistics of row rho(cq): the block's maximum over this lane's four keys and the
@@ -163,38 +170,43 @@ __global__ void __launch_bounds__(WARPS * 32, 1) attn_f32_kernel(AttnArgs a)
             bm = fmaxf(bm, __shfl_xor_sync(FULL, bm, 8));
             bm = fmaxf(bm, __shfl_xor_sync(FULL, bm, 16));
             const float mnew = fmaxf(mrun, bm);
-            const float al = expf(mrun - mnew);
+            const float al = exp2f(mrun - mnew);
             float p[4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) p[j] = expf(s[j] - mnew);
+            for (int j = 0; j < 4; ++j) p[j] = exp2f(s[j] - mnew);
             lrun = lrun * al + ((p[0] + p[1]) + (p[2] + p[3]));
             mrun = mnew;
             if (__any_sync(FULL, al != 1.0f)) {   // once the maxima have settled every factor is exactly 1
 #pragma unroll
-                for (int r = 0; r < ROWS; ++r) {
-                    const float ar = __shfl_sync(FULL, al, kgrp | rho(r));
+                for (int i = 0; i < ROWS; ++i) {
+                    const float ar = __shfl_xor_sync(FULL, al, rho(i));
+                    const uint64_t aa = pk2(ar, ar);
 #pragma unroll
-                    for (int c = 0; c < 8; ++c) o[r][c] *= ar;
+                    for (int c = 0; c < 4; ++c) o2[i][c] = mul2(o2[i][c], aa);
                 }
             }
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const int key = 4 * j + k4;
-                const float4 vlo = *reinterpret_cast<const float4 *>(vs + key * HD + 4 * cq);
-                const float4 vhi = *reinterpret_cast<const float4 *>(vs + key * HD + 32 + 4 * cq);
+                const ulonglong2 vlo = *reinterpret_cast<const ulonglong2 *>(vs + key * HD + 4 * cq);
+                const ulonglong2 vhi = *reinterpret_cast<const ulonglong2 *>(vs + key * HD + 32 + 4 * cq);
 #pragma unroll
-                for (int r = 0; r < ROWS; ++r) {
-                    const float pr = __shfl_sync(FULL, p[j], kgrp | rho(r));   // weight of (row r, this lane's key)
-                    o[r][0] = fmaf(pr, vlo.x, o[r][0]); o[r][1] = fmaf(pr, vlo.y, o[r][1]);
-                    o[r][2] = fmaf(pr, vlo.z, o[r][2]); o[r][3] = fmaf(pr, vlo.w, o[r][3]);
-                    o[r][4] = fmaf(pr, vhi.x, o[r][4]); o[r][5] = fmaf(pr, vhi.y, o[r][5]);
-                    o[r][6] = fmaf(pr, vhi.z, o[r][6]); o[r][7] = fmaf(pr, vhi.w, o[r][7]);
+                for (int i = 0; i < ROWS; ++i) {
+                    const float pr = __shfl_xor_sync(FULL, p[j], rho(i));   // weight of (register i's row, this lane's key)
+                    const uint64_t pp = pk2(pr, pr);
+                    o2[i][0] = fma2(pp, vlo.x, o2[i][0]); o2[i][1] = fma2(pp, vlo.y, o2[i][1]);
+                    o2[i][2] = fma2(pp, vhi.x, o2[i][2]); o2[i][3] = fma2(pp, vhi.y, o2[i][3]);
                 }
             }
         }
+        float o[ROWS][8];
+#pragma unroll
+        for (int i = 0; i < ROWS; ++i)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) upk2(o2[i][c], o[i][2 * c], o[i][2 * c + 1]);
         cp_wait<0>();   // only empty groups are left
         // totals over the four key slots (lane bits 3 and 4): the row sums everywhere, the outputs by two
-        // halving exchanges that leave rows 4 bit3 + 2 bit4 + {0, 1} with the lane
+        // halving exchanges that leave registers 4 bit3 + 2 bit4 + {0, 1} (rows: those ^ perm) with the lane
         lrun += __shfl_xor_sync(FULL, lrun, 8);
         lrun += __shfl_xor_sync(FULL, lrun, 16);
         const bool b3 = lane & 8, b4 = lane & 16;
@@ -215,7 +227,7 @@ __global__ void __launch_bounds__(WARPS * 32, 1) attn_f32_kernel(AttnArgs a)
         const int rbase = (b3 ? 4 : 0) + (b4 ? 2 : 0);
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
-            const int r = rbase + i;
+            const int r = (rbase + i) ^ perm;
             const float lr = __shfl_sync(FULL, lrun, rho(r));
             if (r < H) {
                 const size_t off = (size_t)(env * H + r) * a.o_stride + h * HD + 4 * cq;

@@ -3,6 +3,7 @@
 #pragma once
 #include "actgen_internal.h"
 #include "split3.cuh"
+#include "f32x2.cuh"
 
 #include <cuda.h>
 
@@ -43,29 +44,6 @@ __device__ __forceinline__ float gelu_erf(float z)
     p = fmaf(p, t, 0.127414796f);
     const float q = p * t * e;
     return z * (z >= 0.f ? 1.0f - q : q);
-}
-// Two fp32 values per instruction (fma / mul / add .f32x2: IEEE per lane, the same results as the scalar
-// forms).  The epilogue's arithmetic shares the schedulers with the single TMA and MMA threads, and across
-// all epilogue kinds the tensor pipe's active share falls one for one as the epilogue's issue share rises,
-// so halving its instruction count is worth more than any reordering.
-__device__ __forceinline__ uint64_t pk2(float a, float b)
-{
-    uint64_t r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
-    return r;
-}
-__device__ __forceinline__ void upk2(uint64_t v, float &a, float &b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v)); }
-__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c)
-{
-    uint64_t d;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-    return d;
-}
-__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b)
-{
-    uint64_t d;
-    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
 }
 // gelu_erf of two values at once: the same approximation with the polynomial and the products in packed
 // form; only |z|, the reciprocal and the exponential stay scalar.  With q = 1/2 (a1 t + ... + a5 t^5) exp(-z^2/2),
