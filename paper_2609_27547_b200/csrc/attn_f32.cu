@@ -17,7 +17,9 @@
 //
 // Keys and values stream through a per-warp ring of 16-key stages filled by cp.async (zero fill
 // past the prefix), so a warp's global-memory latency hides behind its own arithmetic and the
-// eight warps of a CTA never wait on one another.  Keys are visited in blocks of 16 in index
+// eight warps of a CTA never wait on one another.  The copies run two stages ahead across item
+// boundaries (an item's first stage carries its query block), so short prefixes and the 8-key
+// self-attention do not pay a round trip to memory per item.  Keys are visited in blocks of 16 in index
 // order with a running maximum and sum; an item's arithmetic involves nothing but the item, so
 // the result does not depend on the grid size or on what else is in the batch.
 #include "actgen_internal.h"
@@ -37,7 +39,8 @@ constexpr int SK = 16;            // keys per stage
 constexpr int NST = 3;            // stages per warp
 constexpr int PLANE_FLOATS = SK * HD;
 constexpr int STAGE_FLOATS = 2 * PLANE_FLOATS;                 // keys, then values
-constexpr int SMEM_BYTES = WARPS * NST * STAGE_FLOATS * 4;     // 192 KB
+constexpr int WARP_FLOATS = NST * STAGE_FLOATS + 2 * ROWS * HD;   // a warp's ring and its two query blocks: 28 KB
+constexpr int SMEM_BYTES = WARPS * (WARP_FLOATS * 4 + 16);         // plus the prefix lengths of those two items
 constexpr unsigned FULL = 0xffffffffu;
 
 __device__ __forceinline__ void cp16(uint32_t dst, const void *src, uint32_t nbytes)
@@ -54,93 +57,129 @@ template <int N> __device__ __forceinline__ void cp_wait() { asm volatile("cp.as
 // rho is its own inverse (the column group whose lane holds row r) and distributes over xor
 __device__ __forceinline__ int rho(int r) { return ((r >> 2) & 1) | (r & 2) | ((r & 1) << 2); }
 
+// Where the copies of a warp stand: the next stage to request belongs to block b of `item`.
+struct Cursor {
+    int item, seq, b, nblk, P, kvs;     // seq = how many items this warp has started before this one
+    const float *kbase, *vbase, *qg;
+};
+
 __global__ void __launch_bounds__(WARPS * 32, 1) attn_f32_kernel(AttnArgs a)
 {
     extern __shared__ __align__(16) float smem[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int k4 = lane >> 3, cq = lane & 7;
-    float *ring = smem + (size_t)warp * NST * STAGE_FLOATS;
-    const uint32_t ring_u = (uint32_t)__cvta_generic_to_shared(ring);
+    float *ring = smem + (size_t)warp * WARP_FLOATS;
+    float *qring = ring + NST * STAGE_FLOATS;                  // two query blocks: items alternate
+    int *pmeta = reinterpret_cast<int *>(smem + (size_t)WARPS * WARP_FLOATS) + warp * 4;   // their prefix lengths
+    const uint32_t ring_u = (uint32_t)__cvta_generic_to_shared(ring), qring_u = (uint32_t)__cvta_generic_to_shared(qring);
     const int H = a.H;
-    const float scale = 1.0f / sqrtf((float)HD);
-    const int items = a.n_envs * a.n_heads;
+    const float qs = 1.4426950408889634f / sqrtf((float)HD);   // scores in units of log 2: the weights are exp2
+    const int items = a.n_envs * a.n_heads, stride = gridDim.x * WARPS;
+    const int perm = rho(cq);
     pdl_launch_dependents();
     pdl_wait();
-    for (int item = blockIdx.x * WARPS + warp; item < items; item += gridDim.x * WARPS) {
+
+    auto seek = [&](Cursor &c, int item) {
+        c.item = item; c.b = 0;
+        if (item >= items) return;
         const int env = item / a.n_heads, h = item - env * a.n_heads;
-        const float *kbase, *vbase;
-        int P, kvs;
         if (a.self) {
-            kbase = (const float *)a.k_self + (size_t)env * H * a.kv_stride + h * HD;
-            vbase = (const float *)a.v_self + (size_t)env * H * a.kv_stride + h * HD;
-            P = H; kvs = a.kv_stride;
+            c.kbase = (const float *)a.k_self + (size_t)env * H * a.kv_stride + h * HD;
+            c.vbase = (const float *)a.v_self + (size_t)env * H * a.kv_stride + h * HD;
+            c.P = H; c.kvs = a.kv_stride;
         } else {
             const EnvMeta m = a.meta[env];
-            P = m.P; kvs = a.d;
-            const int pr = a.plane_rows ? a.plane_rows : P;
-            kbase = (const float *)m.kv + (size_t)a.kv_plane * 2 * pr * a.d + h * HD;
-            vbase = kbase + (size_t)pr * a.d;
+            c.P = m.P; c.kvs = a.d;
+            const int pr = a.plane_rows ? a.plane_rows : m.P;
+            c.kbase = (const float *)m.kv + (size_t)a.kv_plane * 2 * pr * a.d + h * HD;
+            c.vbase = c.kbase + (size_t)pr * a.d;
         }
-        const int nblk = (P + SK - 1) / SK;
-        __syncwarp();   // the previous item's last stage has been read by every lane
-        // stage b of the item: 16 keys x 256 bytes of each plane, 16 bytes per copy, two keys per warp instruction
-        auto issue = [&](int b) {
-            if (b < nblk && b * SK + SK <= P) {   // a whole stage: no predicates
-                const uint32_t dst = ring_u + (uint32_t)((b % NST) * STAGE_FLOATS * 4);
-                const size_t row0 = (size_t)b * SK * kvs;
+        c.nblk = c.P > SK ? (c.P + SK - 1) / SK : 1;
+        c.qg = (const float *)a.q + (size_t)env * H * a.q_stride + h * HD;
+    };
+    // Requests the cursor's stage into ring slot `slot` (16 keys x 256 bytes of each plane, 16 bytes per copy, two
+    // keys per warp instruction; an item's first stage brings its query block and prefix length along) and moves
+    // the cursor on, into the next item when this one is exhausted.  One commit group per call, empty at the end.
+    auto issue_next = [&](Cursor &c, int slot) {
+        if (c.item < items) {
+            const uint32_t dst = ring_u + (uint32_t)(slot * STAGE_FLOATS * 4);
+            if (c.b == 0) {
+                const uint32_t qdst = qring_u + (uint32_t)((c.seq & 1) * ROWS * HD * 4);
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const int c = lane + 32 * u, key = c >> 4, col = (c & 15) << 2;
-                    cp16(dst + (uint32_t)((key * HD + col) * 4), kbase + row0 + (size_t)key * kvs + col, 16u);
-                    cp16(dst + (uint32_t)((PLANE_FLOATS + key * HD + col) * 4), vbase + row0 + (size_t)key * kvs + col, 16u);
+                for (int u = 0; u < 4; ++u) {
+                    const int ch = lane + 32 * u, r = ch >> 4, col = (ch & 15) << 2;
+                    cp16(qdst + (uint32_t)((r * HD + col) * 4), c.qg + (size_t)(r < H ? r : 0) * a.q_stride + col, r < H ? 16u : 0u);
                 }
-            } else if (b < nblk) {                 // the last, partial stage: keys past the prefix are filled with zeros
-                const uint32_t dst = ring_u + (uint32_t)((b % NST) * STAGE_FLOATS * 4);
+                if (lane == 0) pmeta[c.seq & 1] = c.P;
+            }
+            if (c.b * SK + SK <= c.P) {   // a whole stage: no predicates
+                const size_t row0 = (size_t)c.b * SK * c.kvs;
 #pragma unroll
                 for (int u = 0; u < 8; ++u) {
-                    const int c = lane + 32 * u, key = c >> 4, col = (c & 15) << 2;
-                    const bool in = b * SK + key < P;
-                    const size_t src = (size_t)(in ? b * SK + key : 0) * kvs + col;
-                    cp16(dst + (uint32_t)((key * HD + col) * 4), kbase + src, in ? 16u : 0u);
-                    cp16(dst + (uint32_t)((PLANE_FLOATS + key * HD + col) * 4), vbase + src, in ? 16u : 0u);
+                    const int ch = lane + 32 * u, key = ch >> 4, col = (ch & 15) << 2;
+                    cp16(dst + (uint32_t)((key * HD + col) * 4), c.kbase + row0 + (size_t)key * c.kvs + col, 16u);
+                    cp16(dst + (uint32_t)((PLANE_FLOATS + key * HD + col) * 4), c.vbase + row0 + (size_t)key * c.kvs + col, 16u);
+                }
+            } else {                      // the last, partial stage: keys past the prefix are filled with zeros
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int ch = lane + 32 * u, key = ch >> 4, col = (ch & 15) << 2;
+                    const bool in = c.b * SK + key < c.P;
+                    const size_t src = (size_t)(in ? c.b * SK + key : 0) * c.kvs + col;
+                    cp16(dst + (uint32_t)((key * HD + col) * 4), c.kbase + src, in ? 16u : 0u);
+                    cp16(dst + (uint32_t)((PLANE_FLOATS + key * HD + col) * 4), c.vbase + src, in ? 16u : 0u);
                 }
             }
-            cp_commit();   // one group per call, empty past the last block: the wait below counts groups
-        };
-#pragma unroll
-        for (int b = 0; b < NST - 1; ++b) issue(b);
+            if (++c.b == c.nblk) {
+                const int seq = c.seq + 1;
+                seek(c, c.item + stride);
+                c.seq = seq;
+            }
+        }
+        cp_commit();
+    };
 
+    // The copies run NST - 1 stages ahead of the arithmetic, across item boundaries: while an item's last blocks
+    // are computed the next item's first blocks (and queries) are already on their way.
+    Cursor ic;
+    ic.seq = 0;
+    seek(ic, blockIdx.x * WARPS + warp);
+    int g = 0;   // stages computed so far by this warp; stage g lives in ring slot g % NST
+#pragma unroll
+    for (int t = 0; t < NST - 1; ++t) issue_next(ic, t);
+
+    int seq = 0;
+    for (int item = blockIdx.x * WARPS + warp; item < items; item += stride, ++seq) {
+        const int env = item / a.n_heads, h = item - env * a.n_heads;
         // rows in a lane-dependent order: register i holds row i ^ perm.  The halving exchanges of the score fold then
         // keep the low registers and send the high ones in EVERY lane (no selects), and the lane that owns the
         // weight of register i's row is simply lane ^ rho(i).
-        const int perm = rho(cq);
-        const float qs = scale * 1.4426950408889634f;   // scores in units of log 2: the weights are exp2
-        uint64_t q2[ROWS][4];
-        const float *qg = (const float *)a.q + (size_t)env * H * a.q_stride + h * HD;
-#pragma unroll
-        for (int i = 0; i < ROWS; ++i) {
-            const int r = i ^ perm;
-            float4 lo = make_float4(0.f, 0.f, 0.f, 0.f), hi = lo;
-            if (r < H) {
-                lo = *reinterpret_cast<const float4 *>(qg + (size_t)r * a.q_stride + 4 * cq);
-                hi = *reinterpret_cast<const float4 *>(qg + (size_t)r * a.q_stride + 32 + 4 * cq);
-            }
-            q2[i][0] = pk2(lo.x * qs, lo.y * qs); q2[i][1] = pk2(lo.z * qs, lo.w * qs);
-            q2[i][2] = pk2(hi.x * qs, hi.y * qs); q2[i][3] = pk2(hi.z * qs, hi.w * qs);
-        }
-        uint64_t o2[ROWS][4];
+        uint64_t q2[ROWS][4], o2[ROWS][4];
 #pragma unroll
         for (int i = 0; i < ROWS; ++i)
 #pragma unroll
             for (int c = 0; c < 4; ++c) o2[i][c] = 0ull;
         float mrun = -INFINITY, lrun = 0.f;   // running maximum and (this lane's keys') sum of row rho(cq)
+        int P = 0, nblk = 1;
 
-        for (int b = 0; b < nblk; ++b) {
-            __syncwarp();            // every lane is done with the stage the next copies overwrite
-            issue(b + NST - 1);
-            cp_wait<NST - 1>();      // this lane's copies of stage b have landed ...
-            __syncwarp();            // ... and so have the other lanes'
-            const float *ks = ring + (b % NST) * STAGE_FLOATS, *vs = ks + PLANE_FLOATS;
+        for (int b = 0; b < nblk; ++b, ++g) {
+            cp_wait<NST - 2>();      // this lane's copies of stage g have landed ...
+            __syncwarp();            // ... and so have the other lanes'; everyone is done with stage g - 1
+            if (b == 0) {
+                P = pmeta[seq & 1];
+                nblk = P > SK ? (P + SK - 1) / SK : 1;
+                const float *qsm = qring + (seq & 1) * ROWS * HD;
+#pragma unroll
+                for (int i = 0; i < ROWS; ++i) {
+                    const float4 lo = *reinterpret_cast<const float4 *>(qsm + (i ^ perm) * HD + 4 * cq);
+                    const float4 hi = *reinterpret_cast<const float4 *>(qsm + (i ^ perm) * HD + 32 + 4 * cq);
+                    q2[i][0] = pk2(lo.x * qs, lo.y * qs); q2[i][1] = pk2(lo.z * qs, lo.w * qs);
+                    q2[i][2] = pk2(hi.x * qs, hi.y * qs); q2[i][3] = pk2(hi.z * qs, hi.w * qs);
+                }
+            }
+            issue_next(ic, (g + NST - 1) % NST);   // into the slot of stage g - 1 (and, for a new item, over the queries
+                                                   // and prefix length of the item before this one: read above)
+            const float *ks = ring + (g % NST) * STAGE_FLOATS, *vs = ks + PLANE_FLOATS;
             float s[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
@@ -204,7 +243,6 @@ __global__ void __launch_bounds__(WARPS * 32, 1) attn_f32_kernel(AttnArgs a)
         for (int i = 0; i < ROWS; ++i)
 #pragma unroll
             for (int c = 0; c < 4; ++c) upk2(o2[i][c], o[i][2 * c], o[i][2 * c + 1]);
-        cp_wait<0>();   // only empty groups are left
         // totals over the four key slots (lane bits 3 and 4): the row sums everywhere, the outputs by two
         // halving exchanges that leave registers 4 bit3 + 2 bit4 + {0, 1} (rows: those ^ perm) with the lane
         lrun += __shfl_xor_sync(FULL, lrun, 8);
@@ -244,6 +282,7 @@ __global__ void __launch_bounds__(WARPS * 32, 1) attn_f32_kernel(AttnArgs a)
             }
         }
     }
+    cp_wait<0>();   // only empty groups are left
 }
 
 }  // namespace af
