@@ -98,6 +98,41 @@ def test_fp32_projections_on_tensor_cores_and_on_the_plain_alus():
     print("fp32 max chunk-relative error: tensor cores %.2e, FFMA %.2e" % (chunk_rel_err(got, ref), chunk_rel_err(alu, ref)))
 
 
+@pytest.mark.parametrize("H,A,P", [(8, 7, (15, 17)), (5, 3, (1, 40)), (1, 2, (1, 3)), (8, 7, (250, 530)), (7, 7, (16, 16))])
+def test_fp32_warp_per_item_attention_edge_shapes(H, A, P):
+    """The fp32 attention kernel that gives every (environment, head) to one warp (head_dim 64, H <= 8):
+    fewer than eight query rows, prefixes shorter than / equal to / just past one 16-key stage and many
+    stages long, more items than warps so that a warp's copies run on into its next item (whose prefix
+    length differs).  Against the oracle, across quotas, and alone."""
+    w = synth.scaled(synth.WORKLOADS[0], B=41, dtype="f32", H=H, A=A, P=P, K=3, mixed_steps=True)
+    wt, envs = _setup(w)
+    ref = oracle_run(w, wt, envs)
+    ids = list(range(w.B))
+    r = Runner(w, wt, envs)
+    got = stack(r.run([ids]), ids)
+    assert chunk_rel_err(got, ref) <= TOL["f32"]
+    for q in (2, 5, 148):                 # 2 CTAs x 8 warps for 164 items: about ten items per warp
+        assert np.array_equal(stack(r.run([ids], quota=q), ids), got), "quota %d" % q
+    assert np.array_equal(stack(r.run([[e] for e in ids[:5]] + [ids[5:]], quota=3), ids), got)
+    r.close()
+    r = Runner(w, wt, envs, flags=B.FLAG_FORCE_SIMT)   # the block-per-four-items kernel on the same inputs
+    alu = stack(r.run([ids]), ids)
+    r.close()
+    assert chunk_rel_err(alu, ref) <= TOL["f32"]
+
+
+def test_fp32_other_head_dims_take_the_general_attention_kernel():
+    """head_dim 32 and 128 in fp32 are outside the warp-per-item kernel: the general one serves them."""
+    for d, nh in ((128, 4), (256, 2)):
+        w = synth.scaled(synth.WORKLOADS[0], B=11, dtype="f32", d=d, n_heads=nh, P=(3, 70), mixed_steps=True)
+        wt, envs = _setup(w)
+        ref = oracle_run(w, wt, envs)
+        r = Runner(w, wt, envs)
+        got = stack(r.run([list(range(w.B))]), range(w.B))
+        r.close()
+        assert chunk_rel_err(got, ref) <= TOL["f32"]
+
+
 def test_bf16_plain_alu_kernels_parity():
     """The bf16 model on the plain-ALU kernels (the path taken when d is not a multiple of 256,
     and on request)."""
