@@ -87,6 +87,9 @@ def parse_args(argv=None):
     ap.add_argument("--inflight", type=int, default=16, help="groups queued before a batch is launched")
     ap.add_argument("--fused", action="store_true",
                     help="run every batch through the persistent step kernel (one resident grid for all Euler steps)")
+    ap.add_argument("--sm-split", action="store_true",
+                    help="harness: the step as one batch on the quota against two half-batches side by side on two streams, "
+                         "each on a share of the quota (does an SM split overlap the K/V stream with the projections?)")
     ap.add_argument("--sweep", action="store_true",
                     help="one line per other configuration: configs[0..2], and configs[3] at quotas 148/74/37/16 with and "
                          "without the streaming co-runner (the committed summary of these lines sits with the profiles)")
@@ -631,6 +634,72 @@ def run_pgen_sweep(args):
                                "quota_sms": [max(1, round(N_SMS * q / 100)) for q in quotas], "batch": batches, "rate": rate}}))
 
 
+def run_sm_split(args):
+    """Can the HBM-bound K/V stream of one half of the environments hide behind the tensor-bound projections of
+    the other half?  Times a step (a) as one batch on the whole quota and (b) as two half-batches submitted to two
+    streams, each with a share of the quota, so that the two run side by side and drift out of phase (one in
+    attention while the other is in its projections).  Same arithmetic per environment in both (bit-identical
+    results: checked here)."""
+    import torch
+    from paper_2609_27547_b200 import binding as B
+    from paper_2609_27547_b200 import synth
+    torch.cuda.set_device(0)
+    w = synth.WORKLOADS[args.config]
+    seed = args.seed or synth.DEFAULT_SEED
+    quota = args.quota if args.quota >= 0 else w.quota
+    quota = quota or N_SMS
+    nb = args.envs or w.B
+    wt = synth.make_weights(w, seed, device="cuda")
+    envs = [synth.make_env(w, e, seed, device="cuda") for e in range(nb)]
+    gen = B.ActGen(B.cfg_for(w, max_group_envs=nb, max_inflight_groups=1), wt)
+    noise = torch.stack([e.noise for e in envs]).contiguous()
+    out = torch.empty_like(noise)
+    main_s, side = torch.cuda.Stream(), [torch.cuda.Stream(), torch.cuda.Stream()]
+    kv = [e.kv for e in envs]
+
+    def one_batch():
+        gen.submit(list(range(nb)), kv, noise, out, sm_quota=quota, stream=main_s)
+        gen.sync()
+
+    def split(shares):
+        def step():
+            ev = torch.cuda.Event()
+            ev.record(main_s)
+            lo = 0
+            for p, q in enumerate(shares):
+                hi = nb if p == len(shares) - 1 else lo + nb // len(shares)
+                side[p].wait_event(ev)
+                gen.submit(list(range(lo, hi)), kv[lo:hi], noise[lo:hi], out[lo:hi], sm_quota=q, stream=side[p])
+                done = torch.cuda.Event()
+                done.record(side[p])
+                main_s.wait_event(done)
+                lo = hi
+            gen.sync()
+        return step
+
+    def timed(step):
+        for _ in range(max(args.min_warmup, 1)):
+            step()
+        mon = ClockSampler(0)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(main_s)
+        for _ in range(args.steps):
+            step()
+        e1.record(main_s)
+        torch.cuda.synchronize()
+        clk = mon.stop()
+        return e0.elapsed_time(e1) / args.steps, clk.get("sm_mhz"), out.clone()
+
+    res = {"workload": synth.workload_label(args.config), "envs": nb, "quota": quota, "steps": args.steps, "unit": "ms per step"}
+    ms, mhz, ref = timed(one_batch)
+    res["one_batch"] = {"ms": ms, "sm_mhz": mhz}
+    for shares in ([quota // 2, quota - quota // 2], [quota, quota]):   # the second one occupies 2 x quota SMs: context, not a quota run
+        ms, mhz, got = timed(split(shares))
+        res["two_half_batches_%d_%d" % tuple(shares)] = {"ms": ms, "sm_mhz": mhz, "bit_identical": bool(torch.equal(got, ref))}
+    gen.destroy()
+    print(json.dumps({"sm_split": res}))
+
+
 def main():
     args = parse_args()
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
@@ -641,6 +710,8 @@ def main():
         return run_sweep(args)
     if args.pgen_sweep:
         return run_pgen_sweep(args)
+    if args.sm_split:
+        return run_sm_split(args)
     if args.rollout_sim:
         import torch
         from paper_2609_27547_b200 import rollout_sim as R
