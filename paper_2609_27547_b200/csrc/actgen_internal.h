@@ -130,6 +130,10 @@ bool gemm_tc3_supported(int N, int K);
 cudaError_t launch_split3(const float *src, void *p0, void *p1, void *p2, size_t n, int grid, cudaStream_t st);
 cudaError_t launch_gemm_tc3(const TensorMap128 *ta, const TensorMap128 *tw, const GemmArgs &a, int grid, unsigned long long limit_ns,
                             int *status, cudaStream_t st);
+// the same on CTA pairs (256 x 256 tiles; N a multiple of 256, grid >= 2): bit-identical results (gemm_tc3p.cu)
+bool gemm_tc3p_supported(int N, int K);
+cudaError_t launch_gemm_tc3p(const TensorMap128 *ta, const TensorMap128 *tw, const GemmArgs &a, int grid, unsigned long long limit_ns,
+                             int *status, cudaStream_t st);
 
 // ---- the persistent step kernel (one resident grid for all Euler steps of a small batch) ----
 // Per-layer table in device memory: TMA descriptors of the six matrices (128-row boxes) and the gains.

@@ -493,6 +493,19 @@ struct Launcher {
     }
 };
 
+// fp32 models: CTA pairs on 256 x 256 tiles or single CTAs on 128 x 128 tiles (bit-identical results).
+static bool tc3_use_pairs(const ebrl_actgen *h, int M, int N, int K, int grid)
+{
+    if (grid < 2 || !gemm_tc3p_supported(N, K)) return false;
+    if (h->force_shape == 2) return true;
+    if (h->force_shape) return false;
+    // rounds x time per round: a 128 x 128 tile takes about 5.5 us at K = 256, a 256 x 256 pair tile about 9.5 us (measured;
+    // both scale with K).  Pairs win where a CTA gets several tiles -- small quotas, wide projections.
+    const long rows128 = (M + 127) / 128, rows256 = (M + 255) / 256;
+    const long r1 = (rows128 * (N / 128) + grid - 1) / grid, rp = (rows256 * (N / 256) + grid / 2 - 1) / (grid / 2);
+    return rp * 19 <= r1 * 11;
+}
+
 cudaError_t launch_attn(ebrl_actgen *h, const AttnArgs &a, int grid, cudaStream_t st)
 {
     if (h->use_attn_mma) return launch_attn_mma(a, grid, h->attn_lookahead, h->wait_ns, h->status_d, st);
@@ -611,7 +624,10 @@ cudaError_t enqueue_batch(ebrl_actgen *h, Slot &s, int S, const int32_t *n_activ
                         const TensorMap128 *ta3 = A == s.xg ? s.t_xg3 : (A == s.att ? s.t_att3 : s.t_u3);
                         if (epi == EPI_RESID) { g.xg = s.xg3[0]; g.out_t1 = s.xg3[1]; g.out_t2 = s.xg3[2]; }
                         if (epi == EPI_SCALE_GELU) { g.C = s.u3[0]; g.out_t1 = s.u3[1]; g.out_t2 = s.u3[2]; }
-                        ln.run(EBRL_KC_GEMM, 2.0 * M * N * K, bytes, [&] { return launch_gemm_tc3(ta3, w3, g, grid, h->wait_ns, h->status_d, st); });
+                        if (tc3_use_pairs(h, M, N, K, grid))
+                            ln.run(EBRL_KC_GEMM, 2.0 * M * N * K, bytes, [&] { return launch_gemm_tc3p(ta3, w3, g, grid, h->wait_ns, h->status_d, st); });
+                        else
+                            ln.run(EBRL_KC_GEMM, 2.0 * M * N * K, bytes, [&] { return launch_gemm_tc3(ta3, w3, g, grid, h->wait_ns, h->status_d, st); });
                     } else if (h->use_tc) {
                         const int shape = pick_tile_shape(h, M, N, grid);
                         if (shape == 2)

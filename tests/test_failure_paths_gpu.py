@@ -63,9 +63,10 @@ def _expect_timeout_then_recover(flags, monkeypatch=None, shape=None, dtype="bf1
     assert chunk_rel_err(got, oracle_run(w, wt, envs)) <= TOL[dtype]
 
 
-def test_fp32_tensor_core_projection_kernel_gives_up_cleanly():
-    """The split-operand kernel of the fp32 models (six operand tiles per stage)."""
-    _expect_timeout_then_recover(B.FLAG_TEST_DROP_GEMM_COPIES, dtype="f32")
+@pytest.mark.parametrize("shape", ["128", "2"])
+def test_fp32_tensor_core_projection_kernels_give_up_cleanly(monkeypatch, shape):
+    """The split-operand kernels of the fp32 models (six operand tiles per stage): single CTAs and CTA pairs."""
+    _expect_timeout_then_recover(B.FLAG_TEST_DROP_GEMM_COPIES, monkeypatch, shape, dtype="f32")
 
 
 @pytest.mark.parametrize("shape", ["128", "256", "2"])

@@ -133,6 +133,31 @@ def test_fp32_other_head_dims_take_the_general_attention_kernel():
         assert chunk_rel_err(got, ref) <= TOL["f32"]
 
 
+def test_fp32_tensor_core_gemm_on_pairs_and_on_single_ctas_agree(monkeypatch):
+    """The fp32 tensor-core GEMM runs on CTA pairs (256 x 256 tiles) or on single CTAs (128 x 128), chosen per
+    projection; forced in turn (`EBRL_GEMM_SHAPE` = 2 / 128, read when the handle is created) on 37 envs x H = 8
+    = 296 rows (one full 256-row pair tile plus a 40-row tail in the leader CTA only) of a d = 512 model: each
+    against the oracle, and bit-identical to each other and to the library's own choice at several quotas."""
+    w = synth.scaled(synth.WORKLOADS[0], B=37, dtype="f32", d=512, n_heads=8, L=2, K=3, P=(1, 97), mixed_steps=True)
+    wt, envs = _setup(w)
+    ref = oracle_run(w, wt, envs)
+    ids = list(range(w.B))
+    got = {}
+    for shape in ("128", "2"):
+        monkeypatch.setenv("EBRL_GEMM_SHAPE", shape)
+        r = Runner(w, wt, envs)
+        got[shape] = stack(r.run([ids]), ids)
+        assert np.array_equal(stack(r.run([ids], quota=5), ids), got[shape])
+        r.close()
+        assert chunk_rel_err(got[shape], ref) <= TOL["f32"], shape
+    assert np.array_equal(got["128"], got["2"])
+    monkeypatch.delenv("EBRL_GEMM_SHAPE")
+    r = Runner(w, wt, envs)
+    for q in (0, 2, 3, 16):
+        assert np.array_equal(stack(r.run([ids], quota=q), ids), got["2"]), "quota %d" % q
+    r.close()
+
+
 def test_bf16_plain_alu_kernels_parity():
     """The bf16 model on the plain-ALU kernels (the path taken when d is not a multiple of 256,
     and on request)."""
