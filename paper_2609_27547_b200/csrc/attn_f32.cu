@@ -176,6 +176,7 @@ __global__ void __launch_bounds__(WARPS * 32, 1) attn_f32_kernel(AttnArgs a)
                     q2[i][0] = pk2(lo.x * qs, lo.y * qs); q2[i][1] = pk2(lo.z * qs, lo.w * qs);
                     q2[i][2] = pk2(hi.x * qs, hi.y * qs); q2[i][3] = pk2(hi.z * qs, hi.w * qs);
                 }
+                __syncwarp();        // every lane has read the queries and the prefix length before anyone's copies replace them
             }
             issue_next(ic, (g + NST - 1) % NST);   // into the slot of stage g - 1 (and, for a new item, over the queries
                                                    // and prefix length of the item before this one: read above)
