@@ -122,8 +122,10 @@ cudaError_t launch_gemm_tc2(const TensorMap128 &ta, const TensorMap128 &tw, cons
 
 // Tensor-core (mma.sync) attention over bulk-copied K/V rows, bf16 models.
 bool attn_mma_supported(int H, int n_heads, int hd);
-int attn_mma_make_map(TensorMap128 *out, const void *base, uint64_t rows, uint64_t width, int n_heads, int hd);
-cudaError_t launch_attn_mma(const AttnArgs &a, int grid, int lookahead_blocks, unsigned long long limit_ns, int *status, cudaStream_t st);
+int attn_mma_slab_heads(int n_heads, int hd, bool wide);   // heads per slab: up to 16 x 64 or 8 x 128 columns when wide, else up to 8 heads
+int attn_mma_make_map(TensorMap128 *out, const void *base, uint64_t rows, uint64_t width, int slab_heads, int hd);
+cudaError_t launch_attn_mma(const AttnArgs &a, int grid, int slab_heads, int lookahead_blocks, unsigned long long limit_ns, int *status,
+                            cudaStream_t st);
 
 // fp32 GEMM on the tensor cores by splitting each operand into three bf16 terms (six products per k-slice).
 bool gemm_tc3_supported(int N, int K);

@@ -121,6 +121,7 @@ struct ebrl_actgen {
     bool pdl_allowed = true;      // EBRL_PDL=0 turns programmatic dependent launch off
     int attn_lookahead = 2;       // EBRL_ATTN_LOOKAHEAD: key blocks the attention producer asks L2 for ahead of its ring
     bool use_attn_mma = false;    // tensor-core attention (bf16, H <= 16, head_dim 64/128)
+    int attn_hpc = 8;             // heads per slab of the tensor-core attention kernel and its descriptors
     bool use_attn_f32 = false;    // warp-per-item fp32 attention (head_dim 64, H <= 8)
     int *status_d = nullptr;      // device status word written by kernels whose waits ran out
     unsigned long long wait_ns = 0;
@@ -508,7 +509,7 @@ static bool tc3_use_pairs(const ebrl_actgen *h, int M, int N, int K, int grid)
 
 cudaError_t launch_attn(ebrl_actgen *h, const AttnArgs &a, int grid, cudaStream_t st)
 {
-    if (h->use_attn_mma) return launch_attn_mma(a, grid, h->attn_lookahead, h->wait_ns, h->status_d, st);
+    if (h->use_attn_mma) return launch_attn_mma(a, grid, h->attn_hpc, h->attn_lookahead, h->wait_ns, h->status_d, st);
     if (h->use_attn_f32) return launch_attn_f32(a, grid, st);
     return launch_attn_simt(a, h->bf16, grid, st);
 }
@@ -581,7 +582,7 @@ cudaError_t enqueue_batch(ebrl_actgen *h, Slot &s, int S, const int32_t *n_activ
         if ((ln.err = cudaMemsetAsync(s.fctl_d + c.K_steps, 0, sizeof(int) * ((size_t)c.K_steps * s.mt_max + 4 * 256 + 2 * 12 * 4 * 256 + 4 + 4 * 4000), st)) != cudaSuccess) return ln.err;
         FusedArgs f{};
         f.H = H; f.A = c.A; f.d = d; f.md = md; f.n_layers = L; f.n_heads = c.n_heads; f.hd = h->hd;
-        f.hpc = c.n_heads < 8 ? c.n_heads : 8; f.K = c.K_steps; f.S = S; f.ne0 = n_active[0];
+        f.hpc = h->attn_hpc; f.K = c.K_steps; f.S = S; f.ne0 = n_active[0];
         f.kv_layers = c.kv_layers; f.plane_rows = c.d_ctx > 0 ? s.prefix_rows : 0;
         f.eps = c.rms_eps; f.inv_d = 1.0f / (float)d;
         f.meta = s.meta_d; f.n_active = s.fctl_d; f.done = s.fctl_d + c.K_steps; f.mt_max = s.mt_max;
@@ -738,7 +739,7 @@ ebrl_status_t flush_slot(ebrl_actgen *h, Slot &s)
             m.hid = m.kv;
             m.kv = (const char *)s.planes + (size_t)m.row0 * c.d * h->esz;
             // the environment's view of the planes: from its first row to the end of the last plane
-            if (with_maps && attn_mma_make_map(&maps_packed[j], m.kv, (uint64_t)2 * c.n_layers * prefix_rows - m.row0, c.d, c.n_heads, h->hd))
+            if (with_maps && attn_mma_make_map(&maps_packed[j], m.kv, (uint64_t)2 * c.n_layers * prefix_rows - m.row0, c.d, h->attn_hpc, h->hd))
                 return fail(h, EBRL_ERR_CUDA, "cuTensorMapEncodeTiled failed for projected prefix planes");
         }
         if (h->use_tc && make_tmap_bf16(&s.t_hid, s.hid_pack, (uint64_t)c.d_ctx, (uint64_t)prefix_rows, (uint32_t)gemm_tc_box_rows_a()))
@@ -903,7 +904,7 @@ ebrl_status_t submit_impl(ebrl_actgen *h, int32_t n, const int64_t *env_ids, con
         group_maps.resize(n);
         for (int i = 0; i < n; ++i) {
             const int P = (ext && ext->prefix_len) ? ext->prefix_len[i] : c.max_prefix_len;
-            if (attn_mma_make_map(&group_maps[i], kv_dev[i], (uint64_t)c.kv_layers * 2 * P, c.d, c.n_heads, h->hd))
+            if (attn_mma_make_map(&group_maps[i], kv_dev[i], (uint64_t)c.kv_layers * 2 * P, c.d, h->attn_hpc, h->hd))
                 return fail(h, EBRL_ERR_CUDA, "cuTensorMapEncodeTiled failed for the prefix planes of environment %lld", (long long)env_ids[i]);
         }
     }
@@ -1067,6 +1068,12 @@ ebrl_status_t ebrl_actgen_create(const ebrl_actgen_cfg_t *cfg, const ebrl_actgen
     h->fused_ok = h->use_tc && h->use_attn_mma && fused_supported(cfg->H, cfg->A, d, md, cfg->n_heads, h->hd);
     if (const char *e6 = getenv("EBRL_FUSED_MAX_ROWS")) h->fused_max_rows = atol(e6);
     if (const char *e7 = getenv("EBRL_TRACE")) h->trace = atoi(e7) != 0;
+    {   // the attention descriptors are shared with the persistent step kernel, whose slabs are at most 8 heads: wide slabs
+        // only on handles that cannot take that path
+        const bool fused_may_run = h->fused_ok && !(cfg->flags & EBRL_FLAG_NO_FUSED) &&
+                                   ((cfg->flags & EBRL_FLAG_FORCE_FUSED) || h->fused_max_rows > 0);
+        h->attn_hpc = attn_mma_slab_heads(cfg->n_heads, h->hd, !fused_may_run);
+    }
     if ((st = alloc_weight_set(h, h->wset[0])) != EBRL_OK) return bail(st);
     if ((st = upload_weight_set(h, h->wset[0], wts, nullptr, false)) != EBRL_OK) return bail(st);
     h->wset[0].version = 1;
@@ -1132,7 +1139,7 @@ ebrl_status_t ebrl_actgen_create(const ebrl_actgen_cfg_t *cfg, const ebrl_actgen
                 return bail(EBRL_ERR_NOMEM);
             }
             TensorMap128 self_map;
-            if (attn_mma_make_map(&self_map, s.qkv, rows, 3 * (uint64_t)d, cfg->n_heads, h->hd) ||
+            if (attn_mma_make_map(&self_map, s.qkv, rows, 3 * (uint64_t)d, h->attn_hpc, h->hd) ||
                 cudaMemcpy(s.maps_d, &self_map, sizeof self_map, cudaMemcpyHostToDevice) != cudaSuccess) {
                 fail(h, EBRL_ERR_CUDA, "building the TMA descriptor of the QKV buffer failed");
                 return bail(EBRL_ERR_CUDA);

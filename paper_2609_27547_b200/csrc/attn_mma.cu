@@ -24,8 +24,9 @@ namespace am {
 using namespace ptx;
 
 constexpr int NSTAGE = 3;
-constexpr int MAXW = 8;                 // consumer warps = heads per slab
-constexpr int THREADS = (MAXW + 1) * 32;
+// consumer warps = heads per slab: 8 heads of 128 columns or 16 heads of 64 -- a slab is 1024 columns (16 keys per
+// stage) either way, and the narrower heads, whose softmax costs twice as much per byte, get twice the warps to hide it
+__host__ __device__ constexpr int maxw(int hd) { return hd == 64 ? 16 : 8; }
 constexpr int STAGE_ROWS_BYTES = 32768; // payload bytes of K (and of V) per stage
 
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3)
@@ -79,8 +80,9 @@ __device__ __forceinline__ void quad_transpose(uint32_t (&r)[4], int t)
 }
 
 template <int HD>
-__global__ void __launch_bounds__(THREADS, 1) attn_mma_kernel(AttnArgs a, int hpc, int la_blocks, unsigned long long limit_ns, int *status)
+__global__ void __launch_bounds__((maxw(HD) + 1) * 32, 1) attn_mma_kernel(AttnArgs a, int hpc, int la_blocks, unsigned long long limit_ns, int *status)
 {
+    constexpr int MAXW = maxw(HD);
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int W = hpc * HD;                       // slab width in columns
@@ -370,12 +372,20 @@ __global__ void __launch_bounds__(THREADS, 1) attn_mma_kernel(AttnArgs a, int hp
 
 }  // namespace am
 
+// Heads per slab (= consumer warps that work): as many as the kernel has warps for -- 16 heads of 64 columns or 8 of
+// 128 -- when `wide`; 8 otherwise (the persistent step kernel reads the same descriptors and has 8 attention warps).
+int attn_mma_slab_heads(int n_heads, int hd, bool wide)
+{
+    const int top = wide ? am::maxw(hd) : 8;
+    if (n_heads <= top) return n_heads;
+    if (n_heads % top == 0) return top;
+    return 8;
+}
 // Shapes the kernel covers: bf16, H <= 16, head_dim 64 or 128, heads a multiple of the slab.
 bool attn_mma_supported(int H, int n_heads, int hd)
 {
     if (H > 16 || (hd != 64 && hd != 128)) return false;
-    const int hpc = n_heads < am::MAXW ? n_heads : am::MAXW;
-    return n_heads % hpc == 0;
+    return n_heads % attn_mma_slab_heads(n_heads, hd, false) == 0;
 }
 
 typedef CUresult (*EncodeTiledFn3)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
@@ -384,7 +394,7 @@ typedef CUresult (*EncodeTiledFn3)(CUtensorMap *, CUtensorMapDataType, cuuint32_
 
 // 3-D descriptor of a row-major bf16 matrix [rows][width] seen as (64-column group, row, group
 // index): box = one slab of heads x one stage of keys, 128-byte swizzle, zero fill out of range.
-int attn_mma_make_map(TensorMap128 *out, const void *base, uint64_t rows, uint64_t width, int n_heads, int hd)
+int attn_mma_make_map(TensorMap128 *out, const void *base, uint64_t rows, uint64_t width, int hpc, int hd)
 {
     static EncodeTiledFn3 fn = nullptr;
     if (!fn) {
@@ -393,7 +403,6 @@ int attn_mma_make_map(TensorMap128 *out, const void *base, uint64_t rows, uint64
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess) return 1;
         fn = reinterpret_cast<EncodeTiledFn3>(p);
     }
-    const int hpc = n_heads < am::MAXW ? n_heads : am::MAXW;
     const int W = hpc * hd;
     const cuuint64_t dims[3] = {64, rows, width / 64};
     const cuuint64_t strides[2] = {width * 2, 128};
@@ -405,24 +414,23 @@ int attn_mma_make_map(TensorMap128 *out, const void *base, uint64_t rows, uint64
     return r == CUDA_SUCCESS ? 0 : 2;
 }
 
-// la = L2 look-ahead of the producer in key blocks (0 disables).
-cudaError_t launch_attn_mma(const AttnArgs &a, int grid, int la, unsigned long long limit_ns, int *status, cudaStream_t st)
+// hpc = heads per slab, as in the descriptors; la = L2 look-ahead of the producer in key blocks (0 disables).
+cudaError_t launch_attn_mma(const AttnArgs &a, int grid, int hpc, int la, unsigned long long limit_ns, int *status, cudaStream_t st)
 {
-    const int hpc = a.n_heads < am::MAXW ? a.n_heads : am::MAXW;
     const int items = a.n_envs * (a.n_heads / hpc);
     if (items == 0) return cudaSuccess;
     const int g = items < grid ? items : grid;
     const int W = hpc * a.hd;
-    const size_t smem = (size_t)2 * am::NSTAGE * am::stage_keys(W) * (W / 64) * 128 + (size_t)am::MAXW * 16 * a.hd * 2 + 64 + 1024;
+    const size_t smem = (size_t)2 * am::NSTAGE * am::stage_keys(W) * (W / 64) * 128 + (size_t)am::maxw(a.hd) * 16 * a.hd * 2 + 64 + 1024;
     cudaError_t e;
     if (a.hd == 128) {
         e = cudaFuncSetAttribute(am::attn_mma_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        return launch_kernel(am::attn_mma_kernel<128>, g, am::THREADS, smem, st, 1, a, hpc, la, limit_ns, status);
+        return launch_kernel(am::attn_mma_kernel<128>, g, (am::maxw(128) + 1) * 32, smem, st, 1, a, hpc, la, limit_ns, status);
     } else {
         e = cudaFuncSetAttribute(am::attn_mma_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        return launch_kernel(am::attn_mma_kernel<64>, g, am::THREADS, smem, st, 1, a, hpc, la, limit_ns, status);
+        return launch_kernel(am::attn_mma_kernel<64>, g, (am::maxw(64) + 1) * 32, smem, st, 1, a, hpc, la, limit_ns, status);
     }
     return cudaGetLastError();
 }
